@@ -1,0 +1,260 @@
+/*
+ * CPU oracle for the SLiM compressed linear layer.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, plain, fp64 statement of what the GPU library must
+ * compute.  It is used by the tests, by the smoke check and by the timed CPU
+ * baseline of the benchmark; the product path never links, imports or calls
+ * it, and it shares no code, header, table or helper with the CUDA sources.
+ *
+ * What it states (paper sections in brackets):
+ *   - the layer output  Y = X W  with the compressed weight plus low-rank
+ *     adapters,  W ~ W^C + L R              [Sec. 2 "Model Compression", Eq. 1;
+ *                                            Sec. 3.2 "SLiM-LoRA"]
+ *   - W^C is a symmetric uniform 4-bit quantized matrix with one scale per
+ *     tensor                                [Sec. 3.1, Eq. 2 and Eq. 5]
+ *   - pruned to the 2:4 pattern (at most two kept values in every aligned
+ *     group of four along the contraction axis)         [Sec. 1, Sec. 3.2]
+ *   - the adapter product costs O(2 b r d^2) and is added to the sparse
+ *     product                                [App. "Rank Analysis"]
+ *
+ * Layout convention (nn.Linear orientation, i.e. the transpose of the paper's
+ * W in R^{d_in x d_out}):  Q[d_out][d_in] int4 codes, mask[d_out][d_in],
+ * L[d_out][r] (= paper R^T), R[r][d_in] (= paper L^T), X[b][d_in], Y[b][d_out]:
+ *     Y[m][n] = sum_k X[m][k] * s*Q[n][k]*mask[n][k]
+ *             + sum_j ( sum_k X[m][k]*R[j][k] ) * L[n][j]
+ *
+ * The packed storage format is not given by the paper (it delegates storage
+ * to a third-party kernel); the format below is this project's definition:
+ *   vals[n][g]  (one byte per group g of four columns): low nibble = code at
+ *               the lower kept position, high nibble = code at the upper one,
+ *               two's complement;
+ *   meta[n][g/2] (one nibble per group): bits 0-1 = lower kept position,
+ *               bits 2-3 = upper kept position; even g in the low nibble.
+ *   A group with fewer than two kept positions is completed with the lowest
+ *   positions not already kept (their codes are stored as 0) and the pair is
+ *   sorted ascending.  More than two kept positions is an error.
+ *
+ * Every function here is pinned by tests/test_oracle_pins.py against values
+ * that do not come from this file (hand-computed bytes and sums, an
+ * independent float64 matrix product, closed forms, invariants).
+ */
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ORACLE_OK = 0, ORACLE_BAD_ARG = 1, ORACLE_BAD_MASK = 3, ORACLE_CODE_RANGE = 4 };
+
+/* bfloat16 (upper half of an IEEE binary32) to double: exact. */
+static double bf16_to_double(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Sign-extend a 4-bit two's-complement nibble. */
+static int sext4(unsigned nib)
+{
+    nib &= 0xFu;
+    return (nib & 0x8u) ? (int)nib - 16 : (int)nib;
+}
+
+/*
+ * Pack int4 codes and a 2:4 mask into nibble values and 2-bit position
+ * metadata [format defined in the header comment; 2:4 pattern: Sec. 1].
+ * codes, mask: [d_out][d_in] row-major.  vals: [d_out][d_in/4].
+ * meta: [d_out][d_in/8].  d_in must be a multiple of 8.
+ * Returns ORACLE_OK, or the first error found; on error, *bad_row / *bad_group
+ * (if non-NULL) identify the offending group.
+ */
+int oracle_pack(const int8_t *codes, const uint8_t *mask, int d_out, int d_in,
+                uint8_t *vals, uint8_t *meta, int *bad_row, int *bad_group)
+{
+    if (!codes || !mask || !vals || !meta || d_out < 1 || d_in < 8 || d_in % 8 != 0)
+        return ORACLE_BAD_ARG;
+    const int groups = d_in / 4;
+    memset(meta, 0, (size_t)d_out * (size_t)(d_in / 8));
+    for (int n = 0; n < d_out; ++n) {
+        for (int g = 0; g < groups; ++g) {
+            const int8_t *c = codes + (size_t)n * d_in + 4 * g;
+            const uint8_t *mk = mask + (size_t)n * d_in + 4 * g;
+            int keep[4] = {0, 0, 0, 0};
+            int kept = 0;
+            for (int i = 0; i < 4; ++i)
+                if (mk[i]) { keep[i] = 1; ++kept; }
+            if (kept > 2) {
+                if (bad_row) *bad_row = n;
+                if (bad_group) *bad_group = g;
+                return ORACLE_BAD_MASK;
+            }
+            /* complete the pair with the lowest positions not kept; those
+               slots carry the value 0 */
+            int real[4] = {keep[0], keep[1], keep[2], keep[3]};
+            for (int i = 0; i < 4 && kept < 2; ++i)
+                if (!keep[i]) { keep[i] = 1; ++kept; }
+            int pos[2], np = 0;
+            for (int i = 0; i < 4; ++i)
+                if (keep[i]) pos[np++] = i;          /* ascending */
+            int v[2];
+            for (int e = 0; e < 2; ++e) {
+                if (real[pos[e]]) {
+                    int code = c[pos[e]];
+                    if (code < -8 || code > 7) {
+                        if (bad_row) *bad_row = n;
+                        if (bad_group) *bad_group = g;
+                        return ORACLE_CODE_RANGE;
+                    }
+                    v[e] = code;
+                } else {
+                    v[e] = 0;
+                }
+            }
+            vals[(size_t)n * groups + g] =
+                (uint8_t)(((unsigned)v[0] & 0xFu) | (((unsigned)v[1] & 0xFu) << 4));
+            unsigned m = (unsigned)pos[0] | ((unsigned)pos[1] << 2);
+            meta[(size_t)n * (d_in / 8) + (g >> 1)] |= (uint8_t)(m << (4 * (g & 1)));
+        }
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * Inverse of oracle_pack: dense int8 codes (0 where nothing is stored) and a
+ * mask holding 1 at the two stored positions of every group.
+ */
+int oracle_unpack(const uint8_t *vals, const uint8_t *meta, int d_out, int d_in,
+                  int8_t *codes, uint8_t *mask)
+{
+    if (!vals || !meta || !codes || d_out < 1 || d_in < 8 || d_in % 8 != 0)
+        return ORACLE_BAD_ARG;
+    const int groups = d_in / 4;
+    for (int n = 0; n < d_out; ++n) {
+        for (int g = 0; g < groups; ++g) {
+            unsigned vb = vals[(size_t)n * groups + g];
+            unsigned mb = meta[(size_t)n * (d_in / 8) + (g >> 1)];
+            unsigned m = (mb >> (4 * (g & 1))) & 0xFu;
+            int p0 = (int)(m & 3u), p1 = (int)((m >> 2) & 3u);
+            int8_t *c = codes + (size_t)n * d_in + 4 * g;
+            c[0] = c[1] = c[2] = c[3] = 0;
+            if (mask) {
+                uint8_t *mk = mask + (size_t)n * d_in + 4 * g;
+                mk[0] = mk[1] = mk[2] = mk[3] = 0;
+                mk[p0] = 1;
+                mk[p1] = 1;
+            }
+            c[p0] = (int8_t)sext4(vb & 0xFu);
+            c[p1] = (int8_t)sext4(vb >> 4);   /* p0 == p1 cannot come from oracle_pack */
+        }
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * Factored forward  Y = X (s Q)^T + (X R^T) L^T  in fp64, dense loops over the
+ * whole contraction axis (the zeros of the 2:4 pattern are multiplied, not
+ * skipped), no intermediate rounding  [Sec. 2 Eq. 1; Sec. 3.2; App. Rank
+ * Analysis].  X, L, R are bfloat16 bit patterns.  Y is double [b][d_out].
+ * rows: optional list of n_rows token indices to evaluate (NULL = all b rows,
+ * in which case n_rows is ignored); Y then has n_rows rows in list order.
+ */
+int oracle_linear_fwd(const uint16_t *X, int b, const uint8_t *vals, const uint8_t *meta,
+                      float s, const uint16_t *L, const uint16_t *R, int r,
+                      int d_out, int d_in, const int32_t *rows, int n_rows, double *Y)
+{
+    if (!X || !vals || !meta || !Y || b < 1 || d_out < 1 || d_in < 8 || d_in % 8 != 0 || r < 0)
+        return ORACLE_BAD_ARG;
+    if (r > 0 && (!L || !R)) return ORACLE_BAD_ARG;
+    const int nm = rows ? n_rows : b;
+    int8_t *Wd = (int8_t *)malloc((size_t)d_out * d_in);
+    if (!Wd) return ORACLE_BAD_ARG;
+    int rc = oracle_unpack(vals, meta, d_out, d_in, Wd, NULL);
+    if (rc != ORACLE_OK) { free(Wd); return rc; }
+    const double sd = (double)s;
+#pragma omp parallel for schedule(static)
+    for (int mi = 0; mi < nm; ++mi) {
+        const int m = rows ? rows[mi] : mi;
+        double *xrow = (double *)malloc(sizeof(double) * (size_t)d_in);
+        double *t = (double *)malloc(sizeof(double) * (size_t)(r > 0 ? r : 1));
+        for (int k = 0; k < d_in; ++k) xrow[k] = bf16_to_double(X[(size_t)m * d_in + k]);
+        for (int j = 0; j < r; ++j) {
+            double acc = 0.0;
+            for (int k = 0; k < d_in; ++k) acc += xrow[k] * bf16_to_double(R[(size_t)j * d_in + k]);
+            t[j] = acc;
+        }
+        for (int n = 0; n < d_out; ++n) {
+            double acc = 0.0;
+            for (int k = 0; k < d_in; ++k) acc += xrow[k] * (sd * (double)Wd[(size_t)n * d_in + k]);
+            double lr = 0.0;
+            for (int j = 0; j < r; ++j) lr += t[j] * bf16_to_double(L[(size_t)n * r + j]);
+            Y[(size_t)mi * d_out + n] = acc + lr;
+        }
+        free(xrow);
+        free(t);
+    }
+    free(Wd);
+    return ORACLE_OK;
+}
+
+/*
+ * Dense form of the same layer: builds W_eff = s Q + L R explicitly
+ * ([d_out][d_in], fp64) and returns Y = X W_eff^T  [Sec. 3.2: W ~ W^C + L R].
+ * Used to check the factored routine against the unfactored definition.
+ * W_eff_out (optional, [d_out][d_in]) receives the dense matrix.
+ */
+int oracle_linear_fwd_dense(const uint16_t *X, int b, const uint8_t *vals, const uint8_t *meta,
+                            float s, const uint16_t *L, const uint16_t *R, int r,
+                            int d_out, int d_in, double *Y, double *W_eff_out)
+{
+    if (!X || !vals || !meta || !Y || b < 1 || d_out < 1 || d_in < 8 || d_in % 8 != 0 || r < 0)
+        return ORACLE_BAD_ARG;
+    if (r > 0 && (!L || !R)) return ORACLE_BAD_ARG;
+    int8_t *Wd = (int8_t *)malloc((size_t)d_out * d_in);
+    double *We = (double *)malloc(sizeof(double) * (size_t)d_out * d_in);
+    if (!Wd || !We) { free(Wd); free(We); return ORACLE_BAD_ARG; }
+    int rc = oracle_unpack(vals, meta, d_out, d_in, Wd, NULL);
+    if (rc != ORACLE_OK) { free(Wd); free(We); return rc; }
+    const double sd = (double)s;
+    for (int n = 0; n < d_out; ++n)
+        for (int k = 0; k < d_in; ++k) {
+            double w = sd * (double)Wd[(size_t)n * d_in + k];
+            for (int j = 0; j < r; ++j)
+                w += bf16_to_double(L[(size_t)n * r + j]) * bf16_to_double(R[(size_t)j * d_in + k]);
+            We[(size_t)n * d_in + k] = w;
+        }
+    for (int m = 0; m < b; ++m)
+        for (int n = 0; n < d_out; ++n) {
+            double acc = 0.0;
+            for (int k = 0; k < d_in; ++k)
+                acc += bf16_to_double(X[(size_t)m * d_in + k]) * We[(size_t)n * d_in + k];
+            Y[(size_t)m * d_out + n] = acc;
+        }
+    if (W_eff_out) memcpy(W_eff_out, We, sizeof(double) * (size_t)d_out * d_in);
+    free(Wd);
+    free(We);
+    return ORACLE_OK;
+}
+
+/*
+ * Inference FLOP-reduction ratio of a compressed transformer
+ * [App. "Computation Reduction Analysis", Eq. 13]: dense over compressed flop
+ * count for n blocks of hidden size d, feed-forward ratio a, vocabulary V,
+ * 2:4 sparsity on every block linear and adapters of rank ratio rr (0 = none).
+ * The batch size cancels.
+ */
+double oracle_flop_reduction(double d, double n, double a, double V, double rr)
+{
+    double dense = n * (4.0 * d * d + 2.0 * d * d * a) + d * V;
+    double comp = n * (4.0 * d * d / 2.0 + 4.0 * 2.0 * d * d * rr + 2.0 * d * d * a / 2.0 +
+                       2.0 * (d * d * rr + d * d * rr * a)) + d * V;
+    return dense / comp;
+}
+
+/* Number of OpenMP threads oracle_linear_fwd will use (1 without OpenMP). */
+#ifdef _OPENMP
+#include <omp.h>
+int oracle_num_threads(void) { return omp_get_max_threads(); }
+#else
+int oracle_num_threads(void) { return 1; }
+#endif

@@ -1,0 +1,220 @@
+"""Pins for the CPU oracle: every expected value here comes from outside
+oracle/ (hand arithmetic, numpy's own float64 matmul, integer arithmetic, the
+paper's printed table, invariants)."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2410_09615_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf(x):
+    return inputs.f32_to_bf16_bits(np.asarray(x, np.float32))
+
+
+# ---------------------------------------------------------------- P4: by hand
+HAND_CODES = np.array([[3, -2, 0, 5, -8, 7, 1, 0],
+                       [-1, -8, 4, 2, 6, 0, 0, -3]], np.int8)
+HAND_MASK = np.array([[1, 0, 0, 1, 0, 1, 1, 0],
+                      [0, 1, 1, 0, 0, 0, 0, 1]], np.uint8)
+
+
+def test_pack_bytes_by_hand():
+    vals, meta = oracle.pack(HAND_CODES, HAND_MASK)
+    # row 0: group 0 keeps positions (0,3) codes (3,5)   -> 0x53, index nibble 0|3<<2 = 0xC
+    #        group 1 keeps positions (1,2) codes (7,1)   -> 0x17, index nibble 1|2<<2 = 0x9
+    # row 1: group 0 keeps positions (1,2) codes (-8,4)  -> 0x48, 0x9
+    #        group 1 keeps only position 3 (code -3): completed with position 0 (value 0)
+    #                 -> positions (0,3) codes (0,-3)    -> 0xD0, 0xC
+    assert vals.tolist() == [[0x53, 0x17], [0x48, 0xD0]]
+    assert meta.tolist() == [[0x9C], [0xC9]]
+
+
+def test_unpack_by_hand():
+    vals = np.array([[0x53, 0x17], [0x48, 0xD0]], np.uint8)
+    meta = np.array([[0x9C], [0xC9]], np.uint8)
+    codes, mask = oracle.unpack(vals, meta)
+    assert codes.tolist() == [[3, 0, 0, 5, 0, 7, 1, 0], [0, -8, 4, 0, 0, 0, 0, -3]]
+    assert mask.tolist() == [[1, 0, 0, 1, 0, 1, 1, 0], [0, 1, 1, 0, 1, 0, 0, 1]]
+
+
+def test_forward_by_hand():
+    vals, meta = oracle.pack(HAND_CODES, HAND_MASK)
+    X = bf([[1, 2, -1, 0.5, 3, -2, 4, 1]])
+    R = bf([[0.5, 0, 0, 1, 0, 0, 0.25, 2]])
+    L = bf([[1.5], [-0.5]])
+    # row 0 of the kept weight: [3,0,0,5,0,7,1,0] . x = 3 + 2.5 - 14 + 4 = -4.5 ; * 0.5 = -2.25
+    # row 1:                    [0,-8,4,0,0,0,0,-3] . x = -16 - 4 - 3 = -23    ; * 0.5 = -11.5
+    # t = R . x = 0.5 + 0.5 + 1 + 2 = 4 ; adapters add 1.5*4 = 6 and -0.5*4 = -2
+    Y = oracle.linear_fwd(X, vals, meta, 0.5, L, R)
+    assert Y.tolist() == [[3.75, -13.5]]
+    Yd = oracle.linear_fwd_dense(X, vals, meta, 0.5, L, R)
+    assert Yd.tolist() == [[3.75, -13.5]]
+    # without adapters only the sparse term remains
+    assert oracle.linear_fwd(X, vals, meta, 0.5, None, None).tolist() == [[-2.25, -11.5]]
+
+
+# ------------------------------------------------------- P1/P2: structure
+def random_codes_mask(rng, d_out, d_in, kept_choices=(0, 1, 2)):
+    codes = rng.integers(-8, 8, size=(d_out, d_in)).astype(np.int8)
+    mask = np.zeros((d_out, d_in // 4, 4), np.uint8)
+    kept = rng.choice(kept_choices, size=(d_out, d_in // 4))
+    for n in range(d_out):
+        for g in range(d_in // 4):
+            pos = rng.permutation(4)[: kept[n, g]]
+            mask[n, g, pos] = 1
+    return codes, mask.reshape(d_out, d_in)
+
+
+def test_round_trip_and_invariants():
+    rng = np.random.default_rng(1)
+    codes, mask = random_codes_mask(rng, 24, 64)
+    # make sure -8, 0-at-kept-slot and every group population occur
+    codes[0, :4] = [-8, 0, -8, 0]
+    mask[0, :4] = [1, 1, 0, 0]
+    vals, meta = oracle.pack(codes, mask)
+    assert vals.shape == (24, 16) and meta.shape == (24, 8)
+    c2, m2 = oracle.unpack(vals, meta)
+    kept = mask.astype(bool)
+    # stored positions are a superset of the kept ones, exactly two per group
+    assert (m2.reshape(24, 16, 4).sum(-1) == 2).all()
+    assert (m2.astype(bool) | ~kept).all()
+    assert (c2 == np.where(kept, codes, 0)).all()
+    # 2:4 invariant on the decoded weight
+    assert ((c2.reshape(24, 16, 4) != 0).sum(-1) <= 2).all()
+    # every index nibble is an ascending pair i0 < i1
+    nib = np.stack([meta & 0xF, meta >> 4], -1).reshape(24, 16)
+    assert set(np.unique(nib).tolist()) <= {0x4, 0x8, 0xC, 0x9, 0xD, 0xE}
+    assert ((nib & 3) < (nib >> 2)).all()
+    # packing is idempotent on its own output
+    v3, t3 = oracle.pack(c2, m2)
+    assert (v3 == vals).all() and (t3 == meta).all()
+
+
+def test_pack_layout_one_hot():
+    """A single kept weight lands in exactly one nibble whose place follows the format."""
+    d_out, d_in = 3, 32
+    for n, k, code in [(0, 0, 5), (1, 7, -8), (2, 30, -1), (1, 17, 7)]:
+        codes = np.zeros((d_out, d_in), np.int8)
+        mask = np.zeros((d_out, d_in), np.uint8)
+        codes[n, k] = code
+        mask[n, k] = 1
+        vals, meta = oracle.pack(codes, mask)
+        g, i = divmod(k, 4)
+        # the group is completed with the lowest other position
+        other = 0 if i != 0 else 1
+        p0, p1 = sorted((i, other))
+        exp_v = np.zeros_like(vals)
+        exp_v[n, g] = (code & 0xF) << (0 if p0 == i else 4)
+        assert (vals == exp_v).all()
+        got = (int(meta[n, g // 2]) >> (4 * (g % 2))) & 0xF
+        assert got == (p0 | (p1 << 2))
+        # all other groups hold the default pair (0,1) = 0x4
+        m_all = np.stack([meta & 0xF, meta >> 4], -1).reshape(d_out, d_in // 4)
+        m_all[n, g] = 0x4
+        assert (m_all == 0x4).all()
+
+
+def test_pack_errors():
+    codes = np.zeros((2, 8), np.int8)
+    mask = np.zeros((2, 8), np.uint8)
+    mask[1, 4:7] = 1
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.pack(codes, mask)
+    assert e.value.code == oracle.BAD_MASK and (e.value.row, e.value.group) == (1, 1)
+    mask[:] = 0
+    mask[0, 2] = 1
+    codes[0, 2] = 9
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.pack(codes, mask)
+    assert e.value.code == oracle.CODE_RANGE and (e.value.row, e.value.group) == (0, 0)
+    # out-of-range codes at pruned positions are ignored
+    mask[:] = 0
+    vals, meta = oracle.pack(codes, mask)
+    assert (vals == 0).all()
+
+
+# ------------------------------------- P3/P5: identity and independent matmul
+@pytest.mark.parametrize("d_in,d_out,r,b", [(64, 48, 16, 5), (128, 32, 48, 3), (32, 80, 0, 4)])
+def test_forward_matches_numpy_float64(d_in, d_out, r, b):
+    ly = inputs.make_layer(d_in, d_out, r, b, seed=7)
+    vals, meta = oracle.pack(ly.codes, ly.mask)
+    Y = oracle.linear_fwd(ly.X, vals, meta, ly.s, ly.L, ly.R)
+    # independent restatement with numpy's float64 matmul from the *unpacked inputs*
+    Wc = np.float64(np.float32(ly.s)) * (ly.codes.astype(np.float64) * ly.mask)
+    Xf = inputs.bf16_bits_to_f64(ly.X)
+    if r:
+        W_eff = Wc + inputs.bf16_bits_to_f64(ly.L) @ inputs.bf16_bits_to_f64(ly.R)
+    else:
+        W_eff = Wc
+    Yn = Xf @ W_eff.T
+    scale = np.abs(Yn).max()
+    assert np.abs(Y - Yn).max() <= 1e-12 * scale
+    Yd, We = oracle.linear_fwd_dense(ly.X, vals, meta, ly.s, ly.L, ly.R, return_weight=True)
+    assert np.abs(Yd - Yn).max() <= 1e-12 * scale
+    assert np.abs(We - W_eff).max() <= 1e-15
+    # a row subset equals the same rows of the full result, in list order
+    rows = [b - 1, 0]
+    Ys = oracle.linear_fwd(ly.X, vals, meta, ly.s, ly.L, ly.R, rows=rows)
+    assert (Ys == Y[rows]).all()
+
+
+# ----------------------------------------------------- P6: integer-exact case
+def test_forward_integer_exact():
+    rng = np.random.default_rng(3)
+    d_in, d_out, r, b = 96, 40, 16, 6
+    codes, mask = random_codes_mask(rng, d_out, d_in)
+    vals, meta = oracle.pack(codes, mask)
+    Xi = rng.integers(-4, 5, size=(b, d_in))
+    Li = rng.integers(-2, 3, size=(d_out, r))
+    Ri = rng.integers(-2, 3, size=(r, d_in))
+    Y = oracle.linear_fwd(bf(Xi), vals, meta, 1.0, bf(Li), bf(Ri))
+    Wi = codes.astype(np.int64) * mask
+    exact = Xi @ Wi.T + (Xi @ Ri.T) @ Li.T       # int64 arithmetic
+    assert (Y == exact.astype(np.float64)).all()
+
+
+def test_one_hot_activations_read_weight_columns():
+    rng = np.random.default_rng(4)
+    d_in, d_out = 32, 24
+    codes, mask = random_codes_mask(rng, d_out, d_in, kept_choices=(2,))
+    vals, meta = oracle.pack(codes, mask)
+    X = np.eye(d_in, dtype=np.float32)
+    Y = oracle.linear_fwd(bf(X), vals, meta, 0.25, None, None)
+    assert (Y == 0.25 * (codes.astype(np.float64) * mask).T).all()
+
+
+# ------------------------------------------------- P8: degenerate reductions
+def test_degenerate_cases():
+    ly = inputs.make_layer(64, 32, 16, 4, seed=11)
+    vals, meta = oracle.pack(ly.codes, ly.mask)
+    Xf = inputs.bf16_bits_to_f64(ly.X)
+    Lf, Rf = inputs.bf16_bits_to_f64(ly.L), inputs.bf16_bits_to_f64(ly.R)
+    full = oracle.linear_fwd(ly.X, vals, meta, ly.s, ly.L, ly.R)
+    sparse_only = oracle.linear_fwd(ly.X, vals, meta, ly.s, None, None)
+    # zero weight -> pure low-rank term
+    zv, zm = oracle.pack(np.zeros_like(ly.codes), np.zeros_like(ly.mask))
+    lowrank = oracle.linear_fwd(ly.X, zv, zm, ly.s, ly.L, ly.R)
+    assert np.abs(lowrank - (Xf @ Rf.T) @ Lf.T).max() <= 1e-13
+    assert np.abs(full - (sparse_only + lowrank)).max() <= 1e-12
+    # doubling s doubles only the sparse term (2*s is exact in fp32)
+    doubled = oracle.linear_fwd(ly.X, vals, meta, 2 * ly.s, ly.L, ly.R)
+    assert np.abs(doubled - (2 * sparse_only + lowrank)).max() <= 1e-12
+    # zero adapters equal no adapters
+    z = oracle.linear_fwd(ly.X, vals, meta, ly.s, np.zeros_like(ly.L), np.zeros_like(ly.R))
+    assert (z == sparse_only).all()
+
+
+# ---------------------------------------- P7: the paper's printed FLOP table
+def test_flop_reduction_matches_printed_table():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "flop_reduction_table.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert len(rows) == 4
+    for _name, d, n, dff, V, rr, printed in rows:
+        d, n, dff, V, rr, printed = int(d), int(n), int(dff), int(V), float(rr), float(printed)
+        got = oracle.flop_reduction(d, n, dff / d, V, rr)
+        assert abs(got - printed) <= 0.005 + 1e-9, (got, printed)
