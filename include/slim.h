@@ -1,0 +1,160 @@
+/*
+ * libslim — the SLiM compressed linear layer on NVIDIA B200 (sm_100a).
+ *
+ *     Y = X (s Q)^T + (X R^T) L^T
+ *
+ * Q holds symmetric-uniform 4-bit integer codes with one scale s per tensor
+ * (paper Sec. 3.1, Eq. 2 / Eq. 5), pruned to the 2:4 pattern: at most two kept
+ * values in every aligned group of four along d_in (Sec. 1, Sec. 3.2).  L and R
+ * are the rank-r adapters that correct the compression error, W ~ W^C + L R
+ * (Sec. 3.2); the layer output is Y = X W (Sec. 2, Eq. 1) and the adapter product
+ * is evaluated factored, at O(2 b r d^2) cost (App. "Rank Analysis").
+ *
+ * Orientation (nn.Linear, the transpose of the paper's W in R^{d_in x d_out}):
+ *   X [b, d_in]  bf16 row-major          activations, b tokens
+ *   Q [d_out, d_in] int4 codes           row n = output feature n
+ *   L [d_out, r] bf16 row-major          (the paper's right adapter, transposed)
+ *   R [r, d_in]  bf16 row-major          (the paper's left adapter, transposed)
+ *   Y [b, d_out] bf16 row-major
+ *
+ * Packed weight (the paper leaves storage to a third-party kernel; this is the
+ * library's own format):
+ *   vals [d_out, d_in/4] u8   one byte per group of four columns: low nibble =
+ *                             code at the lower stored position, high nibble =
+ *                             code at the upper one (two's complement)
+ *   meta [d_out, d_in/8] u8   one nibble per group: bits 0-1 lower position,
+ *                             bits 2-3 upper position (lower < upper); even
+ *                             groups in the low nibble of a byte
+ *   A group with fewer than two kept positions is completed with the lowest
+ *   positions not kept, stored with value 0.
+ *
+ * General rules for every call:
+ *   - Every data pointer is a DEVICE pointer owned by the caller and must be
+ *     16-byte aligned; the library allocates no device memory and keeps no
+ *     state besides a per-device attribute cache.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *     the default stream) and the call returns without synchronising.
+ *   - The return value reports errors the host can see (bad arguments,
+ *     unsupported shape or device, a failed launch).  Errors found on the
+ *     device (a 2:4 group with more than two kept values, a code outside
+ *     [-8, 7], a bounded wait that expired) are OR-ed as bits
+ *     (1u << slim_status_t) into *status_dev, a device uint32 the caller
+ *     zeroes and reads back; status_dev may be NULL.  Nothing traps.
+ */
+#ifndef SLIM_H
+#define SLIM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SLIM_OK = 0,
+    SLIM_ERR_INVALID_ARG = 1,        /* null / misaligned pointer, b < 1, negative size */
+    SLIM_ERR_UNSUPPORTED_SHAPE = 2,  /* d_in % 64, d_out % 16 or r % 16 not zero */
+    SLIM_ERR_BAD_MASK = 3,           /* device: more than two kept values in a group */
+    SLIM_ERR_CODE_RANGE = 4,         /* device: kept code outside [-8, 7] */
+    SLIM_ERR_WORKSPACE = 5,          /* workspace NULL or smaller than slim_workspace_bytes */
+    SLIM_ERR_CUDA = 6,               /* a CUDA runtime call or launch failed */
+    SLIM_ERR_TIMEOUT = 7,            /* device: a bounded wait expired */
+    SLIM_ERR_ARCH = 8                /* current device is not compute capability 10.x */
+} slim_status_t;
+
+/* Kernel families the dispatcher chooses from (slim_linear_fwd_ex). */
+typedef enum {
+    SLIM_KERNEL_AUTO = 0,    /* by batch size: decode for b <= 16, prefill above */
+    SLIM_KERNEL_SIMPLE = 1,  /* CUDA-core kernel, any legal shape; correctness anchor */
+    SLIM_KERNEL_DECODE = 2,  /* streaming sparse tensor-core kernel for small batches */
+    SLIM_KERNEL_PREFILL = 3  /* tcgen05 sparse tensor-core kernel for many tokens */
+} slim_kernel_t;
+
+/*
+ * Pack int4 codes and a 2:4 mask into `vals` and `meta` (format above; 2:4
+ * pattern: Sec. 1; 4-bit symmetric codes: Sec. 3.1 Eq. 2).  Integer-only and
+ * bit-exact.
+ *   codes [d_out, d_in] int8, values in [-8, 7] at kept positions (others ignored)
+ *   mask  [d_out, d_in] u8, non-zero = kept
+ *   vals  [d_out, d_in/4] u8 (out),  meta [d_out, d_in/8] u8 (out)
+ * d_in must be a multiple of 64.  Groups that violate the 2:4 pattern or hold an
+ * out-of-range code are written as zeros (value 0x00, index nibble 0x4) and
+ * flagged in *status_dev.
+ */
+slim_status_t slim_pack(const int8_t* codes, const uint8_t* mask, int d_out, int d_in,
+                        uint8_t* vals, uint8_t* meta, uint32_t* status_dev, void* cuda_stream);
+
+/*
+ * Inverse of slim_pack: dense int8 codes (0 where nothing is stored) and a mask
+ * holding 1 at the two stored positions of every group.  `mask` may be NULL.
+ */
+slim_status_t slim_unpack(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in,
+                          int8_t* codes, uint8_t* mask, void* cuda_stream);
+
+/*
+ * Bytes of device scratch slim_linear_fwd needs for this problem (split-K
+ * partial sums, the adapter intermediate T = X R^T, and synchronisation words).
+ * Returns 0 for illegal arguments.  The first SLIM_WORKSPACE_SYNC_BYTES bytes
+ * hold counters that must be zero before the first call that uses the buffer
+ * (slim_workspace_reset does that); each call leaves them zero again unless it
+ * reported SLIM_ERR_TIMEOUT.  Calls that share a workspace must not overlap
+ * on the GPU.
+ */
+#define SLIM_WORKSPACE_SYNC_BYTES 256
+size_t slim_workspace_bytes(int b, int d_out, int d_in, int r);
+
+/* Zero the synchronisation words of a workspace (asynchronous, on the stream). */
+slim_status_t slim_workspace_reset(void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The layer forward (Sec. 2 Eq. 1 with W ~ W^C + L R, Sec. 3.2; factored
+ * adapter product, App. "Rank Analysis"):
+ *     Y[m][n] = s * sum_k X[m][k] Q[n][k]  +  sum_j (sum_k X[m][k] R[j][k]) L[n][j]
+ * Products are bf16 x bf16 accumulated in fp32; the intermediate T = X R^T may
+ * be rounded once to bf16; Y is rounded to bf16 (nearest even).
+ *   X [b, d_in] bf16, vals/meta as produced by slim_pack, s fp32 scale,
+ *   L [d_out, r] bf16, R [r, d_in] bf16 (both NULL iff r == 0), Y [b, d_out] bf16 (out).
+ * Shape rules: b >= 1, d_in % 64 == 0, d_out % 16 == 0, r % 16 == 0.
+ * The kernel is chosen from b: the streaming decode kernel for b <= 16, the
+ * tcgen05 prefill kernel above.
+ */
+slim_status_t slim_linear_fwd(const void* X, int b, const uint8_t* vals, const uint8_t* meta,
+                              float s, const void* L, const void* R, int r, int d_out, int d_in,
+                              void* Y, void* workspace, size_t workspace_bytes,
+                              uint32_t* status_dev, void* cuda_stream);
+
+/* Same operation with the kernel family forced (tests, benchmarks). */
+slim_status_t slim_linear_fwd_ex(const void* X, int b, const uint8_t* vals, const uint8_t* meta,
+                                 float s, const void* L, const void* R, int r, int d_out, int d_in,
+                                 void* Y, void* workspace, size_t workspace_bytes,
+                                 uint32_t* status_dev, void* cuda_stream, slim_kernel_t kernel);
+
+/*
+ * Host-buffer form of the same operation, for callers whose activations live
+ * in host memory: X_host and Y_host are HOST pointers (pinned memory gives
+ * asynchronous copies; no alignment rule); the packed weight, the adapters and
+ * the workspace stay DEVICE pointers (weights are resident, activations
+ * travel).  Copies X in, runs slim_linear_fwd, copies Y out, all on
+ * `cuda_stream`, and synchronises that stream before returning.  x_dev / y_dev
+ * are caller-owned device staging buffers of b*d_in and b*d_out bf16 elements.
+ */
+slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* vals,
+                                   const uint8_t* meta, float s, const void* L, const void* R,
+                                   int r, int d_out, int d_in, void* Y_host, void* x_dev,
+                                   void* y_dev, void* workspace, size_t workspace_bytes,
+                                   uint32_t* status_dev, void* cuda_stream);
+
+/* The kernel family slim_linear_fwd would pick for this problem. */
+slim_kernel_t slim_select_kernel(int b, int d_out, int d_in, int r);
+
+/* Number of kernels the last slim_linear_fwd* call on this host thread launched. */
+int slim_last_launch_count(void);
+
+const char* slim_strerror(slim_status_t status);
+const char* slim_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLIM_H */

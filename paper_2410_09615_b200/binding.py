@@ -1,0 +1,194 @@
+"""ctypes binding of ``libslim.so`` with the same names as ``include/slim.h``.
+
+Argument marshalling only: tensors are torch CUDA tensors (torch supplies device
+memory and streams), every step of the computation runs in the library's
+kernels.  If the library is missing or a call fails, a :class:`SlimError` is
+raised; there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libslim.so")
+
+(SLIM_OK, SLIM_ERR_INVALID_ARG, SLIM_ERR_UNSUPPORTED_SHAPE, SLIM_ERR_BAD_MASK, SLIM_ERR_CODE_RANGE,
+ SLIM_ERR_WORKSPACE, SLIM_ERR_CUDA, SLIM_ERR_TIMEOUT, SLIM_ERR_ARCH) = range(9)
+KERNEL_AUTO, KERNEL_SIMPLE, KERNEL_DECODE, KERNEL_PREFILL = range(4)
+KERNEL_NAMES = {KERNEL_AUTO: "auto", KERNEL_SIMPLE: "simple", KERNEL_DECODE: "decode", KERNEL_PREFILL: "prefill"}
+WORKSPACE_SYNC_BYTES = 256
+
+# every symbol include/slim.h declares, with (restype, argtypes)
+_P, _I, _F, _SZ = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+SIGNATURES = {
+    "slim_pack": (_I, [_P, _P, _I, _I, _P, _P, _P, _P]),
+    "slim_unpack": (_I, [_P, _P, _I, _I, _P, _P, _P]),
+    "slim_workspace_bytes": (_SZ, [_I, _I, _I, _I]),
+    "slim_workspace_reset": (_I, [_P, _SZ, _P]),
+    "slim_linear_fwd": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P]),
+    "slim_linear_fwd_ex": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P, _I]),
+    "slim_linear_fwd_host": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _P, _P, _SZ, _P, _P]),
+    "slim_select_kernel": (_I, [_I, _I, _I, _I]),
+    "slim_last_launch_count": (_I, []),
+    "slim_strerror": (ctypes.c_char_p, [_I]),
+    "slim_version": (ctypes.c_char_p, []),
+}
+
+
+class SlimError(RuntimeError):
+    def __init__(self, code: int, where: str, text: str = ""):
+        super().__init__(f"{where}: {text or code} (status {code})")
+        self.code = code
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libslim.so`` (built in-tree by ``build.py``); raise if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise SlimError(-1, "load", f"{LIB_PATH} not found: run paper_2410_09615_b200/build.py")
+        l = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = l
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().slim_strerror(code).decode()
+
+
+def _check(code: int, where: str):
+    if code != SLIM_OK:
+        raise SlimError(code, where, strerror(code))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t, dtype, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def bf16_from_bits(bits: np.ndarray, device="cuda") -> torch.Tensor:
+    """uint16 bfloat16 bit patterns (host) -> torch.bfloat16 tensor on ``device``."""
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(device)
+
+
+def bits_from_bf16(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def read_status(status: torch.Tensor) -> int:
+    return int(status.item()) & 0xFFFFFFFF
+
+
+def raise_on_status(bits: int, where: str):
+    for code in (SLIM_ERR_BAD_MASK, SLIM_ERR_CODE_RANGE, SLIM_ERR_TIMEOUT):
+        if bits & (1 << code):
+            raise SlimError(code, where, strerror(code))
+
+
+def slim_pack(codes: torch.Tensor, mask: torch.Tensor, vals=None, meta=None, status=None, check=True):
+    """codes int8 [d_out, d_in], mask uint8 [d_out, d_in] -> (vals, meta) uint8 tensors."""
+    _dev(codes, torch.int8, "codes"), _dev(mask, torch.uint8, "mask")
+    d_out, d_in = codes.shape
+    if vals is None:
+        vals = torch.empty((d_out, d_in // 4), dtype=torch.uint8, device=codes.device)
+    if meta is None:
+        meta = torch.empty((d_out, d_in // 8), dtype=torch.uint8, device=codes.device)
+    own_status = status is None and check
+    if own_status:
+        status = torch.zeros(1, dtype=torch.int32, device=codes.device)
+    _check(lib().slim_pack(_ptr(codes), _ptr(mask), d_out, d_in, _ptr(vals), _ptr(meta), _ptr(status), _stream()),
+           "slim_pack")
+    if own_status:
+        raise_on_status(read_status(status), "slim_pack")
+    return vals, meta
+
+
+def slim_unpack(vals: torch.Tensor, meta: torch.Tensor, want_mask=True):
+    _dev(vals, torch.uint8, "vals"), _dev(meta, torch.uint8, "meta")
+    d_out, d_in = vals.shape[0], vals.shape[1] * 4
+    codes = torch.empty((d_out, d_in), dtype=torch.int8, device=vals.device)
+    mask = torch.empty((d_out, d_in), dtype=torch.uint8, device=vals.device) if want_mask else None
+    _check(lib().slim_unpack(_ptr(vals), _ptr(meta), d_out, d_in, _ptr(codes), _ptr(mask), _stream()), "slim_unpack")
+    return codes, mask
+
+
+def slim_workspace_bytes(b: int, d_out: int, d_in: int, r: int) -> int:
+    return int(lib().slim_workspace_bytes(b, d_out, d_in, r))
+
+
+def slim_select_kernel(b: int, d_out: int, d_in: int, r: int) -> int:
+    return int(lib().slim_select_kernel(b, d_out, d_in, r))
+
+
+def slim_last_launch_count() -> int:
+    return int(lib().slim_last_launch_count())
+
+
+def new_workspace(b: int, d_out: int, d_in: int, r: int, device="cuda") -> torch.Tensor:
+    """Allocate a workspace of the required size with zeroed synchronisation words."""
+    n = slim_workspace_bytes(b, d_out, d_in, r)
+    if n == 0:
+        raise SlimError(SLIM_ERR_UNSUPPORTED_SHAPE, "slim_workspace_bytes", "illegal shape")
+    return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def slim_workspace_reset(workspace: torch.Tensor):
+    _check(lib().slim_workspace_reset(_ptr(workspace), workspace.numel(), _stream()), "slim_workspace_reset")
+
+
+def slim_linear_fwd(X, vals, meta, s: float, L, R, Y=None, workspace=None, status=None,
+                    kernel: int = KERNEL_AUTO):
+    """Y = X (s Q)^T + (X R^T) L^T on the current stream.  Returns Y (bf16 [b, d_out])."""
+    _dev(X, torch.bfloat16, "X"), _dev(vals, torch.uint8, "vals"), _dev(meta, torch.uint8, "meta")
+    b, d_in = X.shape
+    d_out = vals.shape[0]
+    r = 0 if L is None else L.shape[1]
+    if r:
+        _dev(L, torch.bfloat16, "L"), _dev(R, torch.bfloat16, "R")
+        if tuple(L.shape) != (d_out, r) or tuple(R.shape) != (r, d_in):
+            raise ValueError("adapter shapes do not match the weight")
+    if vals.shape[1] * 4 != d_in or tuple(meta.shape) != (d_out, d_in // 8):
+        raise ValueError("packed weight does not match X")
+    if Y is None:
+        Y = torch.empty((b, d_out), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = new_workspace(b, d_out, d_in, r, X.device)
+    fn = lib().slim_linear_fwd_ex
+    _check(fn(_ptr(X), b, _ptr(vals), _ptr(meta), float(s), _ptr(L) if r else None, _ptr(R) if r else None,
+              r, d_out, d_in, _ptr(Y), _ptr(workspace), workspace.numel(), _ptr(status), _stream(), int(kernel)),
+           "slim_linear_fwd")
+    return Y
+
+
+def slim_linear_fwd_host(X_host: torch.Tensor, vals, meta, s: float, L, R, Y_host: torch.Tensor,
+                         x_dev, y_dev, workspace, status=None):
+    """Host-buffer form: X_host / Y_host are (pinned) CPU bf16 tensors; copies
+    run inside the call and the stream is synchronised before it returns."""
+    b, d_in = X_host.shape
+    d_out = vals.shape[0]
+    r = 0 if L is None else L.shape[1]
+    _check(lib().slim_linear_fwd_host(ctypes.c_void_p(X_host.data_ptr()), b, _ptr(vals), _ptr(meta), float(s),
+                                      _ptr(L) if r else None, _ptr(R) if r else None, r, d_out, d_in,
+                                      ctypes.c_void_p(Y_host.data_ptr()), _ptr(x_dev), _ptr(y_dev),
+                                      _ptr(workspace), workspace.numel(), _ptr(status), _stream()),
+           "slim_linear_fwd_host")
+    return Y_host

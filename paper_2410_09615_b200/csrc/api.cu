@@ -1,0 +1,188 @@
+// C-ABI entry points of libslim: argument checks, dispatch by batch size,
+// per-device attribute cache.  All arithmetic lives in the kernel files.
+#include <mutex>
+#include "common.cuh"
+
+namespace slim {
+
+static DeviceInfo g_info[64];
+static std::mutex g_info_mutex;
+static thread_local int t_launches = 0;
+
+void count_launch(int n) { t_launches += n; }
+void reset_launch_count() { t_launches = 0; }
+
+const DeviceInfo* device_info(slim_status_t* err) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = SLIM_ERR_CUDA; return nullptr; }
+    DeviceInfo& di = g_info[dev];
+    if (!di.ready) {
+        std::lock_guard<std::mutex> lock(g_info_mutex);
+        if (!di.ready) {
+            cudaDeviceProp prop;
+            if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { *err = SLIM_ERR_CUDA; return nullptr; }
+            di.cc_major = prop.major;
+            di.sm_count = prop.multiProcessorCount;
+            if (prop.major == 10) {
+                di.decode_ctas_per_sm[0] = decode_query_residency(1);
+                di.decode_ctas_per_sm[1] = decode_query_residency(2);
+            }
+            di.ready = true;
+        }
+    }
+    if (di.cc_major != 10) { *err = SLIM_ERR_ARCH; return nullptr; }
+    return &di;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static slim_status_t check_weight_shape(int d_out, int d_in) {
+    if (d_out < 1 || d_in < 1) return SLIM_ERR_INVALID_ARG;
+    if (d_in % 64 != 0 || d_out % 16 != 0) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    return SLIM_OK;
+}
+
+static slim_kernel_t select_kernel(int b, int d_out, int d_in, int r) {
+    if (b <= 16 && decode_supports(b, d_out, d_in, r)) return SLIM_KERNEL_DECODE;
+    return SLIM_KERNEL_SIMPLE;
+}
+
+static size_t workspace_bytes(int b, int d_out, int d_in, int r) {
+    size_t need = simple_workspace_bytes(b, d_out, d_in, r);
+    const size_t d = decode_workspace_bytes(b, d_out, d_in, r);
+    if (d > need) need = d;
+    need = (need + 255) / 256 * 256;
+    return SLIM_WORKSPACE_SYNC_BYTES + need;
+}
+
+}  // namespace slim
+
+using namespace slim;
+
+extern "C" {
+
+slim_status_t slim_pack(const int8_t* codes, const uint8_t* mask, int d_out, int d_in,
+                        uint8_t* vals, uint8_t* meta, uint32_t* status_dev, void* cuda_stream)
+{
+    reset_launch_count();
+    if (!codes || !mask || !vals || !meta) return SLIM_ERR_INVALID_ARG;
+    slim_status_t st = check_weight_shape(d_out, d_in);
+    if (st != SLIM_OK) return st;
+    if (!aligned16(codes) || !aligned16(mask) || !aligned16(vals) || !aligned16(meta)) return SLIM_ERR_INVALID_ARG;
+    if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return SLIM_ERR_INVALID_ARG;
+    return launch_pack(codes, mask, d_out, d_in, vals, meta, status_dev, (cudaStream_t)cuda_stream);
+}
+
+slim_status_t slim_unpack(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in,
+                          int8_t* codes, uint8_t* mask, void* cuda_stream)
+{
+    reset_launch_count();
+    if (!vals || !meta || !codes) return SLIM_ERR_INVALID_ARG;
+    slim_status_t st = check_weight_shape(d_out, d_in);
+    if (st != SLIM_OK) return st;
+    if (!aligned16(codes) || !aligned16(vals) || !aligned16(meta) || (mask && !aligned16(mask))) return SLIM_ERR_INVALID_ARG;
+    return launch_unpack(vals, meta, d_out, d_in, codes, mask, (cudaStream_t)cuda_stream);
+}
+
+size_t slim_workspace_bytes(int b, int d_out, int d_in, int r)
+{
+    if (b < 1 || r < 0 || r % 16 != 0 || check_weight_shape(d_out, d_in) != SLIM_OK) return 0;
+    return workspace_bytes(b, d_out, d_in, r);
+}
+
+slim_status_t slim_workspace_reset(void* workspace, size_t workspace_bytes_, void* cuda_stream)
+{
+    if (!workspace || workspace_bytes_ < SLIM_WORKSPACE_SYNC_BYTES) return SLIM_ERR_WORKSPACE;
+    return cudaMemsetAsync(workspace, 0, SLIM_WORKSPACE_SYNC_BYTES, (cudaStream_t)cuda_stream) == cudaSuccess
+               ? SLIM_OK : SLIM_ERR_CUDA;
+}
+
+slim_kernel_t slim_select_kernel(int b, int d_out, int d_in, int r)
+{
+    if (b < 1 || r < 0 || r % 16 != 0 || check_weight_shape(d_out, d_in) != SLIM_OK) return SLIM_KERNEL_AUTO;
+    return select_kernel(b, d_out, d_in, r);
+}
+
+slim_status_t slim_linear_fwd_ex(const void* X, int b, const uint8_t* vals, const uint8_t* meta,
+                                 float s, const void* L, const void* R, int r, int d_out, int d_in,
+                                 void* Y, void* workspace, size_t workspace_bytes_,
+                                 uint32_t* status_dev, void* cuda_stream, slim_kernel_t kernel)
+{
+    reset_launch_count();
+    if (!X || !vals || !meta || !Y || b < 1 || r < 0) return SLIM_ERR_INVALID_ARG;
+    if ((r > 0) != (L != nullptr) || (r > 0) != (R != nullptr)) return SLIM_ERR_INVALID_ARG;
+    slim_status_t st = check_weight_shape(d_out, d_in);
+    if (st != SLIM_OK) return st;
+    if (r % 16 != 0) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(X) || !aligned16(vals) || !aligned16(meta) || !aligned16(Y) || !aligned16(L) || !aligned16(R) ||
+        !aligned16(workspace))
+        return SLIM_ERR_INVALID_ARG;
+    if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return SLIM_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes_ < workspace_bytes(b, d_out, d_in, r)) return SLIM_ERR_WORKSPACE;
+    slim_status_t derr;
+    if (!device_info(&derr)) return derr;
+    if (kernel == SLIM_KERNEL_AUTO) kernel = select_kernel(b, d_out, d_in, r);
+    const __nv_bfloat16* Xb = static_cast<const __nv_bfloat16*>(X);
+    const __nv_bfloat16* Lb = static_cast<const __nv_bfloat16*>(L);
+    const __nv_bfloat16* Rb = static_cast<const __nv_bfloat16*>(R);
+    __nv_bfloat16* Yb = static_cast<__nv_bfloat16*>(Y);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    switch (kernel) {
+    case SLIM_KERNEL_SIMPLE:
+        return launch_simple(Xb, b, vals, meta, s, Lb, Rb, r, d_out, d_in, Yb, workspace, stream);
+    case SLIM_KERNEL_DECODE:
+        if (b > 16 || !decode_supports(b, d_out, d_in, r)) return SLIM_ERR_UNSUPPORTED_SHAPE;
+        return launch_decode(Xb, b, vals, meta, s, Lb, Rb, r, d_out, d_in, Yb, workspace, status_dev, stream);
+    default:
+        return SLIM_ERR_UNSUPPORTED_SHAPE;
+    }
+}
+
+slim_status_t slim_linear_fwd(const void* X, int b, const uint8_t* vals, const uint8_t* meta,
+                              float s, const void* L, const void* R, int r, int d_out, int d_in,
+                              void* Y, void* workspace, size_t workspace_bytes_,
+                              uint32_t* status_dev, void* cuda_stream)
+{
+    return slim_linear_fwd_ex(X, b, vals, meta, s, L, R, r, d_out, d_in, Y, workspace, workspace_bytes_,
+                              status_dev, cuda_stream, SLIM_KERNEL_AUTO);
+}
+
+slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* vals,
+                                   const uint8_t* meta, float s, const void* L, const void* R,
+                                   int r, int d_out, int d_in, void* Y_host, void* x_dev,
+                                   void* y_dev, void* workspace, size_t workspace_bytes_,
+                                   uint32_t* status_dev, void* cuda_stream)
+{
+    if (!X_host || !Y_host || !x_dev || !y_dev || b < 1 || d_in < 1 || d_out < 1) return SLIM_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(x_dev, X_host, (size_t)b * d_in * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return SLIM_ERR_CUDA;
+    slim_status_t st = slim_linear_fwd(x_dev, b, vals, meta, s, L, R, r, d_out, d_in, y_dev, workspace,
+                                       workspace_bytes_, status_dev, cuda_stream);
+    if (st != SLIM_OK) return st;
+    if (cudaMemcpyAsync(Y_host, y_dev, (size_t)b * d_out * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return SLIM_ERR_CUDA;
+    return cudaStreamSynchronize(stream) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+}
+
+int slim_last_launch_count(void) { return t_launches; }
+
+const char* slim_strerror(slim_status_t status)
+{
+    switch (status) {
+    case SLIM_OK: return "ok";
+    case SLIM_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, bad size)";
+    case SLIM_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (d_in % 64, d_out % 16, r % 16 must be 0)";
+    case SLIM_ERR_BAD_MASK: return "a 2:4 group keeps more than two values";
+    case SLIM_ERR_CODE_RANGE: return "a kept code lies outside [-8, 7]";
+    case SLIM_ERR_WORKSPACE: return "workspace missing or too small";
+    case SLIM_ERR_CUDA: return "CUDA runtime error";
+    case SLIM_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case SLIM_ERR_ARCH: return "device is not compute capability 10.x";
+    }
+    return "unknown status";
+}
+
+const char* slim_version(void) { return "libslim 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,49 @@
+// Shared device/host helpers of libslim (CUDA side only).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "slim.h"
+
+namespace slim {
+
+// Bit a device-detected error sets in the caller's status word.
+__device__ __forceinline__ void flag_error(uint32_t* status_dev, int code) {
+    if (status_dev) atomicOr(status_dev, 1u << code);
+}
+
+__host__ __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Per-device facts the launchers need (filled once per device, read-only after).
+struct DeviceInfo {
+    bool ready;
+    int cc_major;
+    int sm_count;
+    int decode_ctas_per_sm[2];   // cooperative residency of the decode kernel, NT = 1, 2
+};
+const DeviceInfo* device_info(slim_status_t* err);
+
+// Launch bookkeeping for slim_last_launch_count().
+void count_launch(int n);
+void reset_launch_count();
+
+// ---- launchers (defined in the kernel files) --------------------------------
+slim_status_t launch_pack(const int8_t* codes, const uint8_t* mask, int d_out, int d_in,
+                          uint8_t* vals, uint8_t* meta, uint32_t* status_dev, cudaStream_t st);
+slim_status_t launch_unpack(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in,
+                            int8_t* codes, uint8_t* mask, cudaStream_t st);
+
+size_t simple_workspace_bytes(int b, int d_out, int d_in, int r);
+slim_status_t launch_simple(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
+                            float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
+                            int d_out, int d_in, __nv_bfloat16* Y, void* ws, cudaStream_t st);
+
+bool decode_supports(int b, int d_out, int d_in, int r);
+size_t decode_workspace_bytes(int b, int d_out, int d_in, int r);
+slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
+                            float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
+                            int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
+                            cudaStream_t st);
+int decode_query_residency(int nt);
+
+}  // namespace slim

@@ -14,6 +14,8 @@ Recipe (one layer):
           (ties: lower index wins)             NVIDIA 2:4 pattern
   L ~ N(0, 0.02^2) [d_out, r],  R ~ N(0, 0.02^2) [r, d_in],  X ~ N(0, 1) [b, d_in],
   each rounded to bfloat16 (round to nearest even) and carried as uint16 bits.
+Streams: numpy PCG64 seeded with [seed, 1] (weights), [seed, 2] (adapters),
+[seed, 3] (activations), [seed, 4] (row samples).
 """
 from __future__ import annotations
 
@@ -71,39 +73,65 @@ class Layer:
 
 
 def top2_mask(W: np.ndarray) -> np.ndarray:
-    """2:4 magnitude mask along the last axis; ties resolved to the lower index."""
+    """2:4 magnitude mask along the last axis; ties resolved to the lower index.
+    An element is kept when fewer than two others of its group beat it, where
+    "beats" means larger magnitude, or equal magnitude at a lower index."""
     d_out, d_in = W.shape
     a = np.abs(W).reshape(d_out, d_in // 4, 4)
-    # stable argsort of -|w| keeps the lower index first among equals
-    order = np.argsort(-a, axis=-1, kind="stable")
-    mask = np.zeros_like(a, dtype=np.uint8)
-    np.put_along_axis(mask, order[..., :2], 1, axis=-1)
+    mask = np.empty(a.shape, dtype=np.uint8)
+    for i in range(4):
+        beaten = np.zeros(a.shape[:2], dtype=np.uint8)
+        for j in range(4):
+            if j < i:
+                beaten += a[..., j] >= a[..., i]
+            elif j > i:
+                beaten += a[..., j] > a[..., i]
+        mask[..., i] = beaten < 2
     return mask.reshape(d_out, d_in)
 
 
-def make_weights(d_out: int, d_in: int, rng: np.random.Generator):
-    W = rng.standard_normal((d_out, d_in), dtype=np.float32) * np.float32(0.02)
+def make_weights(d_out: int, d_in: int, seed: int):
+    """(s, codes, mask) of one layer; row blocks are generated one after another
+    from a single stream so that large layers do not need several full-size
+    temporaries."""
+    rng = np.random.default_rng([int(seed), 1])
+    W = np.empty((d_out, d_in), np.float32)
+    step = max(1, (1 << 24) // d_in)
+    for r0 in range(0, d_out, step):
+        blk = W[r0:r0 + step]
+        rng.standard_normal(blk.shape, dtype=np.float32, out=blk)
+    W *= np.float32(0.02)
     s = np.float32(np.max(np.abs(W))) / np.float32(7.0)
-    codes = np.clip(np.rint(W / s), -8, 7).astype(np.int8)
-    mask = top2_mask(W)
+    codes = np.empty((d_out, d_in), np.int8)
+    mask = np.empty((d_out, d_in), np.uint8)
+    for r0 in range(0, d_out, step):
+        blk = W[r0:r0 + step]
+        codes[r0:r0 + step] = np.clip(np.rint(blk / s), -8, 7).astype(np.int8)
+        mask[r0:r0 + step] = top2_mask(blk)
     return float(s), codes, mask
 
 
-def make_layer(d_in: int, d_out: int, r: int, b: int, seed: int) -> Layer:
-    rng = np.random.default_rng(seed)
-    s, codes, mask = make_weights(d_out, d_in, rng)
-    if r > 0:
-        L = f32_to_bf16_bits(rng.standard_normal((d_out, r), dtype=np.float32) * np.float32(0.02))
-        R = f32_to_bf16_bits(rng.standard_normal((r, d_in), dtype=np.float32) * np.float32(0.02))
-    else:
-        L = R = None
-    X = f32_to_bf16_bits(rng.standard_normal((b, d_in), dtype=np.float32))
-    return Layer(d_in, d_out, r, b, seed, s, codes, mask, L, R, X)
+def make_adapters(d_out: int, d_in: int, r: int, seed: int):
+    if r <= 0:
+        return None, None
+    rng = np.random.default_rng([int(seed), 2])
+    L = f32_to_bf16_bits(rng.standard_normal((d_out, r), dtype=np.float32) * np.float32(0.02))
+    R = f32_to_bf16_bits(rng.standard_normal((r, d_in), dtype=np.float32) * np.float32(0.02))
+    return L, R
 
 
 def make_activations(b: int, d_in: int, seed: int) -> np.ndarray:
-    rng = np.random.default_rng(seed)
+    rng = np.random.default_rng([int(seed), 3])
     return f32_to_bf16_bits(rng.standard_normal((b, d_in), dtype=np.float32))
+
+
+def make_layer(d_in: int, d_out: int, r: int, b: int, seed: int, weights=None) -> Layer:
+    """All host arrays of one case.  ``weights`` = a cached (s, codes, mask) triple
+    to reuse across cases that share a weight; otherwise generated from ``seed``."""
+    s, codes, mask = weights if weights is not None else make_weights(d_out, d_in, seed)
+    L, R = make_adapters(d_out, d_in, r, seed)
+    X = make_activations(b, d_in, seed)
+    return Layer(d_in, d_out, r, b, seed, s, codes, mask, L, R, X)
 
 
 # ---------------------------------------------------------------------------
@@ -130,29 +158,36 @@ CONFIGS = {
 
 
 def config_cases(cfg: int):
-    """Yield (layer_name, d_in, d_out, r, b, seed) for every case of a configuration."""
+    """Yield (layer_name, d_in, d_out, r, b, seed, weight_seed) for every case of a
+    configuration.  Cases that differ only in batch size or rank share the
+    layer's weight (``weight_seed``); adapters and activations use ``seed``."""
     c = CONFIGS[cfg]
     for li, (name, d_in, d_out, _count) in enumerate(c["shapes"]):
+        wseed = 1000 * cfg + 10 * li
         for bi, b in enumerate(c["batches"]):
             if c["ranks"] == "fixed64":
-                yield name, d_in, d_out, 64, b, 0
+                yield name, d_in, d_out, 64, b, 0, 0
                 continue
             for ri, ratio in enumerate(c["ranks"]):
                 r = rank_for_ratio(ratio, d_in, d_out)
-                seed = 1000 * cfg + 10 * li + bi + 100 * ri
-                yield name, d_in, d_out, r, b, seed
+                yield name, d_in, d_out, r, b, wseed + bi + 100 * ri, wseed
 
 
-def sample_rows(b: int, tile: int = 128, seed: int = 0) -> np.ndarray:
-    """Token rows on which a large-batch output is compared one by one: every
-    row of the first and of the last ``tile`` rows, plus one seeded row in every
-    other tile."""
-    if b <= 2 * tile:
+def sample_rows(b: int, tile: int = 128, seed: int = 0, dense_edges: bool = True) -> np.ndarray:
+    """Token rows on which a large-batch output is compared one by one: the
+    first and the last ``tile`` rows (all of them, or their first / middle / last
+    row when ``dense_edges`` is False) plus one seeded row in every other tile."""
+    if b <= 2 * tile and dense_edges:
         return np.arange(b, dtype=np.int32)
-    rng = np.random.default_rng(seed)
-    rows = list(range(tile)) + list(range(b - tile, b))
+    rng = np.random.default_rng([int(seed), 4])
+    if dense_edges:
+        rows = list(range(tile)) + list(range(b - tile, b))
+    else:
+        e = min(tile, b)
+        rows = [0, e // 2, e - 1, b - e, b - 1 - e // 2, b - 1]
     for t in range(1, (b - 1) // tile):
         lo, hi = t * tile, min((t + 1) * tile, b - tile)
         if hi > lo:
             rows.append(int(rng.integers(lo, hi)))
+    rows = [x for x in rows if 0 <= x < b]
     return np.array(sorted(set(rows)), dtype=np.int32)

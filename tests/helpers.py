@@ -1,0 +1,53 @@
+"""Shared helpers of the GPU parity tests (host arrays -> device, oracle calls)."""
+from __future__ import annotations
+
+import functools
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2410_09615_b200 import binding, inputs, parity
+
+
+@functools.lru_cache(maxsize=2)
+def cached_weights(d_out: int, d_in: int, seed: int):
+    """(s, codes, mask, oracle vals, oracle meta) of one layer, host side."""
+    s, codes, mask = inputs.make_weights(d_out, d_in, seed)
+    vals, meta = oracle.pack(codes, mask)
+    return s, codes, mask, vals, meta
+
+
+def to_dev(a: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def run_case(d_in, d_out, r, b, seed, wseed=None, kernel=binding.KERNEL_AUTO, rows=None, check_pack=True):
+    """Generate one case, pack it on the GPU (bit-exact check against the oracle's
+    bytes), run the forward through the C-ABI and compare with the oracle on
+    ``rows`` (None = every token).  Returns the comparison record."""
+    wseed = seed if wseed is None else wseed
+    s, codes, mask, ovals, ometa = cached_weights(d_out, d_in, wseed)
+    ly = inputs.make_layer(d_in, d_out, r, b, seed, weights=(s, codes, mask))
+    vals, meta = binding.slim_pack(to_dev(codes), to_dev(mask))
+    if check_pack:
+        assert torch.equal(vals.cpu(), torch.from_numpy(ovals)), "vals differ from the oracle's bytes"
+        assert torch.equal(meta.cpu(), torch.from_numpy(ometa)), "meta differ from the oracle's bytes"
+    X = binding.bf16_from_bits(ly.X)
+    L = binding.bf16_from_bits(ly.L) if r else None
+    R = binding.bf16_from_bits(ly.R) if r else None
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = binding.new_workspace(b, d_out, d_in, r)
+    Y = binding.slim_linear_fwd(X, vals, meta, s, L, R, workspace=ws, status=status, kernel=kernel)
+    launches = binding.slim_last_launch_count()
+    torch.cuda.synchronize()
+    assert binding.read_status(status) == 0, f"device status {binding.read_status(status):#x}"
+    # the synchronisation words are left clean for the next call
+    assert int(ws[:binding.WORKSPACE_SYNC_BYTES].to(torch.int32).sum().item()) == 0
+    y = inputs.bf16_bits_to_f64(binding.bits_from_bf16(Y))
+    if rows is not None:
+        y = y[np.asarray(rows)]
+    y_ref = oracle.linear_fwd(ly.X, ovals, ometa, s, ly.L, ly.R, rows=rows)
+    res = parity.compare(y, y_ref)
+    res["launches"] = launches
+    return res

@@ -42,7 +42,7 @@ def test_top2_mask_ties_take_lower_index():
 def test_config_table_covers_all_five():
     n = {c: len(list(inputs.config_cases(c))) for c in range(5)}
     assert n == {0: 1, 1: 6, 2: 3, 3: 9, 4: 48}
-    assert ("single", 512, 512, 64, 8, 0) in list(inputs.config_cases(0))
+    assert ("single", 512, 512, 64, 8, 0, 0) in list(inputs.config_cases(0))
 
 
 def test_sample_rows():
@@ -52,6 +52,9 @@ def test_sample_rows():
     tiles = set((rows // 128).tolist())
     assert tiles == set(range(16))
     assert inputs.sample_rows(16).tolist() == list(range(16))
+    few = inputs.sample_rows(4096, dense_edges=False)
+    assert few[0] == 0 and few[-1] == 4095 and len(few) < 40
+    assert set((few // 128).tolist()) == set(range(32))
 
 
 def test_parity_rule():
