@@ -1,0 +1,515 @@
+#!/usr/bin/env python
+"""Benchmark of the SLiM compressed linear layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload: the LLaMA-2-7B decode layer set.  One step = the seven linears of one
+transformer block (4 x 4096->4096, 2 x 4096->11008, 1 x 11008->4096; int4 2:4
+weights, per-layer fp32 scale, rank-416 bf16 adapters) run once at batch 1 and
+once at batch 16: 14 calls of slim_linear_fwd.  Two full sets of packed weights
+and adapters (141 MB each) alternate, so 282 MB stream through the 126 MB L2
+between two uses of the same bytes and every call reads its weights from HBM.
+The step is captured in a CUDA graph and replayed; time is taken with CUDA
+events on the launching stream, max over ranks.  Prints one JSON line.
+
+With N > 1 every rank runs the same step on its own GPU (independent replicas,
+no collective on the data path).
+
+--impl reference times the CPU oracle (oracle/) on this machine's host cores on the
+same workload: each step runs each distinct (shape, batch) call once and
+weights it by how often the block uses it.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2410_09615_b200 import inputs  # noqa: E402
+
+METRIC = "slim_linear_us_per_call"
+UNIT = "us/call"
+WORKLOAD = "llama2_7b_decode_layer_set"
+BATCHES = (1, 16)
+SHAPES = inputs.LLAMA2_SHAPES["7b"]            # (name, d_in, d_out, count per block)
+CALLS_PER_STEP = sum(c for *_x, c in SHAPES) * len(BATCHES)
+HBM_FALLBACK_GBS = 6650.0                      # earlier measurement on this machine
+NOMINAL_HBM_GBS = 8000.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch from an
+# ncu capture (profiles/), keyed by (d_in, d_out, r, b); None = not captured for
+# the current kernel.
+NCU_TRAFFIC_BYTES = {}
+
+
+def algorithmic_bytes(d_in, d_out, r, b):
+    """Bytes one forward call must move: 3 bits per dense weight (4-bit code of
+    the kept half plus 2-bit index each), bf16 adapters, X, Y and the scale."""
+    return 0.375 * d_out * d_in + 2.0 * r * (d_in + d_out) + 2.0 * b * (d_in + d_out) + 4.0
+
+
+def executed_flops(d_in, d_out, r, b):
+    return 2.0 * b * d_out * d_in / 2.0 + 2.0 * b * r * (d_in + d_out)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return HBM_FALLBACK_GBS, "fallback"
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU while a region runs
+    (NVML, read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = (pynvml.nvmlDeviceGetHandleByUUID(index) if isinstance(index, (str, bytes))
+                      else pynvml.nvmlDeviceGetHandleByIndex(index))
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def _reason_names(self, mask):
+        nv = self.nv
+        table = [("hw_slowdown", "nvmlClocksEventReasonHwSlowdown", "nvmlClocksThrottleReasonHwSlowdown"),
+                 ("hw_thermal_slowdown", "nvmlClocksEventReasonHwThermalSlowdown", "nvmlClocksThrottleReasonHwThermalSlowdown"),
+                 ("sw_thermal_slowdown", "nvmlClocksEventReasonSwThermalSlowdown", "nvmlClocksThrottleReasonSwThermalSlowdown"),
+                 ("sw_power_cap", "nvmlClocksEventReasonSwPowerCap", "nvmlClocksThrottleReasonSwPowerCap"),
+                 ("hw_power_brake", "nvmlClocksEventReasonHwPowerBrakeSlowdown", "nvmlClocksThrottleReasonHwPowerBrakeSlowdown")]
+        out = []
+        for name, a, b in table:
+            bit = getattr(nv, a, None) or getattr(nv, b, None)
+            if bit and (mask & bit):
+                out.append(name)
+        return out
+
+    def _once(self):
+        try:
+            self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+            try:
+                mask = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+            except Exception:
+                mask = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+            self.reasons.update(self._reason_names(mask))
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self._once()
+            time.sleep(self.period)
+
+    def start(self):
+        if self.ok:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        if self.ok and self._thr:
+            self._once()
+            self._stop.set()
+            self._thr.join()
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ host data
+def host_layers():
+    """The three distinct layers of the block, generated once on the host."""
+    out = []
+    for li, (name, d_in, d_out, count) in enumerate(SHAPES):
+        r = inputs.default_rank(d_in, d_out)
+        wseed = 1000 + 10 * li
+        s, codes, mask = inputs.make_weights(d_out, d_in, wseed)
+        L, R = inputs.make_adapters(d_out, d_in, r, wseed)
+        out.append(dict(name=name, d_in=d_in, d_out=d_out, r=r, count=count, s=s, codes=codes, mask=mask,
+                        L=L, R=R, X={b: inputs.make_activations(b, d_in, wseed + bi) for bi, b in enumerate(BATCHES)}))
+    return out
+
+
+# ------------------------------------------------------------------ reference arm
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    layers = host_layers()
+    for ly in layers:
+        ly["vals"], ly["meta"] = oracle.pack(ly["codes"], ly["mask"])
+
+    def step():
+        t_weighted = 0.0
+        for ly in layers:
+            for b in BATCHES:
+                t0 = time.perf_counter()
+                oracle.linear_fwd(ly["X"][b], ly["vals"], ly["meta"], ly["s"], ly["L"], ly["R"])
+                t_weighted += (time.perf_counter() - t0) * ly["count"]
+        return t_weighted
+
+    for _ in range(args.warmup):
+        step()
+    total = sum(step() for _ in range(args.steps))
+    ms_per_step = 1e3 * total / args.steps
+    value = 1e3 * ms_per_step / CALLS_PER_STEP
+    sample = ("each step runs the oracle once per distinct (layer shape, batch) pair, all token rows, "
+              "and weights the time by the number of such linears in the block (4/2/1)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "batches": list(BATCHES), "calls_per_step": CALLS_PER_STEP},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------ GPU arm
+def run_ours(args):
+    import ctypes
+    import torch
+    import torch.distributed as dist
+    from paper_2410_09615_b200 import binding as K
+    from paper_2410_09615_b200 import build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    build.build()
+    lib = K.lib()
+    dev = torch.device("cuda", local)
+
+    # ---- weights: packed on the GPU by slim_pack, two full sets of the block
+    layers = host_layers()
+    n_sets = 2
+    slots = []            # one entry per linear of the block and per set
+    for ly in layers:
+        codes_d, mask_d = torch.from_numpy(ly["codes"]).to(dev), torch.from_numpy(ly["mask"]).to(dev)
+        vals, meta = K.slim_pack(codes_d, mask_d)
+        del codes_d, mask_d
+        ly["vals"], ly["meta"] = vals, meta
+        ly["Ld"], ly["Rd"] = K.bf16_from_bits(ly["L"], dev), K.bf16_from_bits(ly["R"], dev)
+        ly["Xd"] = {b: K.bf16_from_bits(ly["X"][b], dev) for b in BATCHES}
+        ly["Yd"] = {b: torch.empty((b, ly["d_out"]), dtype=torch.bfloat16, device=dev) for b in BATCHES}
+        ly["copies"] = [[(vals.clone(), meta.clone(), ly["Ld"].clone(), ly["Rd"].clone())
+                         for _ in range(ly["count"])] for _ in range(n_sets)]
+    ws_bytes = max(K.slim_workspace_bytes(b, ly["d_out"], ly["d_in"], ly["r"]) for ly in layers for b in BATCHES)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    set_bytes = sum(c[0].numel() + c[1].numel() + 2 * c[2].numel() + 2 * c[3].numel()
+                    for ly in layers for c in ly["copies"][0])
+
+    fwd = lib.slim_linear_fwd
+    P = ctypes.c_void_p
+
+    def call_args(ly, b, copy):
+        vals, meta, L, R = copy
+        return (P(ly["Xd"][b].data_ptr()), b, P(vals.data_ptr()), P(meta.data_ptr()), ctypes.c_float(ly["s"]),
+                P(L.data_ptr()), P(R.data_ptr()), ly["r"], ly["d_out"], ly["d_in"], P(ly["Yd"][b].data_ptr()),
+                P(ws.data_ptr()), ws_bytes, P(status.data_ptr()))
+
+    # the 14 calls of one step: batch 1 on weight set 0, batch 16 on weight set 1
+    step_calls = []
+    for si, b in enumerate(BATCHES):
+        for ly in layers:
+            for copy in ly["copies"][si % n_sets]:
+                step_calls.append((ly, b, call_args(ly, b, copy)))
+    assert len(step_calls) == CALLS_PER_STEP
+
+    def issue_step(stream_ptr):
+        for _ly, _b, a in step_calls:
+            rc = fwd(*a, stream_ptr)
+            if rc != 0:
+                raise RuntimeError(f"slim_linear_fwd failed: {K.strerror(rc)}")
+
+    stream = torch.cuda.Stream(device=dev)
+    sp = P(stream.cuda_stream)
+    with torch.cuda.stream(stream):
+        issue_step(sp)                      # first call fills the per-device cache outside any capture
+    stream.synchronize()
+    launches_per_step = 0
+    for _ly, _b, a in step_calls:
+        fwd(*a, sp)
+        launches_per_step += lib.slim_last_launch_count()
+    stream.synchronize()
+
+    graph, launch_mode = None, "stream"
+    if not args.no_graph:
+        try:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                issue_step(P(torch.cuda.current_stream().cuda_stream))
+            graph, launch_mode = g, "cuda_graph"
+        except Exception as e:             # capture refused: time plain stream launches
+            sys.stderr.write(f"[bench] graph capture failed ({e}); timing stream launches\n")
+            torch.cuda.synchronize()
+            graph = None
+
+    def run_steps(n):
+        with torch.cuda.stream(stream):
+            for _ in range(n):
+                if graph is not None:
+                    graph.replay()
+                else:
+                    issue_step(sp)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        gpu_id = local
+    sampler = ClockSampler(gpu_id)
+    if not sampler.ok:
+        sampler = ClockSampler(local)
+    run_steps(args.warmup)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+    run_steps(args.steps)
+    with torch.cuda.stream(stream):
+        e1.record(stream)
+    barrier()
+    sampler.stop()
+    elapsed_ms = e0.elapsed_time(e1)
+    if K.read_status(status) != 0:
+        raise RuntimeError(f"device status {K.read_status(status):#x}")
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = 1e3 * ms_per_step / (CALLS_PER_STEP * world)
+
+    # ---- roofline of the dominant kernel over the timed region
+    step_bytes = sum(algorithmic_bytes(ly["d_in"], ly["d_out"], ly["r"], b) for ly, b, _ in step_calls)
+    peak, peak_kind = measured_peaks()
+    achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC_BYTES and all((ly["d_in"], ly["d_out"], ly["r"], b) in NCU_TRAFFIC_BYTES for ly, b, _ in step_calls):
+        traffic = sum(NCU_TRAFFIC_BYTES[(ly["d_in"], ly["d_out"], ly["r"], b)] for ly, b, _ in step_calls) / len(step_calls)
+    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "traffic": traffic, "bytes_per_launch": step_bytes / len(step_calls),
+                "avg_launch_us": 1e3 * ms_per_step / len(step_calls)}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "batches": list(BATCHES), "calls_per_step": CALLS_PER_STEP,
+                       "layers": [[ly["name"], ly["d_in"], ly["d_out"], ly["r"], ly["count"]] for ly in layers],
+                       "l2": f"inputs larger than L2: {n_sets} weight sets of {set_bytes / 1e6:.0f} MB alternate",
+                       "launch": launch_mode, "parallelism": f"replicas x{world}"},
+            "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
+            "clocks": sampler.summary()}
+
+    if rank == 0 and not args.skip_extras:
+        line["per_case"] = per_case_table(K, lib, layers, ws, ws_bytes, status, stream, peak)
+        line["pack"] = time_pack(K, layers[1], stream)
+    # ---- end to end through the host-buffer entry point
+    line["e2e"] = time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, world, barrier)
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        line["cpu_baseline"] = time_cpu_baseline(layers)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def time_graph_of_calls(lib, calls, stream, replays=20):
+    """Median per-call time (us) of a CUDA graph holding `calls`, replayed."""
+    import ctypes
+    import torch
+    P = ctypes.c_void_p
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        cur = P(torch.cuda.current_stream().cuda_stream)
+        for a in calls:
+            lib.slim_linear_fwd(*a, cur)
+    times = []
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            g.replay()
+        for _ in range(replays):
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            g.replay()
+            a1.record(stream)
+            a1.synchronize()
+            times.append(1e3 * a0.elapsed_time(a1) / len(calls))
+    return float(np.median(times)), float(np.min(times))
+
+
+def per_case_table(K, lib, layers, ws, ws_bytes, status, stream, peak):
+    """Per (layer, batch): us/call over rotating weight copies (> 2x L2 between
+    reuses), algorithmic GB/s and fraction of the HBM roofline."""
+    import ctypes
+    P = ctypes.c_void_p
+    rows = []
+    for ly in layers:
+        per_copy = ly["vals"].numel() + ly["meta"].numel() + 2 * ly["Ld"].numel() + 2 * ly["Rd"].numel()
+        n_copies = int(np.ceil(2 * 126e6 / per_copy)) + 1
+        copies = [(ly["vals"].clone(), ly["meta"].clone(), ly["Ld"].clone(), ly["Rd"].clone()) for _ in range(n_copies)]
+        for b in BATCHES:
+            calls = [(P(ly["Xd"][b].data_ptr()), b, P(c[0].data_ptr()), P(c[1].data_ptr()), ctypes.c_float(ly["s"]),
+                      P(c[2].data_ptr()), P(c[3].data_ptr()), ly["r"], ly["d_out"], ly["d_in"],
+                      P(ly["Yd"][b].data_ptr()), P(ws.data_ptr()), ws_bytes, P(status.data_ptr()))
+                     for c in copies] * 3
+            try:
+                med, best = time_graph_of_calls(lib, calls, stream)
+            except Exception as e:
+                rows.append({"layer": ly["name"], "b": b, "error": str(e)[:80]})
+                continue
+            nbytes = algorithmic_bytes(ly["d_in"], ly["d_out"], ly["r"], b)
+            gbs = nbytes / (med * 1e-6) / 1e9
+            rows.append({"layer": ly["name"], "d_in": ly["d_in"], "d_out": ly["d_out"], "r": ly["r"], "b": b,
+                         "us": round(med, 3), "us_min": round(best, 3), "GBs": round(gbs, 1),
+                         "frac_measured": round(gbs / peak, 4), "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
+                         "executed_TFLOPs": round(executed_flops(ly["d_in"], ly["d_out"], ly["r"], b) / (med * 1e-6) / 1e12, 2)})
+        del copies
+    return rows
+
+
+def time_pack(K, ly, stream):
+    import torch
+    codes, mask = torch.from_numpy(ly["codes"]).cuda(), torch.from_numpy(ly["mask"]).cuda()
+    vals, meta = K.slim_pack(codes, mask)
+    with torch.cuda.stream(stream):
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(3):
+            K.slim_pack(codes, mask, vals, meta, check=False)
+        a0.record(stream)
+        for _ in range(10):
+            K.slim_pack(codes, mask, vals, meta, check=False)
+        a1.record(stream)
+        a1.synchronize()
+    us = 1e3 * a0.elapsed_time(a1) / 10
+    nbytes = 2.375 * ly["d_out"] * ly["d_in"]
+    return {"layer": [ly["d_in"], ly["d_out"]], "us": round(us, 2), "GBs": round(nbytes / us / 1e3, 1),
+            "bytes": "2 B read + 0.375 B written per dense weight"}
+
+
+def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, world, barrier):
+    """Same step through slim_linear_fwd_host: X comes from pinned host memory
+    and Y goes back to pinned host memory inside every call."""
+    import ctypes
+    import torch
+    import torch.distributed as dist
+    P = ctypes.c_void_p
+    host = {}
+    for ly in layers:
+        for b in BATCHES:
+            xh = K.bf16_from_bits(ly["X"][b], "cpu").pin_memory()
+            yh = torch.empty((b, ly["d_out"]), dtype=torch.bfloat16).pin_memory()
+            host[(ly["name"], b)] = (xh, yh)
+    calls, h2d, d2h = [], 0, 0
+    for ly, b, a in step_calls:
+        xh, yh = host[(ly["name"], b)]
+        calls.append((P(xh.data_ptr()), b, a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], P(yh.data_ptr()),
+                      P(ly["Xd"][b].data_ptr()), P(ly["Yd"][b].data_ptr()), a[11], a[12], a[13]))
+        h2d += xh.numel() * 2
+        d2h += yh.numel() * 2
+    sp = P(stream.cuda_stream)
+    steps = max(1, min(args.steps, 200))
+
+    def run(n):
+        for _ in range(n):
+            for c in calls:
+                rc = lib.slim_linear_fwd_host(*c, sp)
+                if rc != 0:
+                    raise RuntimeError(f"slim_linear_fwd_host failed: {K.strerror(rc)}")
+
+    run(min(args.warmup, 20))
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    run(steps)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return {"value": 1e3 * ms / steps / (CALLS_PER_STEP * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "steps": steps, "api": "slim_linear_fwd_host"}
+
+
+def time_cpu_baseline(layers, repeats=8):
+    import oracle
+    t_weighted, t_raw = 0.0, 0.0
+    host = [(ly, ly["vals"].cpu().numpy(), ly["meta"].cpu().numpy()) for ly in layers]
+    for _ in range(repeats):
+        for ly, vals, meta in host:
+            for b in BATCHES:
+                t0 = time.perf_counter()
+                oracle.linear_fwd(ly["X"][b], vals, meta, ly["s"], ly["L"], ly["R"])
+                dt = time.perf_counter() - t0
+                t_raw += dt
+                t_weighted += dt * ly["count"]
+    return {"value": 1e6 * t_weighted / repeats / CALLS_PER_STEP, "unit": UNIT, "cores": oracle.num_threads(),
+            "kind": "oracle",
+            "sample": f"one oracle call per distinct (layer shape, batch) pair of the step, all token rows, "
+                      f"repeated {repeats} times ({t_raw:.1f} s of wall time on all cores), weighted by the "
+                      f"block's 4/2/1 layer counts"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph")
+    ap.add_argument("--skip-extras", action="store_true", help="skip the per-case table and the pack timing")
+    ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        args.steps = min(args.steps, 20)      # the oracle takes seconds per step
+        args.warmup = min(args.warmup, 3)
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
