@@ -145,6 +145,39 @@ slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* val
                                    void* y_dev, void* workspace, size_t workspace_bytes,
                                    uint32_t* status_dev, void* cuda_stream);
 
+/*
+ * Small-batch forward that allocates nothing.  (The paper has no counterpart:
+ * this entry point exists for the deployment constraint described here.)
+ *
+ * Some hosts of this library must not call cudaMalloc while they run: a serving
+ * loop that cannot afford the device-wide synchronisation an allocation causes,
+ * a plug-in living inside a runtime that has handed all device memory to its
+ * own pool, a process working under a fixed memory budget.  Such a caller
+ * cannot provide the workspace slim_linear_fwd asks for, so this variant keeps
+ * the decode kernel's scratch (split-K partial sums and barrier counters) in a
+ * fixed array of SLIM_NOALLOC_SCRATCH_BYTES inside the library's device image.
+ * Every GPU that loads the library holds that array until the process exits.
+ *
+ * Same operation, arguments and rounding as slim_linear_fwd, for b <= 16 and the
+ * shapes the decode kernel takes (d_in % 256 == 0); other problems return
+ * SLIM_ERR_UNSUPPORTED_SHAPE, and a problem whose scratch would exceed the
+ * array returns SLIM_ERR_WORKSPACE (all LLaMA-2 7B/13B/70B layer shapes fit).
+ * The call makes no cudaMalloc / cudaFree and uses no allocating library
+ * routine; inputs and outputs are still the caller's device buffers.
+ *
+ * The first call on a device looks up the array's device address (the device
+ * must be current); make that first call before starting any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's
+ * contents (the counters are cleared on the stream at the start of each call):
+ * two calls that overlap on the GPU - different streams, no ordering between
+ * them - race on it and produce garbage.  Issue them on one stream or order
+ * them with events.
+ */
+#define SLIM_NOALLOC_SCRATCH_BYTES (8u << 20)
+slim_status_t slim_linear_fwd_noalloc(const void* X, int b, const uint8_t* vals, const uint8_t* meta,
+                                      float s, const void* L, const void* R, int r, int d_out,
+                                      int d_in, void* Y, uint32_t* status_dev, void* cuda_stream);
+
 /* The kernel family slim_linear_fwd would pick for this problem. */
 slim_kernel_t slim_select_kernel(int b, int d_out, int d_in, int r);
 

@@ -21,6 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libslim.so")
 KERNEL_AUTO, KERNEL_SIMPLE, KERNEL_DECODE, KERNEL_PREFILL = range(4)
 KERNEL_NAMES = {KERNEL_AUTO: "auto", KERNEL_SIMPLE: "simple", KERNEL_DECODE: "decode", KERNEL_PREFILL: "prefill"}
 WORKSPACE_SYNC_BYTES = 256
+NOALLOC_SCRATCH_BYTES = 8 << 20
 
 # every symbol include/slim.h declares, with (restype, argtypes)
 _P, _I, _F, _SZ = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
@@ -32,6 +33,7 @@ SIGNATURES = {
     "slim_linear_fwd": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P]),
     "slim_linear_fwd_ex": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P, _I]),
     "slim_linear_fwd_host": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _P, _P, _SZ, _P, _P]),
+    "slim_linear_fwd_noalloc": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _P]),
     "slim_select_kernel": (_I, [_I, _I, _I, _I]),
     "slim_last_launch_count": (_I, []),
     "slim_strerror": (ctypes.c_char_p, [_I]),
@@ -192,3 +194,23 @@ def slim_linear_fwd_host(X_host: torch.Tensor, vals, meta, s: float, L, R, Y_hos
                                       _ptr(workspace), workspace.numel(), _ptr(status), _stream()),
            "slim_linear_fwd_host")
     return Y_host
+
+
+def slim_linear_fwd_noalloc(X, vals, meta, s: float, L, R, Y, status=None):
+    """Small-batch forward for callers that must not allocate device memory:
+    the library's built-in scratch array replaces the workspace, and ``Y`` has
+    to be supplied.  Calls on one device share that scratch, so keep them on one
+    stream (or order them); overlapping calls corrupt each other."""
+    _dev(X, torch.bfloat16, "X"), _dev(vals, torch.uint8, "vals"), _dev(meta, torch.uint8, "meta")
+    _dev(Y, torch.bfloat16, "Y")
+    b, d_in = X.shape
+    d_out = vals.shape[0]
+    r = 0 if L is None else L.shape[1]
+    if tuple(Y.shape) != (b, d_out) or vals.shape[1] * 4 != d_in or tuple(meta.shape) != (d_out, d_in // 8):
+        raise ValueError("shapes do not match")
+    if r and (tuple(L.shape) != (d_out, r) or tuple(R.shape) != (r, d_in)):
+        raise ValueError("adapter shapes do not match the weight")
+    _check(lib().slim_linear_fwd_noalloc(_ptr(X), b, _ptr(vals), _ptr(meta), float(s), _ptr(L) if r else None,
+                                         _ptr(R) if r else None, r, d_out, d_in, _ptr(Y), _ptr(status), _stream()),
+           "slim_linear_fwd_noalloc")
+    return Y
