@@ -173,7 +173,7 @@ slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* val
  * them - race on it and produce garbage.  Issue them on one stream or order
  * them with events.
  */
-#define SLIM_NOALLOC_SCRATCH_BYTES (8u << 20)
+#define SLIM_NOALLOC_SCRATCH_BYTES (16u << 20)
 slim_status_t slim_linear_fwd_noalloc(const void* X, int b, const uint8_t* vals, const uint8_t* meta,
                                       float s, const void* L, const void* R, int r, int d_out,
                                       int d_in, void* Y, uint32_t* status_dev, void* cuda_stream);

@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libslim.so")
 KERNEL_AUTO, KERNEL_SIMPLE, KERNEL_DECODE, KERNEL_PREFILL = range(4)
 KERNEL_NAMES = {KERNEL_AUTO: "auto", KERNEL_SIMPLE: "simple", KERNEL_DECODE: "decode", KERNEL_PREFILL: "prefill"}
 WORKSPACE_SYNC_BYTES = 256
-NOALLOC_SCRATCH_BYTES = 8 << 20
+NOALLOC_SCRATCH_BYTES = 16 << 20
 
 # every symbol include/slim.h declares, with (restype, argtypes)
 _P, _I, _F, _SZ = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t

@@ -1,55 +1,111 @@
 // Decode-phase forward (b <= 16): one persistent cooperative kernel that
 // streams the packed weight and the adapters from HBM exactly once.
 //
-// The batch is the N dimension of warp-level tensor-core MMAs (one or two
-// n-tiles of 8 tokens), so the kernel stays bandwidth-bound up to b = 16:
+// Tensor-core mapping.  The batch is the N dimension of warp-level MMAs (one or
+// two n-tiles of 8 tokens), so the kernel stays bandwidth-bound up to b = 16:
 //   * packed weight rows are the SPARSE A operand of
-//     mma.sp::ordered_metadata.m16n8k32 (bf16 x bf16 -> fp32): the library's
-//     value byte of one 2:4 group is exactly one thread's register pair and the
-//     index nibbles are the instruction's metadata, so decoding is nibble ->
-//     exact bf16 integer and nothing else;
-//   * adapter rows (R in phase 1, L in phase 2) are the dense A operand of
-//     mma.m16n8k16.
+//     mma.sp::ordered_metadata.m16n8k32 (bf16 x bf16 -> fp32): the value byte of
+//     one 2:4 group is exactly one thread's A-register pair and a 32-bit word of
+//     the index array is the instruction's metadata for one row, so decoding is
+//     nibble -> exact bf16 integer and nothing else;
+//   * adapter rows (R, then L) are the dense A operand of mma.m16n8k16; inside a
+//     32-column block the k order is permuted so that a thread's A and B
+//     fragments are single 16-byte reads.
 //
-// Work split.  d_in is cut into 256-wide k-blocks; a CTA owns one k-slice of up
-// to 8 blocks, one block per warp, and keeps that warp's activations as MMA B
-// fragments in registers for its whole life.  CTAs are divided into weight CTAs
-// and adapter (R) CTAs in proportion to the bytes each matrix streams.  A CTA
-// loops over 16-row tiles of its matrix; the 8 warps' partial tiles are summed
-// through shared memory and written to the workspace as split-K partials.
-// After one grid-wide barrier (bounded spin on a counter; the launch is
-// cooperative, so all CTAs are resident) every warp finishes 16-row output
-// tiles:  Y = s * sum(partials) + T L^T  with T = sum(partials of X R^T)
-// rounded once to bf16.  Reductions run in a fixed order: results are
-// bit-identical from run to run.
+// Data movement.  Every streamed operand travels HBM -> shared memory through
+// the bulk async copy engine (cp.async.bulk + mbarrier) into a ring of slots
+// (~200 KB in flight per SM), issued by a ninth, producer warp; the eight
+// consumer warps read fragments from shared memory.  Activations live in
+// registers as B fragments.
+//
+// Work split.  d_in is cut into 256-column blocks and into k-slices of <= 8
+// blocks; a CTA belongs to one slice.  Each CTA first takes its share of R
+// chunks (16 rows x 512 columns), then its share of 16-row weight tiles; both
+// leave split-K partial tiles (fp32, MMA fragment order) in the workspace.
+// Because every CTA does its R share first, T = X R^T is complete early: one
+// CTA per 16 columns of T sums the partials and rounds to bf16 while the weight
+// stream is still running (its ring keeps filling meanwhile).  After the weight
+// phase a grid-wide counter releases the last phase, in which every CTA
+// finishes 16-row output tiles:  Y = s * sum(partials) + T L^T, with the L
+// rows already prefetched into the ring.  All waits on other CTAs are bounded
+// spins (the launch is cooperative, so all CTAs are resident); an expired wait
+// sets SLIM_ERR_TIMEOUT and the kernel runs on to its end.  Reductions have a
+// fixed order: results are bit-identical from run to run.
 #include "common.cuh"
 
 namespace slim {
 
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kDecodeThreads = kConsumerThreads + 32;     // + producer warp
+constexpr int kMaxDecodeRank = 3072;
+constexpr int kMaxSlots = 16;
+constexpr uint32_t kSpinLimit = 1u << 22;                  // global counters (each poll sleeps >= 20 ns)
+constexpr uint32_t kMbarSpinLimit = 1u << 26;              // shared-memory barriers
+constexpr int kRChunkCols = 512;                           // columns of one R chunk
+constexpr int kLChunkCols = 512;                           // columns (of r) of one L chunk
+constexpr size_t kSmemBudget = 227 * 1024;
+
+// Synchronisation words in the first bytes of the workspace.
+enum { SYNC_R = 0, SYNC_T = 1, SYNC_W = 2, SYNC_DEPART = 3 };
+
 struct DecodeParams {
     const __nv_bfloat16* X; const uint8_t* vals; const uint8_t* meta;
     const __nv_bfloat16* L; const __nv_bfloat16* R; __nv_bfloat16* Y;
-    float* Ppart; float* Tpart; uint32_t* sync; uint32_t* status;
+    float* Ppart;              // [KS][tilesW][frag]
+    float* Tpart;              // [tilesR][QT][frag]
+    __nv_bfloat16* Tfinal;     // [NT*8][r_pad]
+    uint32_t* sync; uint32_t* status;
     float s;
     int b, r, d_out, d_in;
-    int KS, nblk, GW, GR, r_pad;
+    int KS, nblk, G, QT, r_pad;
+    int n_slots, slot_bytes;
+    int pitch_v, pitch_m, pitch_r, pitch_l;
 };
 
-constexpr int kDecodeThreads = 256;
-constexpr int kWarps = 8;
-constexpr int kMaxDecodeRank = 3072;
-constexpr uint32_t kSpinLimit = 1u << 22;
+// ------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(bar)), "r"(count));
 }
-
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase with the given parity; returns false on expiry.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t it = 0; it < kMbarSpinLimit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+// 1-D bulk copy global -> shared, completion counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void consumer_sync() {          // the eight consumer warps only
+    asm volatile("bar.sync 1, %0;" :: "n"(kConsumerThreads) : "memory");
+}
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint4 lds128(const void* p) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(p)));
     return v;
 }
 
@@ -64,7 +120,6 @@ __device__ __forceinline__ void mma_sp_16832(float* c, const uint32_t* a, const 
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]),
           "r"(bfrag[0]), "r"(bfrag[1]), "r"(bfrag[2]), "r"(bfrag[3]), "r"(e), "n"(SEL));
 }
-
 // D(16x8, fp32) += A(16x16 bf16) * B(16x8 bf16)
 __device__ __forceinline__ void mma_16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                           uint32_t b0, uint32_t b1) {
@@ -78,9 +133,9 @@ __device__ __forceinline__ void mma_16816(float* c, uint32_t a0, uint32_t a1, ui
 // Byte `t` of `w` holds one 2:4 group (two int4 codes).  Returns the two codes
 // as an exact bf16x2: nibble ^ 8 in the mantissa of 128.0 gives 128 + (v + 8);
 // subtracting 136 leaves v in [-8, 7].
-__device__ __forceinline__ uint32_t decode_group(uint32_t w, uint32_t w_shr4, uint32_t byte_sel) {
+__device__ __forceinline__ uint32_t decode_group(uint32_t w, uint32_t byte_sel) {
     uint32_t x;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(x) : "r"(w), "r"(w_shr4), "r"(byte_sel));
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(x) : "r"(w), "r"(w >> 4), "r"(byte_sel));
     uint32_t y;
     asm("lop3.b32 %0, %1, %2, %3, 0x6a;" : "=r"(y) : "r"(x), "r"(0x000F000Fu), "r"(0x43084308u));
     __nv_bfloat162 v = *reinterpret_cast<__nv_bfloat162*>(&y);
@@ -93,236 +148,429 @@ __device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
     return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
 }
 
-// Sum the warps' partial tiles and write one split-K partial (fragment order).
+// ------------------------------------------------------------ work split
+// Everything below is computed identically by the producer and the consumers.
+struct Share {
+    int ks, grp;             // k-slice and position inside the slice's CTA group (-1: no phase-1 work)
+    int blk_begin, nb;       // 256-column blocks of the slice
+    int Qk;                  // R chunks per 16-row R tile in this slice
+    int qoff;                // index of the slice's first chunk among a tile's QT partial slots
+    int r_begin, r_count;    // R chunk units [r_begin, r_begin + r_count)
+    int w_begin, w_count;    // weight tiles
+};
+
+__device__ __forceinline__ Share make_share(const DecodeParams& p, int cta) {
+    Share sh;
+    const int tilesW = p.d_out / 16, tilesR = p.r / 16;
+    if (cta >= p.KS * p.G) {
+        sh.ks = 0; sh.grp = -1; sh.blk_begin = 0; sh.nb = 0; sh.Qk = 0; sh.qoff = 0;
+        sh.r_begin = sh.r_count = sh.w_begin = sh.w_count = 0;
+        return sh;
+    }
+    sh.ks = cta % p.KS; sh.grp = cta / p.KS;
+    sh.blk_begin = (int)((long long)sh.ks * p.nblk / p.KS);
+    sh.nb = (int)((long long)(sh.ks + 1) * p.nblk / p.KS) - sh.blk_begin;
+    sh.Qk = (sh.nb + 1) / 2;
+    int qoff = 0;
+    for (int k = 0; k < sh.ks; ++k) {
+        const int nbk = (int)((long long)(k + 1) * p.nblk / p.KS) - (int)((long long)k * p.nblk / p.KS);
+        qoff += (nbk + 1) / 2;
+    }
+    sh.qoff = qoff;
+    // R chunks: the first CTAs of the group take the remainder; weight tiles: the last ones do
+    const int UR = tilesR * sh.Qk, G = p.G;
+    sh.r_count = UR / G + (sh.grp < UR % G ? 1 : 0);
+    sh.r_begin = sh.grp * (UR / G) + (sh.grp < UR % G ? sh.grp : UR % G);
+    const int rem = tilesW % G;
+    sh.w_count = tilesW / G + (sh.grp >= G - rem ? 1 : 0);
+    sh.w_begin = sh.grp * (tilesW / G) + (sh.grp > G - rem ? sh.grp - (G - rem) : 0);
+    return sh;
+}
+
+// Sum the consumer warps' partial tiles (fragment order) through shared memory.
 template <int NT>
-__device__ __forceinline__ void reduce_and_store(float (*red)[NT * 128], const float (&acc)[NT][4],
-                                                 bool active, int nb, float* dst)
-{
+__device__ __forceinline__ float block_tile_sum(float* red, const float (&acc)[NT][4], bool active, int n_active) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int frag = NT * 128;
     if (active) {
 #pragma unroll
         for (int h = 0; h < NT; ++h)
 #pragma unroll
-            for (int q = 0; q < 4; ++q) red[warp][(h * 4 + q) * 32 + lane] = acc[h][q];
+            for (int q = 0; q < 4; ++q) red[warp * frag + (h * 4 + q) * 32 + lane] = acc[h][q];
     }
-    __syncthreads();
-    if (threadIdx.x < NT * 128) {
-        float sum = 0.f;
-        for (int w = 0; w < nb; ++w) sum += red[w][threadIdx.x];
-        dst[threadIdx.x] = sum;
-    }
-    __syncthreads();
+    consumer_sync();
+    float sum = 0.f;
+    if (threadIdx.x < frag)
+        for (int w = 0; w < n_active; ++w) sum += red[w * frag + threadIdx.x];
+    return sum;
 }
 
 template <int NT>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
 decode_kernel(const DecodeParams p)
 {
-    __shared__ float red[kWarps][NT * 128];
-    extern __shared__ uint4 dyn_smem[];
-    __nv_bfloat16* Ts = reinterpret_cast<__nv_bfloat16*>(dyn_smem);   // [NT*8][r_pad]
+    constexpr int frag = NT * 128;
+    extern __shared__ __align__(128) unsigned char smem[];
+    // layout: ring slots | Ts | red (two buffers) | barriers | flags
+    unsigned char* ring = smem;
+    __nv_bfloat16* Ts = reinterpret_cast<__nv_bfloat16*>(ring + (size_t)p.n_slots * p.slot_bytes);
+    float* red_base = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(Ts) + (size_t)NT * 8 * p.r_pad * 2);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(red_base + 2 * kConsumerWarps * frag);
+    uint64_t* empty_bar = full_bar + kMaxSlots;
+    volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(empty_bar + kMaxSlots);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
     const int tilesW = p.d_out / 16, tilesR = p.r / 16;
-    const int frag = NT * 128;
+    const int n_ctas = gridDim.x;
+    const Share sh = make_share(p, blockIdx.x);
+    const int n_slots = p.n_slots;
+    const int l_chunks = p.r > 0 ? ceil_div(p.r, kLChunkCols) : 0;
+    const size_t vstride = (size_t)p.d_in / 4, mstride = (size_t)p.d_in / 8;
+    const int pitch_m = p.pitch_m;
 
-    // ------------------------------------------------------------ phase 1
-    {
-        const int cta = blockIdx.x;
-        const int nW = p.KS * p.GW;
-        const bool wrole = cta < nW;
-        const int c2 = wrole ? cta : cta - nW;
-        const int ks = c2 % p.KS, grp = c2 / p.KS;
-        const int blk_begin = (int)((long long)ks * p.nblk / p.KS);
-        const int nb = (int)((long long)(ks + 1) * p.nblk / p.KS) - blk_begin;
-        const bool active = warp < nb;
-        const size_t kbase = (size_t)(blk_begin + warp) * 256;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < n_slots; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], kConsumerWarps); }
+        flags[0] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
 
-        if (wrole) {
-            // activations as sparse-MMA B fragments: step j, n-tile h, register i
-            // holds X[g + 8h][kbase + 32j + 2t + 8i .. +1]
-            uint32_t xf[8][NT][4];
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-#pragma unroll
-                for (int h = 0; h < NT; ++h)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int row = g + 8 * h;
-                        xf[j][h][i] = (active && row < p.b)
-                            ? __ldg(reinterpret_cast<const uint32_t*>(p.X + (size_t)row * p.d_in + kbase + 32 * j + 2 * t + 8 * i))
-                            : 0u;
-                    }
-            const uint32_t byte_sel = (uint32_t)t * 0x1111u + 0x4400u;   // bytes {t, t, 4+t, 4+t}
-            const uint32_t meta_sel = (t & 1) ? 0x7632u : 0x5410u;
-            const size_t vstride = (size_t)p.d_in / 4, mstride = (size_t)p.d_in / 8;
-            for (int tile = grp; tile < tilesW; tile += p.GW) {
-                float acc[NT][4];
-#pragma unroll
-                for (int h = 0; h < NT; ++h)
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) acc[h][q] = 0.f;
-                if (active) {
-                    const size_t row0 = (size_t)tile * 16 + g, row1 = row0 + 8;
-                    const uint8_t* v0p = p.vals + row0 * vstride + (kbase >> 2);
-                    const uint8_t* v1p = p.vals + row1 * vstride + (kbase >> 2);
-                    uint4 v0[4], v1[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) { v0[i] = ldg_stream(v0p + 16 * i); v1[i] = ldg_stream(v1p + 16 * i); }
-                    // the metadata of steps 0-3 is supplied by threads 0,1 of a quad,
-                    // that of steps 4-7 by threads 2,3: each loads its own 16 bytes
-                    const uint4 m0 = ldg_stream(p.meta + row0 * mstride + (kbase >> 3) + 16 * (t >> 1));
-                    const uint4 m1 = ldg_stream(p.meta + row1 * mstride + (kbase >> 3) + 16 * (t >> 1));
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t w0a = word_of(v0[j >> 1], (2 * j) & 3), w0b = word_of(v0[j >> 1], (2 * j + 1) & 3);
-                        const uint32_t w1a = word_of(v1[j >> 1], (2 * j) & 3), w1b = word_of(v1[j >> 1], (2 * j + 1) & 3);
-                        uint32_t a[4];
-                        a[0] = decode_group(w0a, w0a >> 4, byte_sel);
-                        a[1] = decode_group(w1a, w1a >> 4, byte_sel);
-                        a[2] = decode_group(w0b, w0b >> 4, byte_sel);
-                        a[3] = decode_group(w1b, w1b >> 4, byte_sel);
-                        // metadata word: low half = row g, high half = row g+8, 16 columns each
-                        uint32_t e;
-                        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(e)
-                            : "r"(word_of(m0, j & 3)), "r"(word_of(m1, j & 3)), "r"(meta_sel));
-#pragma unroll
-                        for (int h = 0; h < NT; ++h) {
-                            if (j < 4) mma_sp_16832<0>(acc[h], a, xf[j][h], e);
-                            else       mma_sp_16832<1>(acc[h], a, xf[j][h], e);
-                        }
-                    }
-                }
-                reduce_and_store<NT>(red, acc, active, nb, p.Ppart + ((size_t)ks * tilesW + tile) * frag);
+    if (warp == kConsumerWarps) {
+        // ============================ producer warp ============================
+        uint32_t it = 0;
+        bool ok = true;
+        auto acquire = [&](uint32_t bytes) -> int {
+            const int slot = it % n_slots;
+            if (it >= (uint32_t)n_slots) {
+                if (lane == 0) ok = mbar_wait(&empty_bar[slot], ((it / n_slots) & 1) ^ 1) && ok;
             }
-        } else {
-            // activations as dense-MMA B fragments: block jj (32 columns), n-tile h:
-            // 16 bytes X[g + 8h][kbase + 32jj + 8t .. +8)
-            uint4 xd[8][NT];
+            if (lane == 0) mbar_arrive_expect_tx(&full_bar[slot], bytes);
+            __syncwarp();
+            ++it;
+            return slot;
+        };
+        // ---- R chunks: 16 rows x (256 or 512) columns of bf16
+        for (int u = sh.r_begin; u < sh.r_begin + sh.r_count; ++u) {
+            const int tile = u / sh.Qk, q = u % sh.Qk;
+            const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
+            const uint32_t row_bytes = (uint32_t)cols * 2;
+            const int slot = acquire(16 * row_bytes);
+            if (lane < 16) {
+                const __nv_bfloat16* src = p.R + ((size_t)tile * 16 + lane) * p.d_in + (size_t)sh.blk_begin * 256 + (size_t)q * kRChunkCols;
+                bulk_g2s(ring + (size_t)slot * p.slot_bytes + (size_t)lane * p.pitch_r, src, row_bytes, &full_bar[slot]);
+            }
+        }
+        // ---- weight tiles: 16 rows of value bytes, then 16 rows of index bytes
+        for (int tile = sh.w_begin; tile < sh.w_begin + sh.w_count; ++tile) {
+            const uint32_t vbytes = (uint32_t)sh.nb * 64, mbytes = (uint32_t)sh.nb * 32;
+            const int slot = acquire(16 * (vbytes + mbytes));
+            unsigned char* base = ring + (size_t)slot * p.slot_bytes;
+            const size_t row = (size_t)tile * 16 + (lane & 15);
+            if (lane < 16)
+                bulk_g2s(base + (size_t)lane * p.pitch_v, p.vals + row * vstride + (size_t)sh.blk_begin * 64, vbytes, &full_bar[slot]);
+            else
+                bulk_g2s(base + 16 * (size_t)p.pitch_v + (size_t)(lane - 16) * pitch_m,
+                         p.meta + row * mstride + (size_t)sh.blk_begin * 32, mbytes, &full_bar[slot]);
+        }
+        // ---- L chunks of the output tiles this CTA finishes
+        for (int tile = blockIdx.x; tile < tilesW && p.r > 0; tile += n_ctas) {
+            for (int lc = 0; lc < l_chunks; ++lc) {
+                const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
+                const uint32_t row_bytes = (uint32_t)cols * 2;
+                const int slot = acquire(16 * row_bytes);
+                if (lane < 16) {
+                    const __nv_bfloat16* src = p.L + ((size_t)tile * 16 + lane) * p.r + (size_t)lc * kLChunkCols;
+                    bulk_g2s(ring + (size_t)slot * p.slot_bytes + (size_t)lane * p.pitch_l, src, row_bytes, &full_bar[slot]);
+                }
+            }
+        }
+        if (lane == 0 && !ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
+        return;      // consumers wait for every copy this warp issued before they leave
+    }
+
+    // ================================ consumer warps ================================
+    uint32_t it = 0;
+    int red_buf = 0;
+    bool ok = true;
+    auto wait_full = [&]() -> int {
+        const int slot = it % n_slots;
+        ok = mbar_wait(&full_bar[slot], (it / n_slots) & 1) && ok;
+        return slot;
+    };
+    auto release = [&](int slot) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[slot]);
+        ++it;
+    };
+    auto next_red = [&]() -> float* {
+        float* r = red_base + red_buf * kConsumerWarps * frag;
+        red_buf ^= 1;
+        return r;
+    };
+    // Release pattern for a grid-wide counter: all stores of the CTA, then one add.
+    auto arrive_counter = [&](int which, uint32_t n) {
+        consumer_sync();
+        if (threadIdx.x == 0) { __threadfence(); atomicAdd(&p.sync[which], n); }
+    };
+    // Thread 0 polls, the result is broadcast to the consumer warps.
+    auto counter_reached = [&](int which, uint32_t target, bool blocking) -> bool {
+        if (threadIdx.x == 0) {
+            bool reached = false;
+            const uint32_t limit = blocking ? kSpinLimit : 1u;
+            for (uint32_t i = 0; i < limit; ++i) {
+                if (ld_acquire(&p.sync[which]) >= target) { reached = true; break; }
+                if (blocking) __nanosleep(20);
+            }
+            if (blocking && !reached) flag_error(p.status, SLIM_ERR_TIMEOUT);
+            flags[0] = (reached || blocking) ? 1u : 0u;
+            __threadfence_block();
+        }
+        consumer_sync();
+        const bool res = flags[0] != 0;
+        consumer_sync();
+        return res;
+    };
+
+    // ---------------------------------------------------------------- phase R
+    if (sh.r_count > 0) {
+        // activations as dense B fragments: chunk q, sub-block jj (32 columns), n-tile h:
+        // 16 bytes X[g + 8h][slice + 512 q + 64 warp + 32 jj + 8 t .. +8)
+        uint4 xd[4][2][NT];
 #pragma unroll
-            for (int jj = 0; jj < 8; ++jj)
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int h = 0; h < NT; ++h) {
                     const int row = g + 8 * h;
-                    xd[jj][h] = (active && row < p.b)
-                        ? __ldg(reinterpret_cast<const uint4*>(p.X + (size_t)row * p.d_in + kbase + 32 * jj + 8 * t))
+                    const int col = q * kRChunkCols + warp * 64 + jj * 32;
+                    xd[q][jj][h] = (col < sh.nb * 256 && row < p.b)
+                        ? __ldg(reinterpret_cast<const uint4*>(p.X + (size_t)row * p.d_in + (size_t)sh.blk_begin * 256 + col + 8 * t))
                         : make_uint4(0, 0, 0, 0);
                 }
-            for (int tile = grp; tile < tilesR; tile += p.GR) {
-                float acc[NT][4];
+        for (int u = sh.r_begin; u < sh.r_begin + sh.r_count; ++u) {
+            const int tile = u / sh.Qk, q = u % sh.Qk;
+            const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
+            const bool active = warp * 64 < cols;
+            const int slot = wait_full();
+            float acc[NT][4];
 #pragma unroll
-                for (int h = 0; h < NT; ++h)
+            for (int h = 0; h < NT; ++h)
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) acc[h][q] = 0.f;
-                if (active) {
-                    const __nv_bfloat16* r0 = p.R + ((size_t)tile * 16 + g) * p.d_in + kbase + 8 * t;
-                    const __nv_bfloat16* r1 = r0 + (size_t)8 * p.d_in;
+                for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
+            if (active) {
+                const unsigned char* base = ring + (size_t)slot * p.slot_bytes + warp * 128 + t * 16;
+                uint4 ra[2], rb[2];
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint4 ra[4], rb[4];
+                for (int jj = 0; jj < 2; ++jj) {
+                    ra[jj] = lds128(base + (size_t)g * p.pitch_r + jj * 64);
+                    rb[jj] = lds128(base + (size_t)(g + 8) * p.pitch_r + jj * 64);
+                }
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            ra[i] = ldg_stream(r0 + 32 * (4 * half + i));
-                            rb[i] = ldg_stream(r1 + 32 * (4 * half + i));
-                        }
+                for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
+                    for (int h = 0; h < NT; ++h) {
+                        // the chunk index is not a compile-time constant: select the fragment set
+                        uint4 xb = xd[0][jj][h];
+                        if (q == 1) xb = xd[1][jj][h];
+                        if (q == 2) xb = xd[2][jj][h];
+                        if (q == 3) xb = xd[3][jj][h];
+                        mma_16816(acc[h], ra[jj].x, rb[jj].x, ra[jj].y, rb[jj].y, xb.x, xb.y);
+                        mma_16816(acc[h], ra[jj].z, rb[jj].z, ra[jj].w, rb[jj].w, xb.z, xb.w);
+                    }
+            }
+            release(slot);
+            const float sum = block_tile_sum<NT>(next_red(), acc, active, min(kConsumerWarps, cols / 64));
+            if (threadIdx.x < frag)
+                p.Tpart[((size_t)tile * p.QT + sh.qoff + q) * frag + threadIdx.x] = sum;
+        }
+    }
+    if (p.r > 0) arrive_counter(SYNC_R, 1);
+
+    // T reduction duty: CTA c owns the 16-column pieces jt = c, c + n_ctas, ...
+    bool t_pending = p.r > 0 && (int)blockIdx.x < tilesR;
+    auto reduce_t = [&]() {
+        for (int jt = blockIdx.x; jt < tilesR; jt += n_ctas) {
+            if (threadIdx.x < frag) {
+                const float* src = p.Tpart + (size_t)jt * p.QT * frag + threadIdx.x;
+                float sum = 0.f;
+#pragma unroll 8
+                for (int sl = 0; sl < p.QT; ++sl) sum += __ldcg(src + (size_t)sl * frag);
+                const int hq = threadIdx.x >> 5, ln = threadIdx.x & 31;
+                const int h = hq >> 2, q = hq & 3;
+                const int j = jt * 16 + (ln >> 2) + 8 * (q >> 1);
+                const int m = 8 * h + 2 * (ln & 3) + (q & 1);
+                p.Tfinal[(size_t)m * p.r_pad + j] = __float2bfloat16_rn(sum);
+            }
+        }
+        int mine = 0;
+        for (int jt = blockIdx.x; jt < tilesR; jt += n_ctas) ++mine;
+        arrive_counter(SYNC_T, (uint32_t)mine);
+        t_pending = false;
+    };
+
+    // ---------------------------------------------------------------- phase W
+    if (sh.w_count > 0) {
+        // activations as sparse B fragments: step j, n-tile h, register i holds
+        // X[g + 8h][slice + 256 warp + 32 j + 2 t + 8 i .. +1]
+        const bool active = warp < sh.nb;
+        uint32_t xf[8][NT][4];
 #pragma unroll
-                            for (int h = 0; h < NT; ++h) {
-                                const uint4 xb = xd[4 * half + i][h];
-                                mma_16816(acc[h], ra[i].x, rb[i].x, ra[i].y, rb[i].y, xb.x, xb.y);
-                                mma_16816(acc[h], ra[i].z, rb[i].z, ra[i].w, rb[i].w, xb.z, xb.w);
-                            }
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int h = 0; h < NT; ++h)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = g + 8 * h;
+                    xf[j][h][i] = (active && row < p.b)
+                        ? __ldg(reinterpret_cast<const uint32_t*>(p.X + (size_t)row * p.d_in + (size_t)(sh.blk_begin + warp) * 256 + 32 * j + 2 * t + 8 * i))
+                        : 0u;
+                }
+        const uint32_t byte_sel = (uint32_t)t * 0x1111u + 0x4400u;   // bytes {t, t, 4+t, 4+t}
+        const uint32_t meta_sel = (t & 1) ? 0x7632u : 0x5410u;
+        // the CTAs with reduction duty look at the R counter once per tile; the load is
+        // issued one tile ahead so that its latency is never waited for
+        uint32_t polled = 0;
+        if (t_pending && threadIdx.x == 0) polled = ld_acquire(&p.sync[SYNC_R]);
+        for (int tile = sh.w_begin; tile < sh.w_begin + sh.w_count; ++tile) {
+            if (t_pending) {
+                if (threadIdx.x == 0) flags[0] = polled >= (uint32_t)n_ctas ? 1u : 0u;
+                consumer_sync();
+                const bool ready = flags[0] != 0;
+                consumer_sync();
+                if (ready) reduce_t();
+                else if (threadIdx.x == 0) polled = ld_acquire(&p.sync[SYNC_R]);
+            }
+            const int slot = wait_full();
+            float acc[NT][4];
+#pragma unroll
+            for (int h = 0; h < NT; ++h)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
+            if (active) {
+                const unsigned char* base = ring + (size_t)slot * p.slot_bytes;
+                const unsigned char* v0p = base + (size_t)g * p.pitch_v + warp * 64;
+                const unsigned char* v1p = v0p + 8 * (size_t)p.pitch_v;
+                const unsigned char* mbase = base + 16 * (size_t)p.pitch_v + warp * 32 + 16 * (t >> 1);
+                uint4 v0[4], v1[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { v0[i] = lds128(v0p + 16 * i); v1[i] = lds128(v1p + 16 * i); }
+                // index words of steps 0-3 come from threads 0,1 of a quad, of steps 4-7 from threads 2,3
+                const uint4 m0 = lds128(mbase + (size_t)g * pitch_m);
+                const uint4 m1 = lds128(mbase + (size_t)(g + 8) * pitch_m);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t a[4];
+                    a[0] = decode_group(word_of(v0[j >> 1], (2 * j) & 3), byte_sel);
+                    a[1] = decode_group(word_of(v1[j >> 1], (2 * j) & 3), byte_sel);
+                    a[2] = decode_group(word_of(v0[j >> 1], (2 * j + 1) & 3), byte_sel);
+                    a[3] = decode_group(word_of(v1[j >> 1], (2 * j + 1) & 3), byte_sel);
+                    // metadata word: low half = row g, high half = row g+8, 16 columns each
+                    uint32_t e;
+                    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(e)
+                        : "r"(word_of(m0, j & 3)), "r"(word_of(m1, j & 3)), "r"(meta_sel));
+#pragma unroll
+                    for (int h = 0; h < NT; ++h) {
+                        if (j < 4) mma_sp_16832<0>(acc[h], a, xf[j][h], e);
+                        else       mma_sp_16832<1>(acc[h], a, xf[j][h], e);
                     }
                 }
-                reduce_and_store<NT>(red, acc, active, nb, p.Tpart + ((size_t)ks * tilesR + tile) * frag);
             }
+            release(slot);
+            const float sum = block_tile_sum<NT>(next_red(), acc, active, sh.nb);
+            if (threadIdx.x < frag)
+                p.Ppart[((size_t)sh.ks * tilesW + tile) * frag + threadIdx.x] = sum;
         }
     }
+    arrive_counter(SYNC_W, 1);
 
-    // ------------------------------------------------- grid-wide barrier
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(&p.sync[0], 1u);
-        bool ok = false;
-        for (uint32_t it = 0; it < kSpinLimit; ++it) {
-            if (ld_acquire(&p.sync[0]) >= gridDim.x) { ok = true; break; }
-            __nanosleep(20);
-        }
-        if (!ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
-        __threadfence();
-        // the last CTA to leave puts the counters back to zero for the next call
-        if (atomicAdd(&p.sync[1], 1u) == gridDim.x - 1) {
-            p.sync[0] = 0u;
-            p.sync[1] = 0u;
-            __threadfence();
-        }
-    }
-    __syncthreads();
-
-    // ------------------------------------------------------------ phase 2
-    const int r_pad = p.r_pad;
+    // ------------------------------------------------ T: finish, then fetch
     if (p.r > 0) {
-        // T = sum over k-slices of the X R^T partials, rounded to bf16, as
-        // Ts[token][j]; columns r .. r_pad are zero
-        for (int idx = threadIdx.x; idx < NT * 8 * (r_pad - p.r); idx += kDecodeThreads) {
-            const int m = idx / (r_pad - p.r), j = p.r + idx % (r_pad - p.r);
-            Ts[m * r_pad + j] = __float2bfloat16_rn(0.f);
-        }
-        for (int idx = threadIdx.x; idx < tilesR * frag; idx += kDecodeThreads) {
-            const int jt = idx / frag, f = idx % frag;
-            float sum = 0.f;
-            for (int ks = 0; ks < p.KS; ++ks) sum += __ldcg(p.Tpart + ((size_t)ks * tilesR + jt) * frag + f);
-            const int hq = f >> 5, ln = f & 31;
-            const int h = hq >> 2, q = hq & 3;
-            const int j = jt * 16 + (ln >> 2) + 8 * (q >> 1);
-            const int m = 8 * h + 2 * (ln & 3) + (q & 1);
-            Ts[m * r_pad + j] = __float2bfloat16_rn(sum);
+        if (t_pending) { counter_reached(SYNC_R, (uint32_t)n_ctas, true); reduce_t(); }
+        counter_reached(SYNC_T, (uint32_t)tilesR, true);
+        const int rp = p.r_pad;
+        for (int idx = threadIdx.x; idx < NT * 8 * (rp / 8); idx += kConsumerThreads) {
+            const int m = idx / (rp / 8), c8 = (idx % (rp / 8)) * 8;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (c8 < p.r) v = __ldcg(reinterpret_cast<const uint4*>(p.Tfinal + (size_t)m * rp + c8));
+            *reinterpret_cast<uint4*>(Ts + (size_t)m * rp + c8) = v;
         }
     }
-    __syncthreads();
+    counter_reached(SYNC_W, (uint32_t)n_ctas, true);      // ends with a consumer_sync: Ts is visible
 
-    for (int tile = blockIdx.x * kWarps + warp; tile < tilesW; tile += gridDim.x * kWarps) {
-        float acc[NT][4];
+    // ---------------------------------------------------------------- phase Y
+    for (int tile = blockIdx.x; tile < tilesW; tile += n_ctas) {
+        float psum = 0.f;
+        if (threadIdx.x < frag) {
+            const float* src = p.Ppart + (size_t)tile * frag + threadIdx.x;
+#pragma unroll 4
+            for (int ks = 0; ks < p.KS; ++ks) psum += __ldcg(src + (size_t)ks * tilesW * frag);
+        }
+        float ysum = 0.f;
+        for (int lc = 0; lc < l_chunks; ++lc) {
+            const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
+            const int slot = wait_full();
+            float acc[NT][4];
 #pragma unroll
-        for (int h = 0; h < NT; ++h)
+            for (int h = 0; h < NT; ++h)
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                float sum = 0.f;
-                for (int ks = 0; ks < p.KS; ++ks)
-                    sum += __ldcg(p.Ppart + ((size_t)ks * tilesW + tile) * frag + (h * 4 + q) * 32 + lane);
-                acc[h][q] = sum * p.s;
-            }
-        if (p.r > 0) {
-            const __nv_bfloat16* l0 = p.L + ((size_t)tile * 16 + g) * p.r + 8 * t;
-            const __nv_bfloat16* l1 = l0 + (size_t)8 * p.r;
-            for (int jj = 0; jj < r_pad / 32; ++jj) {
-                const int kk = 32 * jj + 8 * t;
-                uint4 la = make_uint4(0, 0, 0, 0), lb = la;
-                if (kk < p.r) { la = ldg_stream(l0 + 32 * jj); lb = ldg_stream(l1 + 32 * jj); }
+                for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
+            const unsigned char* base = ring + (size_t)slot * p.slot_bytes;
 #pragma unroll
-                for (int h = 0; h < NT; ++h) {
-                    const uint4 tb = *reinterpret_cast<const uint4*>(Ts + (g + 8 * h) * r_pad + kk);
-                    mma_16816(acc[h], la.x, lb.x, la.y, lb.y, tb.x, tb.y);
-                    mma_16816(acc[h], la.z, lb.z, la.w, lb.w, tb.z, tb.w);
+            for (int rep = 0; rep < 2; ++rep) {
+                const int kk = 32 * (warp + 8 * rep) + 8 * t;       // column inside the chunk
+                if (32 * (warp + 8 * rep) < cols) {
+                    uint4 la = make_uint4(0, 0, 0, 0), lb = la;
+                    if (kk < cols) {
+                        la = lds128(base + (size_t)g * p.pitch_l + kk * 2);
+                        lb = lds128(base + (size_t)(g + 8) * p.pitch_l + kk * 2);
+                    }
+#pragma unroll
+                    for (int h = 0; h < NT; ++h) {
+                        const uint4 tb = lds128(Ts + (size_t)(g + 8 * h) * p.r_pad + lc * kLChunkCols + kk);
+                        mma_16816(acc[h], la.x, lb.x, la.y, lb.y, tb.x, tb.y);
+                        mma_16816(acc[h], la.z, lb.z, la.w, lb.w, tb.z, tb.w);
+                    }
                 }
             }
+            release(slot);
+            ysum += block_tile_sum<NT>(next_red(), acc, true, kConsumerWarps);
         }
-#pragma unroll
-        for (int h = 0; h < NT; ++h)
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int m = 8 * h + 2 * t + (q & 1);
-                const int n = tile * 16 + g + 8 * (q >> 1);
-                if (m < p.b) p.Y[(size_t)m * p.d_out + n] = __float2bfloat16_rn(acc[h][q]);
-            }
+        if (threadIdx.x < frag) {
+            const int hq = threadIdx.x >> 5, ln = threadIdx.x & 31;
+            const int h = hq >> 2, q = hq & 3;
+            const int n = tile * 16 + (ln >> 2) + 8 * (q >> 1);
+            const int m = 8 * h + 2 * (ln & 3) + (q & 1);
+            if (m < p.b) p.Y[(size_t)m * p.d_out + n] = __float2bfloat16_rn(fmaf(psum, p.s, ysum));
+        }
+    }
+
+    // the last CTA to leave puts the counters back to zero for the next call
+    if (threadIdx.x == 0) {
+        if (!ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
+        __threadfence();
+        if (atomicAdd(&p.sync[SYNC_DEPART], 1u) == (uint32_t)n_ctas - 1) {
+            p.sync[SYNC_R] = 0u; p.sync[SYNC_T] = 0u; p.sync[SYNC_W] = 0u; p.sync[SYNC_DEPART] = 0u;
+            __threadfence();
+        }
+    } else if (!ok && lane == 0) {
+        flag_error(p.status, SLIM_ERR_TIMEOUT);
     }
 }
 
 // ------------------------------------------------------------------ host side
-struct DecodePlan { int KS, nblk, GW, GR, r_pad, nt; size_t p_bytes, t_bytes, smem; };
+struct DecodePlan {
+    int nt, KS, nblk, G, QT, r_pad, n_slots, slot_bytes;
+    int pitch_v, pitch_m, pitch_r, pitch_l;
+    size_t p_bytes, tpart_bytes, tfinal_bytes, smem;
+};
+
+static int pitch_64mod128(int bytes) {           // smallest pitch >= bytes with pitch % 128 == 64
+    int p = (bytes + 127) / 128 * 128 + 64;
+    if (p - 128 >= bytes) p -= 128;
+    return p;
+}
 
 static int pad_rank(int r) {
     if (r == 0) return 0;
@@ -331,45 +579,56 @@ static int pad_rank(int r) {
     return rp;
 }
 
-static bool make_plan(int b, int d_out, int d_in, int r, int ctas, DecodePlan* pl) {
-    if (b < 1 || b > 16 || d_in % 256 != 0 || d_out % 16 != 0 || r % 16 != 0 || r > kMaxDecodeRank) return false;
-    pl->nt = b <= 8 ? 1 : 2;
-    pl->nblk = d_in / 256;
-    pl->KS = ceil_div(pl->nblk, kWarps);
-    int G = ctas / pl->KS;
-    if (G < (r > 0 ? 2 : 1)) return false;
-    const int tilesW = d_out / 16, tilesR = r / 16;
-    if (r > 0) {
-        const double bytesR = 2.0 * r * d_in, bytesW = 0.375 * (double)d_out * d_in;
-        int GR = (int)(G * bytesR / (bytesR + bytesW) + 0.5);
-        if (GR < 1) GR = 1;
-        if (GR > G - 1) GR = G - 1;
-        if (GR > tilesR) GR = tilesR;
-        int GW = G - GR;
-        if (GW > tilesW) GW = tilesW;
-        pl->GR = GR; pl->GW = GW;
-    } else {
-        pl->GR = 0; pl->GW = G < tilesW ? G : tilesW;
-    }
-    pl->r_pad = pad_rank(r);
-    const size_t frag = (size_t)pl->nt * 128 * sizeof(float);
-    pl->p_bytes = (size_t)pl->KS * tilesW * frag;
-    pl->t_bytes = (size_t)pl->KS * tilesR * frag;
-    pl->smem = (size_t)pl->nt * 8 * pl->r_pad * sizeof(__nv_bfloat16);
-    return true;
+static bool shape_ok(int b, int d_out, int d_in, int r) {
+    return b >= 1 && b <= 16 && d_in % 256 == 0 && d_out % 16 == 0 && r % 16 == 0 && r >= 0 && r <= kMaxDecodeRank;
 }
 
-constexpr size_t kDecodeMaxDynSmem = 16 * (size_t)(kMaxDecodeRank + 64) * 2;
+static bool make_plan(int b, int d_out, int d_in, int r, int ctas, DecodePlan* pl) {
+    if (!shape_ok(b, d_out, d_in, r)) return false;
+    pl->nt = b <= 8 ? 1 : 2;
+    pl->nblk = d_in / 256;
+    pl->KS = ceil_div(pl->nblk, kConsumerWarps);
+    pl->G = ctas / pl->KS;
+    if (pl->G < 1) return false;
+    int qt = 0, nb_max = 0;
+    for (int k = 0; k < pl->KS; ++k) {
+        const int nbk = (int)((long long)(k + 1) * pl->nblk / pl->KS) - (int)((long long)k * pl->nblk / pl->KS);
+        qt += (nbk + 1) / 2;
+        if (nbk > nb_max) nb_max = nbk;
+    }
+    pl->QT = qt;
+    pl->r_pad = pad_rank(r);
+    pl->pitch_v = 64 * nb_max + 16;
+    pl->pitch_m = 32 * nb_max + (nb_max % 2 == 0 ? 32 : 0);     // 32 modulo 64: rows g, g+1 never share banks
+    pl->pitch_r = pitch_64mod128((nb_max >= 2 ? kRChunkCols : 256) * 2);
+    pl->pitch_l = r > 0 ? pitch_64mod128((r < kLChunkCols ? r : kLChunkCols) * 2) : 0;
+    int slot = 16 * pl->pitch_v + 16 * pl->pitch_m;
+    if (r > 0) {
+        if (16 * pl->pitch_r > slot) slot = 16 * pl->pitch_r;
+        if (16 * pl->pitch_l > slot) slot = 16 * pl->pitch_l;
+    }
+    pl->slot_bytes = (slot + 127) / 128 * 128;
+    const size_t frag = (size_t)pl->nt * 128 * sizeof(float);
+    const size_t fixed = (size_t)pl->nt * 8 * pl->r_pad * 2 + 2 * kConsumerWarps * frag + 2 * kMaxSlots * 8 + 64;
+    if (fixed + 2 * (size_t)pl->slot_bytes > kSmemBudget) return false;
+    int n = (int)((kSmemBudget - fixed) / pl->slot_bytes);
+    pl->n_slots = n > kMaxSlots ? kMaxSlots : n;
+    pl->smem = (size_t)pl->n_slots * pl->slot_bytes + fixed;
+    pl->p_bytes = (size_t)pl->KS * (d_out / 16) * frag;
+    pl->tpart_bytes = (size_t)(r / 16) * pl->QT * frag;
+    pl->tfinal_bytes = ((size_t)pl->nt * 8 * pl->r_pad * 2 + 255) / 256 * 256;
+    return true;
+}
 
 int decode_query_residency(int nt) {
     int n = 0;
     cudaError_t e1, e2;
     if (nt == 1) {
-        e1 = cudaFuncSetAttribute(decode_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecodeMaxDynSmem);
-        e2 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<1>, kDecodeThreads, kDecodeMaxDynSmem);
+        e1 = cudaFuncSetAttribute(decode_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+        e2 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<1>, kDecodeThreads, kSmemBudget);
     } else {
-        e1 = cudaFuncSetAttribute(decode_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecodeMaxDynSmem);
-        e2 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<2>, kDecodeThreads, kDecodeMaxDynSmem);
+        e1 = cudaFuncSetAttribute(decode_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+        e2 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<2>, kDecodeThreads, kSmemBudget);
     }
     if (e1 != cudaSuccess || e2 != cudaSuccess) return 0;
     return n > 1 ? 1 : n;      // one CTA per SM: the plan sizes the grid for that
@@ -389,11 +648,10 @@ bool decode_supports(int b, int d_out, int d_in, int r) {
 }
 
 size_t decode_workspace_bytes(int b, int d_out, int d_in, int r) {
-    // split-K partial tiles; depends on the shape only, not on the device
-    if (b < 1 || b > 16 || d_in % 256 != 0 || d_out % 16 != 0 || r % 16 != 0 || r > kMaxDecodeRank) return 0;
-    const size_t frag = (size_t)(b <= 8 ? 1 : 2) * 128 * sizeof(float);
-    const size_t KS = (size_t)ceil_div(d_in / 256, kWarps);
-    return KS * (size_t)(d_out / 16 + r / 16) * frag;
+    // split-K partial tiles and the bf16 T; depends on the shape only, not on the device
+    DecodePlan pl;
+    if (!make_plan(b, d_out, d_in, r, 1 << 20, &pl)) return 0;
+    return pl.p_bytes + pl.tpart_bytes + pl.tfinal_bytes;
 }
 
 slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
@@ -406,18 +664,23 @@ slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, 
     if (!di) return err;
     DecodePlan pl;
     const int nt = b <= 8 ? 1 : 2;
-    if (!make_plan(b, d_out, d_in, r, decode_ctas(nt), &pl)) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    const int ctas = decode_ctas(nt);
+    if (ctas < 1 || !make_plan(b, d_out, d_in, r, ctas, &pl)) return SLIM_ERR_UNSUPPORTED_SHAPE;
     DecodeParams p;
     p.X = X; p.vals = vals; p.meta = meta; p.L = L; p.R = R; p.Y = Y;
     char* base = reinterpret_cast<char*>(ws);
     p.sync = reinterpret_cast<uint32_t*>(base);
     p.Ppart = reinterpret_cast<float*>(base + SLIM_WORKSPACE_SYNC_BYTES);
     p.Tpart = reinterpret_cast<float*>(base + SLIM_WORKSPACE_SYNC_BYTES + pl.p_bytes);
+    p.Tfinal = reinterpret_cast<__nv_bfloat16*>(base + SLIM_WORKSPACE_SYNC_BYTES + pl.p_bytes + pl.tpart_bytes);
     p.status = status_dev;
     p.s = s; p.b = b; p.r = r; p.d_out = d_out; p.d_in = d_in;
-    p.KS = pl.KS; p.nblk = pl.nblk; p.GW = pl.GW; p.GR = pl.GR; p.r_pad = pl.r_pad;
+    p.KS = pl.KS; p.nblk = pl.nblk; p.G = pl.G; p.QT = pl.QT; p.r_pad = pl.r_pad;
+    p.n_slots = pl.n_slots; p.slot_bytes = pl.slot_bytes;
+    p.pitch_v = pl.pitch_v; p.pitch_m = pl.pitch_m;
+    p.pitch_r = pl.pitch_r; p.pitch_l = pl.pitch_l;
     void* args[] = {&p};
-    const dim3 grid(pl.KS * (pl.GW + pl.GR)), block(kDecodeThreads);
+    const dim3 grid(ctas), block(kDecodeThreads);
     cudaError_t e = nt == 1
         ? cudaLaunchCooperativeKernel((const void*)decode_kernel<1>, grid, block, args, pl.smem, st)
         : cudaLaunchCooperativeKernel((const void*)decode_kernel<2>, grid, block, args, pl.smem, st);
