@@ -492,8 +492,40 @@ def time_cpu_baseline(layers, repeats=8):
                       f"block's 4/2/1 layer counts"}
 
 
+def run_single_case(args):
+    """Plain stream launches of one (d_in, d_out, r, b) case: the command ncu captures."""
+    import torch
+    from paper_2410_09615_b200 import binding as K, build
+    build.build()
+    d_in, d_out, r, b = (int(x) for x in args.case.split(","))
+    s, codes, mask = inputs.make_weights(d_out, d_in, 1)
+    L, R = inputs.make_adapters(d_out, d_in, r, 1)
+    vals, meta = K.slim_pack(torch.from_numpy(codes).cuda(), torch.from_numpy(mask).cuda())
+    Ld = K.bf16_from_bits(L) if r else None
+    Rd = K.bf16_from_bits(R) if r else None
+    X = K.bf16_from_bits(inputs.make_activations(b, d_in, 1))
+    ws = K.new_workspace(b, d_out, d_in, r)
+    Y = torch.empty((b, d_out), dtype=torch.bfloat16, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    for _ in range(args.calls):
+        flush.zero_()                       # evict the weights from L2 between calls
+        e0.record()
+        K.slim_linear_fwd(X, vals, meta, s, Ld, Rd, Y=Y, workspace=ws)
+        e1.record()
+        e1.synchronize()
+        times.append(1e3 * e0.elapsed_time(e1))
+    print(json.dumps({"case": [d_in, d_out, r, b], "calls": args.calls, "us_median": float(np.median(times)),
+                      "us_min": float(np.min(times)), "kernel": K.KERNEL_NAMES[K.slim_select_kernel(b, d_out, d_in, r)],
+                      "algorithmic_bytes": algorithmic_bytes(d_in, d_out, r, b)}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default=None, help="d_in,d_out,r,b: run plain launches of one case (for profilers)")
+    ap.add_argument("--calls", type=int, default=5)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=3000)
     ap.add_argument("--warmup", type=int, default=20)
@@ -502,6 +534,8 @@ def main():
     ap.add_argument("--skip-extras", action="store_true", help="skip the per-case table and the pack timing")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU-oracle baseline")
     args = ap.parse_args()
+    if args.case:
+        return run_single_case(args)
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":

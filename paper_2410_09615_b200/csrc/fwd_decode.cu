@@ -12,11 +12,13 @@
 //     32-column block the k order is permuted so that a thread's A and B
 //     fragments are single 16-byte reads.
 //
-// Data movement.  Every streamed operand travels HBM -> shared memory through
-// the bulk async copy engine (cp.async.bulk + mbarrier) into a ring of slots
-// (~200 KB in flight per SM), issued by a ninth, producer warp; the eight
-// consumer warps read fragments from shared memory.  Activations live in
-// registers as B fragments.
+// Data movement.  Every streamed operand travels HBM -> shared memory as TMA
+// tiles (cp.async.bulk.tensor.2d, 16 rows x 128 bytes, 128-byte swizzle,
+// mbarrier completion) into a ring of 16 KB slots (~190 KB in flight per SM),
+// issued by one lane of a ninth, producer warp; the eight consumer warps read
+// fragments from shared memory.  The producer warp also publishes the CTA's
+// arrivals at the grid-wide counters (fence + atomic), so that the consumers
+// never wait for a fence.  Activations live in registers as B fragments.
 //
 // Work split.  d_in is cut into 256-column blocks and into k-slices of <= 8
 // blocks; a CTA belongs to one slice.  Each CTA first takes its share of R
@@ -31,6 +33,7 @@
 // spins (the launch is cooperative, so all CTAs are resident); an expired wait
 // sets SLIM_ERR_TIMEOUT and the kernel runs on to its end.  Reductions have a
 // fixed order: results are bit-identical from run to run.
+#include <cuda.h>
 #include "common.cuh"
 
 namespace slim {
@@ -45,6 +48,7 @@ constexpr uint32_t kMbarSpinLimit = 1u << 26;              // shared-memory barr
 constexpr int kRChunkCols = 512;                           // columns of one R chunk
 constexpr int kLChunkCols = 512;                           // columns (of r) of one L chunk
 constexpr size_t kSmemBudget = 227 * 1024;
+enum { EV_R = 0, EV_T = 1, EV_W = 2 };                   // consumer -> producer events
 
 // Synchronisation words in the first bytes of the workspace.
 enum { SYNC_R = 0, SYNC_T = 1, SYNC_W = 2, SYNC_DEPART = 3 };
@@ -59,9 +63,10 @@ struct DecodeParams {
     float s;
     int b, r, d_out, d_in;
     int KS, nblk, G, QT, r_pad;
-    int n_slots, slot_bytes;
-    int pitch_v, pitch_m, pitch_r, pitch_l;
+    int n_slots;
 };
+constexpr int kSubTile = 2048;                             // one TMA box: 16 rows x 128 bytes
+constexpr int kSlotBytes = 8 * kSubTile;
 
 // ------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -89,10 +94,25 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     }
     return false;
 }
-// 1-D bulk copy global -> shared, completion counted in bytes on `bar`.
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+// One TMA tile (16 rows x 128 bytes of the tensor behind `tmap`, starting at
+// element column x, row y) into shared memory; completion in bytes on `bar`.
+__device__ __forceinline__ void tma_tile(void* dst, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 :: "r"(smem_u32(dst)), "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+// Byte address inside a 128-byte-swizzled tile of 16 rows: the 16-byte chunk
+// index is XOR-ed with the row number modulo 8.
+__device__ __forceinline__ uint32_t swz(int row, int byte_off) {
+    return (uint32_t)(row * 128 + ((((byte_off >> 4) ^ row) & 7) << 4) + (byte_off & 15));
 }
 __device__ __forceinline__ void consumer_sync() {          // the eight consumer warps only
     asm volatile("bar.sync 1, %0;" :: "n"(kConsumerThreads) : "memory");
@@ -207,17 +227,20 @@ __device__ __forceinline__ float block_tile_sum(float* red, const float (&acc)[N
 
 template <int NT>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
-decode_kernel(const DecodeParams p)
+decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
+              const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmR,
+              const __grid_constant__ CUtensorMap tmL)
 {
     constexpr int frag = NT * 128;
-    extern __shared__ __align__(128) unsigned char smem[];
-    // layout: ring slots | Ts | red (two buffers) | barriers | flags
-    unsigned char* ring = smem;
-    __nv_bfloat16* Ts = reinterpret_cast<__nv_bfloat16*>(ring + (size_t)p.n_slots * p.slot_bytes);
+    extern __shared__ unsigned char smem_raw[];
+    // layout (ring first, 1024-byte aligned for the swizzle): ring slots | Ts | red x2 | barriers | flags
+    unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __nv_bfloat16* Ts = reinterpret_cast<__nv_bfloat16*>(ring + (size_t)p.n_slots * kSlotBytes);
     float* red_base = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(Ts) + (size_t)NT * 8 * p.r_pad * 2);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(red_base + 2 * kConsumerWarps * frag);
     uint64_t* empty_bar = full_bar + kMaxSlots;
-    volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(empty_bar + kMaxSlots);
+    uint64_t* event_bar = empty_bar + kMaxSlots;            // EV_R, EV_T, EV_W
+    volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(event_bar + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
@@ -226,11 +249,12 @@ decode_kernel(const DecodeParams p)
     const Share sh = make_share(p, blockIdx.x);
     const int n_slots = p.n_slots;
     const int l_chunks = p.r > 0 ? ceil_div(p.r, kLChunkCols) : 0;
-    const size_t vstride = (size_t)p.d_in / 4, mstride = (size_t)p.d_in / 8;
-    const int pitch_m = p.pitch_m;
+    int t_mine = 0;                                          // 16-column pieces of T this CTA sums
+    if (p.r > 0) for (int jt = blockIdx.x; jt < tilesR; jt += n_ctas) ++t_mine;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < n_slots; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], kConsumerWarps); }
+        for (int i = 0; i < 3; ++i) mbar_init(&event_bar[i], kConsumerWarps);
         flags[0] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -238,69 +262,84 @@ decode_kernel(const DecodeParams p)
 
     if (warp == kConsumerWarps) {
         // ============================ producer warp ============================
+        if (lane != 0) return;
         uint32_t it = 0;
         bool ok = true;
-        auto acquire = [&](uint32_t bytes) -> int {
+        bool pend[3] = {p.r > 0, t_mine > 0, true};
+        // Publish the CTA's arrivals: the consumers signal an event after their
+        // stores; this thread makes them visible device-wide and bumps the counter.
+        auto service = [&]() {
+            if (pend[EV_R] && mbar_test(&event_bar[EV_R], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_R], 1u); pend[EV_R] = false; }
+            if (pend[EV_T] && mbar_test(&event_bar[EV_T], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_T], (uint32_t)t_mine); pend[EV_T] = false; }
+            if (pend[EV_W] && mbar_test(&event_bar[EV_W], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_W], 1u); pend[EV_W] = false; }
+        };
+        auto acquire = [&](uint32_t bytes) -> unsigned char* {
             const int slot = it % n_slots;
             if (it >= (uint32_t)n_slots) {
-                if (lane == 0) ok = mbar_wait(&empty_bar[slot], ((it / n_slots) & 1) ^ 1) && ok;
+                const uint32_t parity = ((it / n_slots) & 1) ^ 1;
+                uint32_t spins = 0;
+                while (!mbar_test(&empty_bar[slot], parity)) {
+                    service();
+                    if (++spins > kMbarSpinLimit) { ok = false; break; }
+                }
             }
-            if (lane == 0) mbar_arrive_expect_tx(&full_bar[slot], bytes);
-            __syncwarp();
+            mbar_arrive_expect_tx(&full_bar[slot], bytes);
             ++it;
-            return slot;
+            return ring + (size_t)slot * kSlotBytes;
         };
-        // ---- R chunks: 16 rows x (256 or 512) columns of bf16
+        // ---- R chunks: 16 rows x (256 or 512) columns of bf16 = 4 or 8 tiles of 64 columns
         for (int u = sh.r_begin; u < sh.r_begin + sh.r_count; ++u) {
             const int tile = u / sh.Qk, q = u % sh.Qk;
             const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
-            const uint32_t row_bytes = (uint32_t)cols * 2;
-            const int slot = acquire(16 * row_bytes);
-            if (lane < 16) {
-                const __nv_bfloat16* src = p.R + ((size_t)tile * 16 + lane) * p.d_in + (size_t)sh.blk_begin * 256 + (size_t)q * kRChunkCols;
-                bulk_g2s(ring + (size_t)slot * p.slot_bytes + (size_t)lane * p.pitch_r, src, row_bytes, &full_bar[slot]);
-            }
+            const int n_sub = cols / 64;
+            uint64_t* bar = &full_bar[it % n_slots];
+            unsigned char* dst = acquire((uint32_t)n_sub * kSubTile);
+            for (int i = 0; i < n_sub; ++i)
+                tma_tile(dst + i * kSubTile, &tmR, sh.blk_begin * 256 + q * kRChunkCols + 64 * i, tile * 16, bar);
         }
-        // ---- weight tiles: 16 rows of value bytes, then 16 rows of index bytes
+        service();
+        // ---- weight tiles: value bytes (128 per tile row = 2 blocks), then index bytes (4 blocks)
+        const int v_sub = (sh.nb + 1) / 2, m_sub = (sh.nb + 3) / 4;
         for (int tile = sh.w_begin; tile < sh.w_begin + sh.w_count; ++tile) {
-            const uint32_t vbytes = (uint32_t)sh.nb * 64, mbytes = (uint32_t)sh.nb * 32;
-            const int slot = acquire(16 * (vbytes + mbytes));
-            unsigned char* base = ring + (size_t)slot * p.slot_bytes;
-            const size_t row = (size_t)tile * 16 + (lane & 15);
-            if (lane < 16)
-                bulk_g2s(base + (size_t)lane * p.pitch_v, p.vals + row * vstride + (size_t)sh.blk_begin * 64, vbytes, &full_bar[slot]);
-            else
-                bulk_g2s(base + 16 * (size_t)p.pitch_v + (size_t)(lane - 16) * pitch_m,
-                         p.meta + row * mstride + (size_t)sh.blk_begin * 32, mbytes, &full_bar[slot]);
+            uint64_t* bar = &full_bar[it % n_slots];
+            unsigned char* dst = acquire((uint32_t)(v_sub + m_sub) * kSubTile);
+            for (int i = 0; i < v_sub; ++i) tma_tile(dst + i * kSubTile, &tmV, sh.blk_begin * 64 + 128 * i, tile * 16, bar);
+            for (int i = 0; i < m_sub; ++i) tma_tile(dst + (4 + i) * kSubTile, &tmM, sh.blk_begin * 32 + 128 * i, tile * 16, bar);
+            service();
         }
-        // ---- L chunks of the output tiles this CTA finishes
+        // ---- L chunks of the output tiles this CTA finishes (512 columns of r = 8 tiles)
         for (int tile = blockIdx.x; tile < tilesW && p.r > 0; tile += n_ctas) {
             for (int lc = 0; lc < l_chunks; ++lc) {
                 const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
-                const uint32_t row_bytes = (uint32_t)cols * 2;
-                const int slot = acquire(16 * row_bytes);
-                if (lane < 16) {
-                    const __nv_bfloat16* src = p.L + ((size_t)tile * 16 + lane) * p.r + (size_t)lc * kLChunkCols;
-                    bulk_g2s(ring + (size_t)slot * p.slot_bytes + (size_t)lane * p.pitch_l, src, row_bytes, &full_bar[slot]);
-                }
+                const int n_sub = ceil_div(cols, 64);
+                uint64_t* bar = &full_bar[it % n_slots];
+                unsigned char* dst = acquire((uint32_t)n_sub * kSubTile);
+                for (int i = 0; i < n_sub; ++i)
+                    tma_tile(dst + i * kSubTile, &tmL, lc * kLChunkCols + 64 * i, tile * 16, bar);
+                service();
             }
         }
-        if (lane == 0 && !ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
-        return;      // consumers wait for every copy this warp issued before they leave
+        // ---- remaining arrivals
+        for (uint32_t spins = 0; (pend[EV_R] || pend[EV_T] || pend[EV_W]); ++spins) {
+            service();
+            if (spins > kMbarSpinLimit) { ok = false; break; }
+        }
+        if (!ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
+        return;      // the consumers wait for every tile this thread requested before they leave
     }
 
     // ================================ consumer warps ================================
     uint32_t it = 0;
     int red_buf = 0;
     bool ok = true;
-    auto wait_full = [&]() -> int {
+    auto wait_full = [&]() -> unsigned char* {
         const int slot = it % n_slots;
         ok = mbar_wait(&full_bar[slot], (it / n_slots) & 1) && ok;
-        return slot;
+        return ring + (size_t)slot * kSlotBytes;
     };
-    auto release = [&](int slot) {
+    auto release = [&]() {
         __syncwarp();
-        if (lane == 0) mbar_arrive(&empty_bar[slot]);
+        if (lane == 0) mbar_arrive(&empty_bar[it % n_slots]);
         ++it;
     };
     auto next_red = [&]() -> float* {
@@ -308,29 +347,40 @@ decode_kernel(const DecodeParams p)
         red_buf ^= 1;
         return r;
     };
-    // Release pattern for a grid-wide counter: all stores of the CTA, then one add.
-    auto arrive_counter = [&](int which, uint32_t n) {
-        consumer_sync();
-        if (threadIdx.x == 0) { __threadfence(); atomicAdd(&p.sync[which], n); }
+    // Every warp's global stores are done: tell the producer warp to publish them.
+    auto signal = [&](int ev) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&event_bar[ev]);
     };
-    // Thread 0 polls, the result is broadcast to the consumer warps.
-    auto counter_reached = [&](int which, uint32_t target, bool blocking) -> bool {
+    // Thread 0 waits (bounded) for a grid-wide counter; all consumer warps leave together.
+    auto wait_counter = [&](int which, uint32_t target) {
         if (threadIdx.x == 0) {
             bool reached = false;
-            const uint32_t limit = blocking ? kSpinLimit : 1u;
-            for (uint32_t i = 0; i < limit; ++i) {
+            for (uint32_t i = 0; i < kSpinLimit; ++i) {
                 if (ld_acquire(&p.sync[which]) >= target) { reached = true; break; }
-                if (blocking) __nanosleep(20);
+                __nanosleep(20);
             }
-            if (blocking && !reached) flag_error(p.status, SLIM_ERR_TIMEOUT);
-            flags[0] = (reached || blocking) ? 1u : 0u;
-            __threadfence_block();
+            if (!reached) flag_error(p.status, SLIM_ERR_TIMEOUT);
         }
         consumer_sync();
-        const bool res = flags[0] != 0;
-        consumer_sync();
-        return res;
     };
+
+    // activations as sparse B fragments for the weight phase: step j, n-tile h, register i
+    // holds X[g + 8h][slice + 256 warp + 32 j + 2 t + 8 i .. +1].  Requested first: they
+    // are needed last, after the R chunks.
+    const bool w_active = warp < sh.nb && sh.w_count > 0;
+    uint32_t xf[8][NT][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+        for (int h = 0; h < NT; ++h)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = g + 8 * h;
+                xf[j][h][i] = (w_active && row < p.b)
+                    ? __ldg(reinterpret_cast<const uint32_t*>(p.X + (size_t)row * p.d_in + (size_t)(sh.blk_begin + warp) * 256 + 32 * j + 2 * t + 8 * i))
+                    : 0u;
+            }
 
     // ---------------------------------------------------------------- phase R
     if (sh.r_count > 0) {
@@ -353,19 +403,20 @@ decode_kernel(const DecodeParams p)
             const int tile = u / sh.Qk, q = u % sh.Qk;
             const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
             const bool active = warp * 64 < cols;
-            const int slot = wait_full();
+            const unsigned char* base = wait_full();
             float acc[NT][4];
 #pragma unroll
             for (int h = 0; h < NT; ++h)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
             if (active) {
-                const unsigned char* base = ring + (size_t)slot * p.slot_bytes + warp * 128 + t * 16;
+                // warp w owns the 64-column tile w of the chunk
+                const unsigned char* sub = base + warp * kSubTile;
                 uint4 ra[2], rb[2];
 #pragma unroll
                 for (int jj = 0; jj < 2; ++jj) {
-                    ra[jj] = lds128(base + (size_t)g * p.pitch_r + jj * 64);
-                    rb[jj] = lds128(base + (size_t)(g + 8) * p.pitch_r + jj * 64);
+                    ra[jj] = lds128(sub + swz(g, jj * 64 + t * 16));
+                    rb[jj] = lds128(sub + swz(g + 8, jj * 64 + t * 16));
                 }
 #pragma unroll
                 for (int jj = 0; jj < 2; ++jj)
@@ -380,16 +431,16 @@ decode_kernel(const DecodeParams p)
                         mma_16816(acc[h], ra[jj].z, rb[jj].z, ra[jj].w, rb[jj].w, xb.z, xb.w);
                     }
             }
-            release(slot);
+            release();
             const float sum = block_tile_sum<NT>(next_red(), acc, active, min(kConsumerWarps, cols / 64));
             if (threadIdx.x < frag)
                 p.Tpart[((size_t)tile * p.QT + sh.qoff + q) * frag + threadIdx.x] = sum;
         }
     }
-    if (p.r > 0) arrive_counter(SYNC_R, 1);
+    if (p.r > 0) signal(EV_R);
 
     // T reduction duty: CTA c owns the 16-column pieces jt = c, c + n_ctas, ...
-    bool t_pending = p.r > 0 && (int)blockIdx.x < tilesR;
+    bool t_pending = t_mine > 0;
     auto reduce_t = [&]() {
         for (int jt = blockIdx.x; jt < tilesR; jt += n_ctas) {
             if (threadIdx.x < frag) {
@@ -404,29 +455,12 @@ decode_kernel(const DecodeParams p)
                 p.Tfinal[(size_t)m * p.r_pad + j] = __float2bfloat16_rn(sum);
             }
         }
-        int mine = 0;
-        for (int jt = blockIdx.x; jt < tilesR; jt += n_ctas) ++mine;
-        arrive_counter(SYNC_T, (uint32_t)mine);
+        signal(EV_T);
         t_pending = false;
     };
 
     // ---------------------------------------------------------------- phase W
     if (sh.w_count > 0) {
-        // activations as sparse B fragments: step j, n-tile h, register i holds
-        // X[g + 8h][slice + 256 warp + 32 j + 2 t + 8 i .. +1]
-        const bool active = warp < sh.nb;
-        uint32_t xf[8][NT][4];
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-#pragma unroll
-            for (int h = 0; h < NT; ++h)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = g + 8 * h;
-                    xf[j][h][i] = (active && row < p.b)
-                        ? __ldg(reinterpret_cast<const uint32_t*>(p.X + (size_t)row * p.d_in + (size_t)(sh.blk_begin + warp) * 256 + 32 * j + 2 * t + 8 * i))
-                        : 0u;
-                }
         const uint32_t byte_sel = (uint32_t)t * 0x1111u + 0x4400u;   // bytes {t, t, 4+t, 4+t}
         const uint32_t meta_sel = (t & 1) ? 0x7632u : 0x5410u;
         // the CTAs with reduction duty look at the R counter once per tile; the load is
@@ -442,23 +476,27 @@ decode_kernel(const DecodeParams p)
                 if (ready) reduce_t();
                 else if (threadIdx.x == 0) polled = ld_acquire(&p.sync[SYNC_R]);
             }
-            const int slot = wait_full();
+            const unsigned char* base = wait_full();
             float acc[NT][4];
 #pragma unroll
             for (int h = 0; h < NT; ++h)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
-            if (active) {
-                const unsigned char* base = ring + (size_t)slot * p.slot_bytes;
-                const unsigned char* v0p = base + (size_t)g * p.pitch_v + warp * 64;
-                const unsigned char* v1p = v0p + 8 * (size_t)p.pitch_v;
-                const unsigned char* mbase = base + 16 * (size_t)p.pitch_v + warp * 32 + 16 * (t >> 1);
+            if (w_active) {
+                // value bytes of block `warp`: tile warp/2, bytes 64 (warp % 2) .. +64 of the row;
+                // index bytes: tile 4 + warp/4, bytes 32 (warp % 4) .. +32
+                const unsigned char* vsub = base + (warp >> 1) * kSubTile;
+                const unsigned char* msub = base + (4 + (warp >> 2)) * kSubTile;
+                const int vo = (warp & 1) * 64, mo = (warp & 3) * 32 + 16 * (t >> 1);
                 uint4 v0[4], v1[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) { v0[i] = lds128(v0p + 16 * i); v1[i] = lds128(v1p + 16 * i); }
+                for (int i = 0; i < 4; ++i) {
+                    v0[i] = lds128(vsub + swz(g, vo + 16 * i));
+                    v1[i] = lds128(vsub + swz(g + 8, vo + 16 * i));
+                }
                 // index words of steps 0-3 come from threads 0,1 of a quad, of steps 4-7 from threads 2,3
-                const uint4 m0 = lds128(mbase + (size_t)g * pitch_m);
-                const uint4 m1 = lds128(mbase + (size_t)(g + 8) * pitch_m);
+                const uint4 m0 = lds128(msub + swz(g, mo));
+                const uint4 m1 = lds128(msub + swz(g + 8, mo));
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     uint32_t a[4];
@@ -477,18 +515,18 @@ decode_kernel(const DecodeParams p)
                     }
                 }
             }
-            release(slot);
-            const float sum = block_tile_sum<NT>(next_red(), acc, active, sh.nb);
+            release();
+            const float sum = block_tile_sum<NT>(next_red(), acc, w_active, sh.nb);
             if (threadIdx.x < frag)
                 p.Ppart[((size_t)sh.ks * tilesW + tile) * frag + threadIdx.x] = sum;
         }
     }
-    arrive_counter(SYNC_W, 1);
+    signal(EV_W);
 
     // ------------------------------------------------ T: finish, then fetch
     if (p.r > 0) {
-        if (t_pending) { counter_reached(SYNC_R, (uint32_t)n_ctas, true); reduce_t(); }
-        counter_reached(SYNC_T, (uint32_t)tilesR, true);
+        if (t_pending) { wait_counter(SYNC_R, (uint32_t)n_ctas); reduce_t(); }
+        wait_counter(SYNC_T, (uint32_t)tilesR);
         const int rp = p.r_pad;
         for (int idx = threadIdx.x; idx < NT * 8 * (rp / 8); idx += kConsumerThreads) {
             const int m = idx / (rp / 8), c8 = (idx % (rp / 8)) * 8;
@@ -497,35 +535,39 @@ decode_kernel(const DecodeParams p)
             *reinterpret_cast<uint4*>(Ts + (size_t)m * rp + c8) = v;
         }
     }
-    counter_reached(SYNC_W, (uint32_t)n_ctas, true);      // ends with a consumer_sync: Ts is visible
+    wait_counter(SYNC_W, (uint32_t)n_ctas);              // ends with a consumer_sync: Ts is visible
 
     // ---------------------------------------------------------------- phase Y
-    for (int tile = blockIdx.x; tile < tilesW; tile += n_ctas) {
-        float psum = 0.f;
-        if (threadIdx.x < frag) {
+    auto load_psum = [&](int tile) -> float {
+        float v = 0.f;
+        if (threadIdx.x < frag && tile < tilesW) {
             const float* src = p.Ppart + (size_t)tile * frag + threadIdx.x;
 #pragma unroll 4
-            for (int ks = 0; ks < p.KS; ++ks) psum += __ldcg(src + (size_t)ks * tilesW * frag);
+            for (int ks = 0; ks < p.KS; ++ks) v += __ldcg(src + (size_t)ks * tilesW * frag);
         }
+        return v;
+    };
+    float psum_next = load_psum(blockIdx.x);
+    for (int tile = blockIdx.x; tile < tilesW; tile += n_ctas) {
+        const float psum = psum_next;
+        psum_next = load_psum(tile + n_ctas);             // one tile ahead
         float ysum = 0.f;
         for (int lc = 0; lc < l_chunks; ++lc) {
             const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
-            const int slot = wait_full();
+            const unsigned char* base = wait_full();
             float acc[NT][4];
 #pragma unroll
             for (int h = 0; h < NT; ++h)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
-            const unsigned char* base = ring + (size_t)slot * p.slot_bytes;
+            // warp w owns the 64-column tile w of the chunk (two 32-column blocks)
+            if (warp * 64 < cols) {
+                const unsigned char* sub = base + warp * kSubTile;
 #pragma unroll
-            for (int rep = 0; rep < 2; ++rep) {
-                const int kk = 32 * (warp + 8 * rep) + 8 * t;       // column inside the chunk
-                if (32 * (warp + 8 * rep) < cols) {
-                    uint4 la = make_uint4(0, 0, 0, 0), lb = la;
-                    if (kk < cols) {
-                        la = lds128(base + (size_t)g * p.pitch_l + kk * 2);
-                        lb = lds128(base + (size_t)(g + 8) * p.pitch_l + kk * 2);
-                    }
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int kk = warp * 64 + jj * 32 + 8 * t;          // column inside the chunk
+                    const uint4 la = lds128(sub + swz(g, jj * 64 + t * 16));   // columns past r read as zero
+                    const uint4 lb = lds128(sub + swz(g + 8, jj * 64 + t * 16));
 #pragma unroll
                     for (int h = 0; h < NT; ++h) {
                         const uint4 tb = lds128(Ts + (size_t)(g + 8 * h) * p.r_pad + lc * kLChunkCols + kk);
@@ -534,7 +576,7 @@ decode_kernel(const DecodeParams p)
                     }
                 }
             }
-            release(slot);
+            release();
             ysum += block_tile_sum<NT>(next_red(), acc, true, kConsumerWarps);
         }
         if (threadIdx.x < frag) {
@@ -547,36 +589,26 @@ decode_kernel(const DecodeParams p)
     }
 
     // the last CTA to leave puts the counters back to zero for the next call
+    if (!ok && lane == 0) flag_error(p.status, SLIM_ERR_TIMEOUT);
     if (threadIdx.x == 0) {
-        if (!ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
         __threadfence();
         if (atomicAdd(&p.sync[SYNC_DEPART], 1u) == (uint32_t)n_ctas - 1) {
             p.sync[SYNC_R] = 0u; p.sync[SYNC_T] = 0u; p.sync[SYNC_W] = 0u; p.sync[SYNC_DEPART] = 0u;
             __threadfence();
         }
-    } else if (!ok && lane == 0) {
-        flag_error(p.status, SLIM_ERR_TIMEOUT);
     }
 }
 
 // ------------------------------------------------------------------ host side
 struct DecodePlan {
-    int nt, KS, nblk, G, QT, r_pad, n_slots, slot_bytes;
-    int pitch_v, pitch_m, pitch_r, pitch_l;
+    int nt, KS, nblk, G, QT, r_pad, n_slots;
     size_t p_bytes, tpart_bytes, tfinal_bytes, smem;
 };
 
-static int pitch_64mod128(int bytes) {           // smallest pitch >= bytes with pitch % 128 == 64
-    int p = (bytes + 127) / 128 * 128 + 64;
-    if (p - 128 >= bytes) p -= 128;
-    return p;
-}
-
 static int pad_rank(int r) {
     if (r == 0) return 0;
-    int rp = (r + 31) / 32 * 32;
-    if (rp % 64 == 0) rp += 32;      // token rows 64 bytes apart modulo 128: conflict-free 16-byte reads
-    return rp;
+    int rp = (r + 63) / 64 * 64;     // the last L chunk is read in whole 64-column tiles
+    return rp + 32;                  // token rows 64 bytes apart modulo 128: conflict-free 16-byte reads
 }
 
 static bool shape_ok(int b, int d_out, int d_in, int r) {
@@ -590,30 +622,20 @@ static bool make_plan(int b, int d_out, int d_in, int r, int ctas, DecodePlan* p
     pl->KS = ceil_div(pl->nblk, kConsumerWarps);
     pl->G = ctas / pl->KS;
     if (pl->G < 1) return false;
-    int qt = 0, nb_max = 0;
+    int qt = 0;
     for (int k = 0; k < pl->KS; ++k) {
         const int nbk = (int)((long long)(k + 1) * pl->nblk / pl->KS) - (int)((long long)k * pl->nblk / pl->KS);
         qt += (nbk + 1) / 2;
-        if (nbk > nb_max) nb_max = nbk;
     }
     pl->QT = qt;
     pl->r_pad = pad_rank(r);
-    pl->pitch_v = 64 * nb_max + 16;
-    pl->pitch_m = 32 * nb_max + (nb_max % 2 == 0 ? 32 : 0);     // 32 modulo 64: rows g, g+1 never share banks
-    pl->pitch_r = pitch_64mod128((nb_max >= 2 ? kRChunkCols : 256) * 2);
-    pl->pitch_l = r > 0 ? pitch_64mod128((r < kLChunkCols ? r : kLChunkCols) * 2) : 0;
-    int slot = 16 * pl->pitch_v + 16 * pl->pitch_m;
-    if (r > 0) {
-        if (16 * pl->pitch_r > slot) slot = 16 * pl->pitch_r;
-        if (16 * pl->pitch_l > slot) slot = 16 * pl->pitch_l;
-    }
-    pl->slot_bytes = (slot + 127) / 128 * 128;
     const size_t frag = (size_t)pl->nt * 128 * sizeof(float);
-    const size_t fixed = (size_t)pl->nt * 8 * pl->r_pad * 2 + 2 * kConsumerWarps * frag + 2 * kMaxSlots * 8 + 64;
-    if (fixed + 2 * (size_t)pl->slot_bytes > kSmemBudget) return false;
-    int n = (int)((kSmemBudget - fixed) / pl->slot_bytes);
+    const size_t fixed = 1024 /* alignment slack */ + (size_t)pl->nt * 8 * pl->r_pad * 2 + 2 * kConsumerWarps * frag +
+                         (2 * kMaxSlots + 4) * 8 + 64;
+    if (fixed + 2 * (size_t)kSlotBytes > kSmemBudget) return false;
+    int n = (int)((kSmemBudget - fixed) / kSlotBytes);
     pl->n_slots = n > kMaxSlots ? kMaxSlots : n;
-    pl->smem = (size_t)pl->n_slots * pl->slot_bytes + fixed;
+    pl->smem = (size_t)pl->n_slots * kSlotBytes + fixed;
     pl->p_bytes = (size_t)pl->KS * (d_out / 16) * frag;
     pl->tpart_bytes = (size_t)(r / 16) * pl->QT * frag;
     pl->tfinal_bytes = ((size_t)pl->nt * 8 * pl->r_pad * 2 + 255) / 256 * 256;
@@ -654,6 +676,37 @@ size_t decode_workspace_bytes(int b, int d_out, int d_in, int r) {
     return pl.p_bytes + pl.tpart_bytes + pl.tfinal_bytes;
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Row-major 2-D tensor [rows][row_elems] of `esize`-byte elements, tiles of 16 rows x 128 bytes.
+static bool make_tile_map(CUtensorMap* map, const void* base, CUtensorMapDataType type, int esize,
+                          uint64_t row_elems, uint64_t rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {row_elems, rows};
+    cuuint64_t strides[1] = {row_elems * (uint64_t)esize};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / esize), 16};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
 slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
                             float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
                             int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
@@ -676,10 +729,16 @@ slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, 
     p.status = status_dev;
     p.s = s; p.b = b; p.r = r; p.d_out = d_out; p.d_in = d_in;
     p.KS = pl.KS; p.nblk = pl.nblk; p.G = pl.G; p.QT = pl.QT; p.r_pad = pl.r_pad;
-    p.n_slots = pl.n_slots; p.slot_bytes = pl.slot_bytes;
-    p.pitch_v = pl.pitch_v; p.pitch_m = pl.pitch_m;
-    p.pitch_r = pl.pitch_r; p.pitch_l = pl.pitch_l;
-    void* args[] = {&p};
+    p.n_slots = pl.n_slots;
+    CUtensorMap tmV, tmM, tmR, tmL;
+    bool ok = make_tile_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out) &&
+              make_tile_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out);
+    if (ok && r > 0)
+        ok = make_tile_map(&tmR, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r) &&
+             make_tile_map(&tmL, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out);
+    else if (ok) { tmR = tmV; tmL = tmV; }       // never used when r == 0
+    if (!ok) return SLIM_ERR_CUDA;
+    void* args[] = {&p, &tmV, &tmM, &tmR, &tmL};
     const dim3 grid(ctas), block(kDecodeThreads);
     cudaError_t e = nt == 1
         ? cudaLaunchCooperativeKernel((const void*)decode_kernel<1>, grid, block, args, pl.smem, st)
