@@ -262,70 +262,78 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
 
     if (warp == kConsumerWarps) {
         // ============================ producer warp ============================
-        if (lane != 0) return;
+        // Lane 0 runs the ring protocol and publishes arrivals; lanes 0-7 each issue
+        // one 2 KB tile of a chunk (a single thread can start only ~6 TMA loads per
+        // microsecond, eight threads in parallel about 20).
         uint32_t it = 0;
         bool ok = true;
-        bool pend[3] = {p.r > 0, t_mine > 0, true};
+        bool pend_r = p.r > 0, pend_t = t_mine > 0, pend_w = true;
         // Publish the CTA's arrivals: the consumers signal an event after their
-        // stores; this thread makes them visible device-wide and bumps the counter.
+        // stores; lane 0 makes them visible device-wide and bumps the counter.
         auto service = [&]() {
-            if (pend[EV_R] && mbar_test(&event_bar[EV_R], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_R], 1u); pend[EV_R] = false; }
-            if (pend[EV_T] && mbar_test(&event_bar[EV_T], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_T], (uint32_t)t_mine); pend[EV_T] = false; }
-            if (pend[EV_W] && mbar_test(&event_bar[EV_W], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_W], 1u); pend[EV_W] = false; }
+            if (pend_r && mbar_test(&event_bar[EV_R], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_R], 1u); pend_r = false; }
+            if (pend_t && mbar_test(&event_bar[EV_T], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_T], (uint32_t)t_mine); pend_t = false; }
+            if (pend_w && mbar_test(&event_bar[EV_W], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_W], 1u); pend_w = false; }
         };
-        auto acquire = [&](uint32_t bytes) -> unsigned char* {
+        // Returns the slot (all lanes) once it is free and its full barrier is armed.
+        auto acquire = [&](uint32_t bytes) -> int {
             const int slot = it % n_slots;
-            if (it >= (uint32_t)n_slots) {
-                const uint32_t parity = ((it / n_slots) & 1) ^ 1;
-                uint32_t spins = 0;
-                while (!mbar_test(&empty_bar[slot], parity)) {
-                    service();
-                    if (++spins > kMbarSpinLimit) { ok = false; break; }
+            if (lane == 0) {
+                service();
+                if (it >= (uint32_t)n_slots) {
+                    const uint32_t parity = ((it / n_slots) & 1) ^ 1;
+                    uint32_t spins = 0;
+                    while (!mbar_test(&empty_bar[slot], parity)) {
+                        service();
+                        if (++spins > kMbarSpinLimit) { ok = false; break; }
+                    }
                 }
+                mbar_arrive_expect_tx(&full_bar[slot], bytes);
             }
-            mbar_arrive_expect_tx(&full_bar[slot], bytes);
+            __syncwarp();
             ++it;
-            return ring + (size_t)slot * kSlotBytes;
+            return slot;
         };
         // ---- R chunks: 16 rows x (256 or 512) columns of bf16 = 4 or 8 tiles of 64 columns
         for (int u = sh.r_begin; u < sh.r_begin + sh.r_count; ++u) {
             const int tile = u / sh.Qk, q = u % sh.Qk;
             const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
             const int n_sub = cols / 64;
-            uint64_t* bar = &full_bar[it % n_slots];
-            unsigned char* dst = acquire((uint32_t)n_sub * kSubTile);
-            for (int i = 0; i < n_sub; ++i)
-                tma_tile(dst + i * kSubTile, &tmR, sh.blk_begin * 256 + q * kRChunkCols + 64 * i, tile * 16, bar);
+            const int slot = acquire((uint32_t)n_sub * kSubTile);
+            if (lane < n_sub)
+                tma_tile(ring + (size_t)slot * kSlotBytes + lane * kSubTile, &tmR,
+                         sh.blk_begin * 256 + q * kRChunkCols + 64 * lane, tile * 16, &full_bar[slot]);
         }
-        service();
         // ---- weight tiles: value bytes (128 per tile row = 2 blocks), then index bytes (4 blocks)
         const int v_sub = (sh.nb + 1) / 2, m_sub = (sh.nb + 3) / 4;
         for (int tile = sh.w_begin; tile < sh.w_begin + sh.w_count; ++tile) {
-            uint64_t* bar = &full_bar[it % n_slots];
-            unsigned char* dst = acquire((uint32_t)(v_sub + m_sub) * kSubTile);
-            for (int i = 0; i < v_sub; ++i) tma_tile(dst + i * kSubTile, &tmV, sh.blk_begin * 64 + 128 * i, tile * 16, bar);
-            for (int i = 0; i < m_sub; ++i) tma_tile(dst + (4 + i) * kSubTile, &tmM, sh.blk_begin * 32 + 128 * i, tile * 16, bar);
-            service();
+            const int slot = acquire((uint32_t)(v_sub + m_sub) * kSubTile);
+            unsigned char* dst = ring + (size_t)slot * kSlotBytes;
+            if (lane < v_sub)
+                tma_tile(dst + lane * kSubTile, &tmV, sh.blk_begin * 64 + 128 * lane, tile * 16, &full_bar[slot]);
+            else if (lane >= 4 && lane < 4 + m_sub)
+                tma_tile(dst + lane * kSubTile, &tmM, sh.blk_begin * 32 + 128 * (lane - 4), tile * 16, &full_bar[slot]);
         }
         // ---- L chunks of the output tiles this CTA finishes (512 columns of r = 8 tiles)
         for (int tile = blockIdx.x; tile < tilesW && p.r > 0; tile += n_ctas) {
             for (int lc = 0; lc < l_chunks; ++lc) {
                 const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
                 const int n_sub = ceil_div(cols, 64);
-                uint64_t* bar = &full_bar[it % n_slots];
-                unsigned char* dst = acquire((uint32_t)n_sub * kSubTile);
-                for (int i = 0; i < n_sub; ++i)
-                    tma_tile(dst + i * kSubTile, &tmL, lc * kLChunkCols + 64 * i, tile * 16, bar);
-                service();
+                const int slot = acquire((uint32_t)n_sub * kSubTile);
+                if (lane < n_sub)
+                    tma_tile(ring + (size_t)slot * kSlotBytes + lane * kSubTile, &tmL,
+                             lc * kLChunkCols + 64 * lane, tile * 16, &full_bar[slot]);
             }
         }
         // ---- remaining arrivals
-        for (uint32_t spins = 0; (pend[EV_R] || pend[EV_T] || pend[EV_W]); ++spins) {
-            service();
-            if (spins > kMbarSpinLimit) { ok = false; break; }
+        if (lane == 0) {
+            for (uint32_t spins = 0; (pend_r || pend_t || pend_w); ++spins) {
+                service();
+                if (spins > kMbarSpinLimit) { ok = false; break; }
+            }
+            if (!ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
         }
-        if (!ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
-        return;      // the consumers wait for every tile this thread requested before they leave
+        return;      // the consumers wait for every tile this warp requested before they leave
     }
 
     // ================================ consumer warps ================================
