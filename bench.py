@@ -226,7 +226,8 @@ def run_ours(args):
         ly["copies"] = [[(vals.clone(), meta.clone(), ly["Ld"].clone(), ly["Rd"].clone())
                          for _ in range(ly["count"])] for _ in range(n_sets)]
     ws_bytes = max(K.slim_workspace_bytes(b, ly["d_out"], ly["d_in"], ly["r"]) for ly in layers for b in BATCHES)
-    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    K.slim_workspace_reset(ws)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     set_bytes = sum(c[0].numel() + c[1].numel() + 2 * c[2].numel() + 2 * c[3].numel()
                     for ly in layers for c in ly["copies"][0])

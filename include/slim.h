@@ -94,17 +94,17 @@ slim_status_t slim_unpack(const uint8_t* vals, const uint8_t* meta, int d_out, i
 
 /*
  * Bytes of device scratch slim_linear_fwd needs for this problem (split-K
- * partial sums, the adapter intermediate T = X R^T, and synchronisation words).
- * Returns 0 for illegal arguments.  The first SLIM_WORKSPACE_SYNC_BYTES bytes
- * hold counters that must be zero before the first call that uses the buffer
- * (slim_workspace_reset does that); each call leaves them zero again unless it
- * reported SLIM_ERR_TIMEOUT.  Calls that share a workspace must not overlap
- * on the GPU.
+ * partial sums, the adapter intermediate T = X R^T, and a call counter).
+ * Returns 0 for illegal arguments.  A workspace must be initialised once with
+ * slim_workspace_reset before its first use (counter zero, every hand-over slot
+ * marked empty); each call leaves it ready for the next one unless it reported
+ * SLIM_ERR_TIMEOUT, after which it must be reset again.  Calls that share a
+ * workspace must not overlap on the GPU.
  */
 #define SLIM_WORKSPACE_SYNC_BYTES 256
 size_t slim_workspace_bytes(int b, int d_out, int d_in, int r);
 
-/* Zero the synchronisation words of a workspace (asynchronous, on the stream). */
+/* Initialise a whole workspace (asynchronous, on the stream). */
 slim_status_t slim_workspace_reset(void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
@@ -168,7 +168,7 @@ slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* val
  * The first call on a device looks up the array's device address (the device
  * must be current); make that first call before starting any stream capture.
  * All calls on a device share the one array, which keeps the previous call's
- * contents (the counters are cleared on the stream at the start of each call):
+ * contents (the part a call uses is re-initialised on the stream at its start):
  * two calls that overlap on the GPU - different streams, no ordering between
  * them - race on it and produce garbage.  Issue them on one stream or order
  * them with events.

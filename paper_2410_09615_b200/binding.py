@@ -146,11 +146,14 @@ def slim_last_launch_count() -> int:
 
 
 def new_workspace(b: int, d_out: int, d_in: int, r: int, device="cuda") -> torch.Tensor:
-    """Allocate a workspace of the required size with zeroed synchronisation words."""
+    """Allocate a workspace of the required size and initialise it (slim_workspace_reset)."""
     n = slim_workspace_bytes(b, d_out, d_in, r)
     if n == 0:
         raise SlimError(SLIM_ERR_UNSUPPORTED_SHAPE, "slim_workspace_bytes", "illegal shape")
-    return torch.zeros(n, dtype=torch.uint8, device=device)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    with torch.cuda.device(ws.device):
+        slim_workspace_reset(ws)
+    return ws
 
 
 def slim_workspace_reset(workspace: torch.Tensor):

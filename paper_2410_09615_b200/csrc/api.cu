@@ -93,8 +93,10 @@ size_t slim_workspace_bytes(int b, int d_out, int d_in, int r)
 slim_status_t slim_workspace_reset(void* workspace, size_t workspace_bytes_, void* cuda_stream)
 {
     if (!workspace || workspace_bytes_ < SLIM_WORKSPACE_SYNC_BYTES) return SLIM_ERR_WORKSPACE;
-    return cudaMemsetAsync(workspace, 0, SLIM_WORKSPACE_SYNC_BYTES, (cudaStream_t)cuda_stream) == cudaSuccess
-               ? SLIM_OK : SLIM_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // hand-over slots start "empty" (all-ones), the call counter at zero
+    if (cudaMemsetAsync(workspace, 0xFF, workspace_bytes_, st) != cudaSuccess) return SLIM_ERR_CUDA;
+    return cudaMemsetAsync(workspace, 0, SLIM_WORKSPACE_SYNC_BYTES, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
 }
 
 slim_kernel_t slim_select_kernel(int b, int d_out, int d_in, int r)

@@ -12,26 +12,31 @@
 //     32-column block the k order is permuted so that a thread's A and B
 //     fragments are single 16-byte reads.
 //
-// Data movement.  Every streamed operand travels HBM -> shared memory as TMA
-// tiles (cp.async.bulk.tensor.2d, 16 rows x 128 bytes, 128-byte swizzle,
-// mbarrier completion) into a ring of 16 KB slots (~190 KB in flight per SM),
-// issued by one lane of a ninth, producer warp; the eight consumer warps read
-// fragments from shared memory.  The producer warp also publishes the CTA's
-// arrivals at the grid-wide counters (fence + atomic), so that the consumers
-// never wait for a fence.  Activations live in registers as B fragments.
+// Data movement.  Every operand travels global -> shared memory as TMA tiles
+// (cp.async.bulk.tensor.2d, 128-byte rows, 128-byte swizzle, mbarrier
+// completion): the CTA's slice of the activations once, then a ring of 16 KB
+// slots for the streamed matrices.  The lanes of a ninth, producer warp issue
+// the tiles of a chunk in parallel (one thread can start only ~6 TMA loads per
+// microsecond); the eight consumer warps read MMA fragments from shared memory.
 //
 // Work split.  d_in is cut into 256-column blocks and into k-slices of <= 8
-// blocks; a CTA belongs to one slice.  Each CTA first takes its share of R
-// chunks (16 rows x 512 columns), then its share of 16-row weight tiles; both
-// leave split-K partial tiles (fp32, MMA fragment order) in the workspace.
-// Because every CTA does its R share first, T = X R^T is complete early: one
-// CTA per 16 columns of T sums the partials and rounds to bf16 while the weight
-// stream is still running (its ring keeps filling meanwhile).  After the weight
-// phase a grid-wide counter releases the last phase, in which every CTA
-// finishes 16-row output tiles:  Y = s * sum(partials) + T L^T, with the L
-// rows already prefetched into the ring.  All waits on other CTAs are bounded
-// spins (the launch is cooperative, so all CTAs are resident); an expired wait
-// sets SLIM_ERR_TIMEOUT and the kernel runs on to its end.  Reductions have a
+// blocks; a CTA belongs to one slice, one block per consumer warp.  Each CTA
+// first takes its share of R chunks (16 rows x 512 columns), then its share of
+// 16-row weight tiles; both leave split-K partial tiles (fp32, MMA fragment
+// order) in the workspace.  A tenth, service warp of one CTA per 16 columns of
+// T = X R^T sums that piece's partials and publishes it in bf16 while the
+// weight stream is still running.  Finally every CTA finishes 16-row output
+// tiles:  Y = s * sum(partials) + T L^T, with the L rows already prefetched
+// into the ring.
+//
+// Cross-CTA hand-over without fences.  A partial-sum slot is written once and
+// read by exactly one thread: it holds a reserved NaN pattern while empty, the
+// reader polls the slot itself until the pattern is gone and puts the pattern
+// back for the next call.  The bf16 pieces of T have many readers, so each
+// 8-byte entry carries the number of the call that wrote it; the call number
+// comes from a counter every CTA increments when it leaves.  All polls are
+// bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on to its
+// end (the launch is cooperative, so all CTAs are resident).  Reductions have a
 // fixed order: results are bit-identical from run to run.
 #include <cuda.h>
 #include "common.cuh"
@@ -40,33 +45,48 @@ namespace slim {
 
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kDecodeThreads = kConsumerThreads + 32;     // + producer warp
+constexpr int kProducerWarp = kConsumerWarps;
+constexpr int kServiceWarp = kConsumerWarps + 1;
+constexpr int kServiceWarps = 2;
+constexpr int kDecodeThreads = kConsumerThreads + 32 + 32 * kServiceWarps;
 constexpr int kMaxDecodeRank = 3072;
+constexpr int kMaxSlices = 16;
 constexpr int kMaxSlots = 16;
-constexpr uint32_t kSpinLimit = 1u << 22;                  // global counters (each poll sleeps >= 20 ns)
+constexpr uint32_t kPollLimit = 1u << 22;                  // polls of a global slot
 constexpr uint32_t kMbarSpinLimit = 1u << 26;              // shared-memory barriers
 constexpr int kRChunkCols = 512;                           // columns of one R chunk
 constexpr int kLChunkCols = 512;                           // columns (of r) of one L chunk
+constexpr int kSubTile = 2048;                             // one TMA box: 16 rows x 128 bytes
+constexpr int kSlotBytes = 8 * kSubTile;
 constexpr size_t kSmemBudget = 227 * 1024;
-enum { EV_R = 0, EV_T = 1, EV_W = 2 };                   // consumer -> producer events
-
-// Synchronisation words in the first bytes of the workspace.
-enum { SYNC_R = 0, SYNC_T = 1, SYNC_W = 2, SYNC_DEPART = 3 };
+// The published T sits at a fixed place in the workspace (right after the call counter) so
+// that calls of different shapes sharing a workspace never read one kind of slot as the other.
+constexpr size_t kTfinalBytes = 16 * (size_t)(((kMaxDecodeRank + 63) / 64 * 64 + 32) / 2) * 8;
+constexpr uint32_t kEmpty = 0xFFFFFFFFu;                   // "no value yet" in a partial-sum slot
+constexpr uint32_t kNanBits = 0x7FFFFFFFu;                 // what a computed all-ones NaN is stored as
 
 struct DecodeParams {
     const __nv_bfloat16* X; const uint8_t* vals; const uint8_t* meta;
     const __nv_bfloat16* L; const __nv_bfloat16* R; __nv_bfloat16* Y;
-    float* Ppart;              // [KS][tilesW][frag]
-    float* Tpart;              // [tilesR][QT][frag]
-    __nv_bfloat16* Tfinal;     // [NT*8][r_pad]
-    uint32_t* sync; uint32_t* status;
+    uint32_t* Ppart;              // [KS][tilesW][frag]      fp32 bits or kEmpty
+    uint32_t* Tpart;              // [tilesR][QT][frag]      fp32 bits or kEmpty
+    uint2* Tfinal;                // [NT*8][r_pad/2]         {bf16 pair, call number}
+    unsigned long long* departures;   // CTAs that ever left a call on this workspace
+    uint32_t* status;
     float s;
     int b, r, d_out, d_in;
     int KS, nblk, G, QT, r_pad;
     int n_slots;
 };
-constexpr int kSubTile = 2048;                             // one TMA box: 16 rows x 128 bytes
-constexpr int kSlotBytes = 8 * kSubTile;
+
+// Optional timeline: built with -DSLIM_DECODE_TRACE, thread 0 of every CTA records
+// the global timer at the phase boundaries (read back with slim_debug_read_trace).
+#ifdef SLIM_DECODE_TRACE
+__device__ unsigned long long g_trace[256 * 32];
+#define STAMP(i) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_trace[blockIdx.x * 32 + (i)] = t_; } } while (0)
+#else
+#define STAMP(i) do { } while (0)
+#endif
 
 // ------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -94,39 +114,60 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     }
     return false;
 }
-// One TMA tile (16 rows x 128 bytes of the tensor behind `tmap`, starting at
-// element column x, row y) into shared memory; completion in bytes on `bar`.
+// One TMA tile (box of the tensor behind `tmap`, starting at element column x,
+// row y) into shared memory; completion in bytes on `bar`.
 __device__ __forceinline__ void tma_tile(void* dst, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  :: "r"(smem_u32(dst)), "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return done != 0;
-}
-// Byte address inside a 128-byte-swizzled tile of 16 rows: the 16-byte chunk
-// index is XOR-ed with the row number modulo 8.
+// Byte address inside a 128-byte-swizzled tile: the 16-byte chunk index is
+// XOR-ed with the row number modulo 8.
 __device__ __forceinline__ uint32_t swz(int row, int byte_off) {
     return (uint32_t)(row * 128 + ((((byte_off >> 4) ^ row) & 7) << 4) + (byte_off & 15));
 }
 __device__ __forceinline__ void consumer_sync() {          // the eight consumer warps only
     asm volatile("bar.sync 1, %0;" :: "n"(kConsumerThreads) : "memory");
 }
-__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
 __device__ __forceinline__ uint4 lds128(const void* p) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(p)));
     return v;
+}
+__device__ __forceinline__ uint32_t lds32(const void* p) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)));
+    return v;
+}
+// Device-scope accesses that bypass L1: the hand-over slots.
+__device__ __forceinline__ uint32_t ld_gpu(const uint32_t* p) {
+    uint32_t v;
+#ifdef SLIM_LD_VOLATILE
+    asm volatile("ld.volatile.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+#else
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+#endif
+    return v;
+}
+__device__ __forceinline__ uint2 ld_gpu2(const uint2* p) {
+    uint2 v;
+    asm volatile("ld.relaxed.gpu.global.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_gpu(uint32_t* p, uint32_t v) {
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_gpu2(uint2* p, uint2 v) {
+    asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1,%2};" :: "l"(p), "r"(v.x), "r"(v.y) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_gpu64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t slot_bits(float v) {    // fp32 bits that never equal kEmpty
+    const uint32_t u = __float_as_uint(v);
+    return u == kEmpty ? kNanBits : u;
 }
 
 // D(16x8, fp32) += A(16x32 bf16, 2:4 sparse, stored 16x16) * B(32x8 bf16).
@@ -169,9 +210,9 @@ __device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
 }
 
 // ------------------------------------------------------------ work split
-// Everything below is computed identically by the producer and the consumers.
+// Computed identically by every warp role.
 struct Share {
-    int ks, grp;             // k-slice and position inside the slice's CTA group (-1: no phase-1 work)
+    int ks, grp;             // k-slice and position inside the slice's CTA group (-1: no streaming work)
     int blk_begin, nb;       // 256-column blocks of the slice
     int Qk;                  // R chunks per 16-row R tile in this slice
     int qoff;                // index of the slice's first chunk among a tile's QT partial slots
@@ -225,22 +266,62 @@ __device__ __forceinline__ float block_tile_sum(float* red, const float (&acc)[N
     return sum;
 }
 
+// Partial-sum slots, `n` (<= kMaxSlices) of them `stride` words apart.
+// slots_request reads them all once; slots_finish re-reads together those still
+// empty until every one holds a value, adds the values in slot order and marks
+// the slots empty again.
+struct SlotBatch { uint32_t v[kMaxSlices]; };
+
+__device__ __forceinline__ void slots_request(SlotBatch& sb, const uint32_t* first, size_t stride, int n) {
+#pragma unroll
+    for (int i = 0; i < kMaxSlices; ++i) sb.v[i] = i < n ? ld_gpu(first + (size_t)i * stride) : 0u;
+}
+
+__device__ __forceinline__ float slots_finish(SlotBatch& sb, uint32_t* first, size_t stride, int n, bool* ok) {
+    for (uint32_t spins = 0;; ++spins) {
+        bool all = true;
+#pragma unroll
+        for (int i = 0; i < kMaxSlices; ++i) all = all && sb.v[i] != kEmpty;
+        if (all) break;
+        if (spins > kPollLimit) { *ok = false; break; }
+#pragma unroll
+        for (int i = 0; i < kMaxSlices; ++i)
+            if (sb.v[i] == kEmpty) sb.v[i] = ld_gpu(first + (size_t)i * stride);
+    }
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < kMaxSlices; ++i) {
+        if (i < n) {
+            sum += __uint_as_float(sb.v[i]);
+            st_gpu(first + (size_t)i * stride, kEmpty);
+        }
+    }
+    return sum;
+}
+
+__device__ __forceinline__ float take_slots(uint32_t* first, size_t stride, int n, bool* ok) {
+    SlotBatch sb;
+    slots_request(sb, first, stride, n);
+    return slots_finish(sb, first, stride, n, ok);
+}
+
 template <int NT>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
-decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
-              const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmR,
-              const __grid_constant__ CUtensorMap tmL)
+decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
+              const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmM,
+              const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmL)
 {
     constexpr int frag = NT * 128;
+    constexpr int x_sub = NT * 8 * 128;                    // one 64-column tile of the activations
     extern __shared__ unsigned char smem_raw[];
-    // layout (ring first, 1024-byte aligned for the swizzle): ring slots | Ts | red x2 | barriers | flags
+    // layout (1024-byte aligned for the swizzle): ring slots | X slice | Ts | red x2 | barriers
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    __nv_bfloat16* Ts = reinterpret_cast<__nv_bfloat16*>(ring + (size_t)p.n_slots * kSlotBytes);
+    unsigned char* xs = ring + (size_t)p.n_slots * kSlotBytes;
+    __nv_bfloat16* Ts = reinterpret_cast<__nv_bfloat16*>(xs + 32 * x_sub);
     float* red_base = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(Ts) + (size_t)NT * 8 * p.r_pad * 2);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(red_base + 2 * kConsumerWarps * frag);
     uint64_t* empty_bar = full_bar + kMaxSlots;
-    uint64_t* event_bar = empty_bar + kMaxSlots;            // EV_R, EV_T, EV_W
-    volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(event_bar + 4);
+    uint64_t* x_bar = empty_bar + kMaxSlots;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
@@ -249,45 +330,30 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
     const Share sh = make_share(p, blockIdx.x);
     const int n_slots = p.n_slots;
     const int l_chunks = p.r > 0 ? ceil_div(p.r, kLChunkCols) : 0;
-    int t_mine = 0;                                          // 16-column pieces of T this CTA sums
-    if (p.r > 0) for (int jt = blockIdx.x; jt < tilesR; jt += n_ctas) ++t_mine;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < n_slots; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], kConsumerWarps); }
-        for (int i = 0; i < 3; ++i) mbar_init(&event_bar[i], kConsumerWarps);
-        flags[0] = 0;
+        mbar_init(x_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    if (warp == kConsumerWarps) {
+    STAMP(0);
+    if (warp == kProducerWarp) {
         // ============================ producer warp ============================
-        // Lane 0 runs the ring protocol and publishes arrivals; lanes 0-7 each issue
-        // one 2 KB tile of a chunk (a single thread can start only ~6 TMA loads per
-        // microsecond, eight threads in parallel about 20).
         uint32_t it = 0;
         bool ok = true;
-        bool pend_r = p.r > 0, pend_t = t_mine > 0, pend_w = true;
-        // Publish the CTA's arrivals: the consumers signal an event after their
-        // stores; lane 0 makes them visible device-wide and bumps the counter.
-        auto service = [&]() {
-            if (pend_r && mbar_test(&event_bar[EV_R], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_R], 1u); pend_r = false; }
-            if (pend_t && mbar_test(&event_bar[EV_T], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_T], (uint32_t)t_mine); pend_t = false; }
-            if (pend_w && mbar_test(&event_bar[EV_W], 0)) { __threadfence(); atomicAdd(&p.sync[SYNC_W], 1u); pend_w = false; }
-        };
+        // ---- the CTA's slice of the activations: 4 tiles of 64 columns per block, rows >= b read as zero
+        if (sh.grp >= 0) {
+            if (lane == 0) mbar_arrive_expect_tx(x_bar, (uint32_t)(sh.nb * 4 * x_sub));
+            __syncwarp();
+            if (lane < sh.nb * 4) tma_tile(xs + lane * x_sub, &tmX, sh.blk_begin * 256 + 64 * lane, 0, x_bar);
+        }
         // Returns the slot (all lanes) once it is free and its full barrier is armed.
         auto acquire = [&](uint32_t bytes) -> int {
             const int slot = it % n_slots;
             if (lane == 0) {
-                service();
-                if (it >= (uint32_t)n_slots) {
-                    const uint32_t parity = ((it / n_slots) & 1) ^ 1;
-                    uint32_t spins = 0;
-                    while (!mbar_test(&empty_bar[slot], parity)) {
-                        service();
-                        if (++spins > kMbarSpinLimit) { ok = false; break; }
-                    }
-                }
+                if (it >= (uint32_t)n_slots) ok = mbar_wait(&empty_bar[slot], ((it / n_slots) & 1) ^ 1) && ok;
                 mbar_arrive_expect_tx(&full_bar[slot], bytes);
             }
             __syncwarp();
@@ -325,15 +391,42 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
                              lc * kLChunkCols + 64 * lane, tile * 16, &full_bar[slot]);
             }
         }
-        // ---- remaining arrivals
-        if (lane == 0) {
-            for (uint32_t spins = 0; (pend_r || pend_t || pend_w); ++spins) {
-                service();
-                if (spins > kMbarSpinLimit) { ok = false; break; }
-            }
-            if (!ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
-        }
+        if (lane == 0 && !ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
         return;      // the consumers wait for every tile this warp requested before they leave
+    }
+
+    if (warp >= kServiceWarp) {
+        // ============================ service warps ============================
+        // Sums the split-K partials of the 16-column pieces jt = c, c + n_ctas, ... of T,
+        // rounds to bf16 and publishes {two neighbouring columns, call number}.
+        if (p.r == 0 || (int)blockIdx.x >= tilesR) return;
+        const uint32_t call = (uint32_t)(ld_gpu64(p.departures) / (unsigned)n_ctas) + 1u;
+        bool ok = true;
+        for (int jt = blockIdx.x; jt < tilesR; jt += n_ctas) {
+            uint32_t* base = p.Tpart + (size_t)jt * p.QT * frag;
+            // Fragment element f = (h*4 + q)*32 + ln is T[token 8h + 2(ln%4) + (q&1)][16 jt + ln/4 + 8(q>>1)]:
+            // elements with ln/4 = 2i and 2i+1 (same h, q, ln%4) are neighbours along the column index.
+            for (int e = (int)threadIdx.x - kServiceWarp * 32; e < frag / 2; e += 32 * kServiceWarps) {
+                const int i = e & 3, t4 = (e >> 2) & 3, hq = e >> 4;
+                const int f0 = hq * 32 + 8 * i + t4, f1 = f0 + 4;
+                float s0 = 0.f, s1 = 0.f;
+                for (int sl0 = 0; sl0 < p.QT; sl0 += kMaxSlices) {
+                    const int n = min(kMaxSlices, p.QT - sl0);
+                    s0 += take_slots(base + (size_t)sl0 * frag + f0, frag, n, &ok);
+                    s1 += take_slots(base + (size_t)sl0 * frag + f1, frag, n, &ok);
+                }
+                const int h = hq >> 2, q = hq & 3;
+                const int m = 8 * h + 2 * t4 + (q & 1);
+                const int j = jt * 16 + 2 * i + 8 * (q >> 1);
+                __nv_bfloat162 pr = __floats2bfloat162_rn(s0, s1);
+                st_gpu2(p.Tfinal + (size_t)m * (p.r_pad / 2) + (j >> 1), make_uint2(*reinterpret_cast<uint32_t*>(&pr), call));
+            }
+        }
+#ifdef SLIM_DECODE_TRACE
+        if (lane == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_trace[blockIdx.x * 32 + 20] = t_; }
+#endif
+        if (!ok && lane == 0) flag_error(p.status, SLIM_ERR_TIMEOUT);
+        return;
     }
 
     // ================================ consumer warps ================================
@@ -355,40 +448,12 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
         red_buf ^= 1;
         return r;
     };
-    // Every warp's global stores are done: tell the producer warp to publish them.
-    auto signal = [&](int ev) {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&event_bar[ev]);
-    };
-    // Thread 0 waits (bounded) for a grid-wide counter; all consumer warps leave together.
-    auto wait_counter = [&](int which, uint32_t target) {
-        if (threadIdx.x == 0) {
-            bool reached = false;
-            for (uint32_t i = 0; i < kSpinLimit; ++i) {
-                if (ld_acquire(&p.sync[which]) >= target) { reached = true; break; }
-                __nanosleep(20);
-            }
-            if (!reached) flag_error(p.status, SLIM_ERR_TIMEOUT);
-        }
-        consumer_sync();
-    };
+    // the number of this call on this workspace (read before any CTA of the call can have left)
+    uint32_t call = 0;
+    if (p.r > 0) call = (uint32_t)(ld_gpu64(p.departures) / (unsigned)n_ctas) + 1u;
 
-    // activations as sparse B fragments for the weight phase: step j, n-tile h, register i
-    // holds X[g + 8h][slice + 256 warp + 32 j + 2 t + 8 i .. +1].  Requested first: they
-    // are needed last, after the R chunks.
-    const bool w_active = warp < sh.nb && sh.w_count > 0;
-    uint32_t xf[8][NT][4];
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-        for (int h = 0; h < NT; ++h)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = g + 8 * h;
-                xf[j][h][i] = (w_active && row < p.b)
-                    ? __ldg(reinterpret_cast<const uint32_t*>(p.X + (size_t)row * p.d_in + (size_t)(sh.blk_begin + warp) * 256 + 32 * j + 2 * t + 8 * i))
-                    : 0u;
-            }
+    if (sh.grp >= 0) ok = mbar_wait(x_bar, 0) && ok;       // the activation slice is in shared memory
+    STAMP(1);
 
     // ---------------------------------------------------------------- phase R
     if (sh.r_count > 0) {
@@ -401,17 +466,16 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
             for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int h = 0; h < NT; ++h) {
-                    const int row = g + 8 * h;
-                    const int col = q * kRChunkCols + warp * 64 + jj * 32;
-                    xd[q][jj][h] = (col < sh.nb * 256 && row < p.b)
-                        ? __ldg(reinterpret_cast<const uint4*>(p.X + (size_t)row * p.d_in + (size_t)sh.blk_begin * 256 + col + 8 * t))
-                        : make_uint4(0, 0, 0, 0);
+                    const int tile64 = q * 8 + warp;        // 64-column tile of the slice
+                    xd[q][jj][h] = tile64 < sh.nb * 4 ? lds128(xs + tile64 * x_sub + swz(g + 8 * h, jj * 64 + t * 16))
+                                                      : make_uint4(0, 0, 0, 0);
                 }
         for (int u = sh.r_begin; u < sh.r_begin + sh.r_count; ++u) {
             const int tile = u / sh.Qk, q = u % sh.Qk;
             const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
             const bool active = warp * 64 < cols;
             const unsigned char* base = wait_full();
+            if (u == sh.r_begin) STAMP(2);
             float acc[NT][4];
 #pragma unroll
             for (int h = 0; h < NT; ++h)
@@ -442,49 +506,33 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
             release();
             const float sum = block_tile_sum<NT>(next_red(), acc, active, min(kConsumerWarps, cols / 64));
             if (threadIdx.x < frag)
-                p.Tpart[((size_t)tile * p.QT + sh.qoff + q) * frag + threadIdx.x] = sum;
+                st_gpu(p.Tpart + ((size_t)tile * p.QT + sh.qoff + q) * frag + threadIdx.x, slot_bits(sum));
         }
     }
-    if (p.r > 0) signal(EV_R);
 
-    // T reduction duty: CTA c owns the 16-column pieces jt = c, c + n_ctas, ...
-    bool t_pending = t_mine > 0;
-    auto reduce_t = [&]() {
-        for (int jt = blockIdx.x; jt < tilesR; jt += n_ctas) {
-            if (threadIdx.x < frag) {
-                const float* src = p.Tpart + (size_t)jt * p.QT * frag + threadIdx.x;
-                float sum = 0.f;
-#pragma unroll 8
-                for (int sl = 0; sl < p.QT; ++sl) sum += __ldcg(src + (size_t)sl * frag);
-                const int hq = threadIdx.x >> 5, ln = threadIdx.x & 31;
-                const int h = hq >> 2, q = hq & 3;
-                const int j = jt * 16 + (ln >> 2) + 8 * (q >> 1);
-                const int m = 8 * h + 2 * (ln & 3) + (q & 1);
-                p.Tfinal[(size_t)m * p.r_pad + j] = __float2bfloat16_rn(sum);
-            }
-        }
-        signal(EV_T);
-        t_pending = false;
-    };
-
+    STAMP(3);
     // ---------------------------------------------------------------- phase W
     if (sh.w_count > 0) {
+        // activations as sparse B fragments: step j, n-tile h, register i holds
+        // X[g + 8h][slice + 256 warp + 32 j + 2 t + 8 i .. +1]
+        const bool w_active = warp < sh.nb;
+        uint32_t xf[8][NT][4];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int h = 0; h < NT; ++h)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int col = 32 * j + 2 * t + 8 * i;          // inside the warp's 256-column block
+                    xf[j][h][i] = w_active ? lds32(xs + (warp * 4 + (col >> 6)) * x_sub + swz(g + 8 * h, (col & 63) * 2)) : 0u;
+                }
         const uint32_t byte_sel = (uint32_t)t * 0x1111u + 0x4400u;   // bytes {t, t, 4+t, 4+t}
         const uint32_t meta_sel = (t & 1) ? 0x7632u : 0x5410u;
-        // the CTAs with reduction duty look at the R counter once per tile; the load is
-        // issued one tile ahead so that its latency is never waited for
-        uint32_t polled = 0;
-        if (t_pending && threadIdx.x == 0) polled = ld_acquire(&p.sync[SYNC_R]);
+        STAMP(4);
         for (int tile = sh.w_begin; tile < sh.w_begin + sh.w_count; ++tile) {
-            if (t_pending) {
-                if (threadIdx.x == 0) flags[0] = polled >= (uint32_t)n_ctas ? 1u : 0u;
-                consumer_sync();
-                const bool ready = flags[0] != 0;
-                consumer_sync();
-                if (ready) reduce_t();
-                else if (threadIdx.x == 0) polled = ld_acquire(&p.sync[SYNC_R]);
-            }
             const unsigned char* base = wait_full();
+            if (tile == sh.w_begin) STAMP(5);
+            if (tile == sh.w_begin + 1) STAMP(6);
             float acc[NT][4];
 #pragma unroll
             for (int h = 0; h < NT; ++h)
@@ -526,39 +574,54 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
             release();
             const float sum = block_tile_sum<NT>(next_red(), acc, w_active, sh.nb);
             if (threadIdx.x < frag)
-                p.Ppart[((size_t)sh.ks * tilesW + tile) * frag + threadIdx.x] = sum;
+                st_gpu(p.Ppart + ((size_t)sh.ks * tilesW + tile) * frag + threadIdx.x, slot_bits(sum));
         }
     }
-    signal(EV_W);
 
-    // ------------------------------------------------ T: finish, then fetch
+    STAMP(7);
+    // the split-K partials of an output tile are requested early: the first tile's now,
+    // the others one tile ahead
+    SlotBatch pb;
+    const size_t p_stride = (size_t)tilesW * frag;
+    if (threadIdx.x < frag && (int)blockIdx.x < tilesW)
+        slots_request(pb, p.Ppart + (size_t)blockIdx.x * frag + threadIdx.x, p_stride, p.KS);
+
+    // ------------------------------------------------ T (bf16) into shared memory
     if (p.r > 0) {
-        if (t_pending) { wait_counter(SYNC_R, (uint32_t)n_ctas); reduce_t(); }
-        wait_counter(SYNC_T, (uint32_t)tilesR);
-        const int rp = p.r_pad;
-        for (int idx = threadIdx.x; idx < NT * 8 * (rp / 8); idx += kConsumerThreads) {
-            const int m = idx / (rp / 8), c8 = (idx % (rp / 8)) * 8;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (c8 < p.r) v = __ldcg(reinterpret_cast<const uint4*>(p.Tfinal + (size_t)m * rp + c8));
-            *reinterpret_cast<uint4*>(Ts + (size_t)m * rp + c8) = v;
+        // a thread fetches column pair jp of every token row: one batch of NT*8 entries,
+        // re-requested together while some are not yet published
+        const int rp = p.r_pad, pairs = rp / 2;
+        for (int jp = threadIdx.x; jp < pairs; jp += kConsumerThreads) {
+            uint2 e[NT * 8];
+            const bool real = 2 * jp < p.r;               // padding columns are zero
+#pragma unroll
+            for (int m = 0; m < NT * 8; ++m) e[m] = make_uint2(0u, real ? call - 1u : call);
+            for (uint32_t spins = 0;; ++spins) {
+                bool all = true;
+#pragma unroll
+                for (int m = 0; m < NT * 8; ++m)
+                    if (e[m].y != call) e[m] = ld_gpu2(p.Tfinal + (size_t)m * pairs + jp);
+#pragma unroll
+                for (int m = 0; m < NT * 8; ++m) all = all && e[m].y == call;
+                if (all) break;
+                if (spins > kPollLimit) { ok = false; break; }
+            }
+#pragma unroll
+            for (int m = 0; m < NT * 8; ++m) *reinterpret_cast<uint32_t*>(Ts + (size_t)m * rp + 2 * jp) = e[m].x;
         }
     }
-    wait_counter(SYNC_W, (uint32_t)n_ctas);              // ends with a consumer_sync: Ts is visible
+    consumer_sync();
+    STAMP(8);
 
     // ---------------------------------------------------------------- phase Y
-    auto load_psum = [&](int tile) -> float {
-        float v = 0.f;
-        if (threadIdx.x < frag && tile < tilesW) {
-            const float* src = p.Ppart + (size_t)tile * frag + threadIdx.x;
-#pragma unroll 4
-            for (int ks = 0; ks < p.KS; ++ks) v += __ldcg(src + (size_t)ks * tilesW * frag);
-        }
-        return v;
-    };
-    float psum_next = load_psum(blockIdx.x);
     for (int tile = blockIdx.x; tile < tilesW; tile += n_ctas) {
-        const float psum = psum_next;
-        psum_next = load_psum(tile + n_ctas);             // one tile ahead
+        float psum = 0.f;
+        if (threadIdx.x < frag) {
+            psum = slots_finish(pb, p.Ppart + (size_t)tile * frag + threadIdx.x, p_stride, p.KS, &ok);
+            if (tile + n_ctas < tilesW)
+                slots_request(pb, p.Ppart + (size_t)(tile + n_ctas) * frag + threadIdx.x, p_stride, p.KS);
+        }
+        if (tile == (int)blockIdx.x) STAMP(9);
         float ysum = 0.f;
         for (int lc = 0; lc < l_chunks; ++lc) {
             const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
@@ -596,15 +659,10 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmV,
         }
     }
 
-    // the last CTA to leave puts the counters back to zero for the next call
+    STAMP(10);
     if (!ok && lane == 0) flag_error(p.status, SLIM_ERR_TIMEOUT);
-    if (threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(&p.sync[SYNC_DEPART], 1u) == (uint32_t)n_ctas - 1) {
-            p.sync[SYNC_R] = 0u; p.sync[SYNC_T] = 0u; p.sync[SYNC_W] = 0u; p.sync[SYNC_DEPART] = 0u;
-            __threadfence();
-        }
-    }
+    consumer_sync();                                       // every poll of this CTA is over
+    if (threadIdx.x == 0) atomicAdd(p.departures, 1ull);
 }
 
 // ------------------------------------------------------------------ host side
@@ -620,7 +678,8 @@ static int pad_rank(int r) {
 }
 
 static bool shape_ok(int b, int d_out, int d_in, int r) {
-    return b >= 1 && b <= 16 && d_in % 256 == 0 && d_out % 16 == 0 && r % 16 == 0 && r >= 0 && r <= kMaxDecodeRank;
+    return b >= 1 && b <= 16 && d_in % 256 == 0 && d_out % 16 == 0 && r % 16 == 0 && r >= 0 && r <= kMaxDecodeRank &&
+           d_in / 256 <= kMaxSlices * kConsumerWarps;
 }
 
 static bool make_plan(int b, int d_out, int d_in, int r, int ctas, DecodePlan* pl) {
@@ -638,15 +697,15 @@ static bool make_plan(int b, int d_out, int d_in, int r, int ctas, DecodePlan* p
     pl->QT = qt;
     pl->r_pad = pad_rank(r);
     const size_t frag = (size_t)pl->nt * 128 * sizeof(float);
-    const size_t fixed = 1024 /* alignment slack */ + (size_t)pl->nt * 8 * pl->r_pad * 2 + 2 * kConsumerWarps * frag +
-                         (2 * kMaxSlots + 4) * 8 + 64;
-    if (fixed + 2 * (size_t)kSlotBytes > kSmemBudget) return false;
+    const size_t fixed = 1024 /* alignment slack */ + 32 * (size_t)pl->nt * 8 * 128 /* X slice */ +
+                         (size_t)pl->nt * 8 * pl->r_pad * 2 + 2 * kConsumerWarps * frag + (2 * kMaxSlots + 2) * 8 + 64;
+    if (fixed + 3 * (size_t)kSlotBytes > kSmemBudget) return false;
     int n = (int)((kSmemBudget - fixed) / kSlotBytes);
     pl->n_slots = n > kMaxSlots ? kMaxSlots : n;
     pl->smem = (size_t)pl->n_slots * kSlotBytes + fixed;
     pl->p_bytes = (size_t)pl->KS * (d_out / 16) * frag;
     pl->tpart_bytes = (size_t)(r / 16) * pl->QT * frag;
-    pl->tfinal_bytes = ((size_t)pl->nt * 8 * pl->r_pad * 2 + 255) / 256 * 256;
+    pl->tfinal_bytes = kTfinalBytes;
     return true;
 }
 
@@ -678,7 +737,7 @@ bool decode_supports(int b, int d_out, int d_in, int r) {
 }
 
 size_t decode_workspace_bytes(int b, int d_out, int d_in, int r) {
-    // split-K partial tiles and the bf16 T; depends on the shape only, not on the device
+    // split-K partial slots and the published bf16 T; depends on the shape only, not on the device
     DecodePlan pl;
     if (!make_plan(b, d_out, d_in, r, 1 << 20, &pl)) return 0;
     return pl.p_bytes + pl.tpart_bytes + pl.tfinal_bytes;
@@ -701,14 +760,14 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Row-major 2-D tensor [rows][row_elems] of `esize`-byte elements, tiles of 16 rows x 128 bytes.
+// Row-major 2-D tensor [rows][row_elems] of `esize`-byte elements, tiles of box_rows x 128 bytes.
 static bool make_tile_map(CUtensorMap* map, const void* base, CUtensorMapDataType type, int esize,
-                          uint64_t row_elems, uint64_t rows) {
+                          uint64_t row_elems, uint64_t rows, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {row_elems, rows};
     cuuint64_t strides[1] = {row_elems * (uint64_t)esize};
-    cuuint32_t box[2] = {(cuuint32_t)(128 / esize), 16};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / esize), (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
@@ -730,23 +789,24 @@ slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, 
     DecodeParams p;
     p.X = X; p.vals = vals; p.meta = meta; p.L = L; p.R = R; p.Y = Y;
     char* base = reinterpret_cast<char*>(ws);
-    p.sync = reinterpret_cast<uint32_t*>(base);
-    p.Ppart = reinterpret_cast<float*>(base + SLIM_WORKSPACE_SYNC_BYTES);
-    p.Tpart = reinterpret_cast<float*>(base + SLIM_WORKSPACE_SYNC_BYTES + pl.p_bytes);
-    p.Tfinal = reinterpret_cast<__nv_bfloat16*>(base + SLIM_WORKSPACE_SYNC_BYTES + pl.p_bytes + pl.tpart_bytes);
+    p.departures = reinterpret_cast<unsigned long long*>(base);
+    p.Tfinal = reinterpret_cast<uint2*>(base + SLIM_WORKSPACE_SYNC_BYTES);
+    p.Ppart = reinterpret_cast<uint32_t*>(base + SLIM_WORKSPACE_SYNC_BYTES + kTfinalBytes);
+    p.Tpart = reinterpret_cast<uint32_t*>(base + SLIM_WORKSPACE_SYNC_BYTES + kTfinalBytes + pl.p_bytes);
     p.status = status_dev;
     p.s = s; p.b = b; p.r = r; p.d_out = d_out; p.d_in = d_in;
     p.KS = pl.KS; p.nblk = pl.nblk; p.G = pl.G; p.QT = pl.QT; p.r_pad = pl.r_pad;
     p.n_slots = pl.n_slots;
-    CUtensorMap tmV, tmM, tmR, tmL;
-    bool ok = make_tile_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out) &&
-              make_tile_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out);
+    CUtensorMap tmX, tmV, tmM, tmR, tmL;
+    bool ok = make_tile_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, nt * 8) &&
+              make_tile_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, 16) &&
+              make_tile_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, 16);
     if (ok && r > 0)
-        ok = make_tile_map(&tmR, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r) &&
-             make_tile_map(&tmL, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out);
+        ok = make_tile_map(&tmR, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 16) &&
+             make_tile_map(&tmL, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, 16);
     else if (ok) { tmR = tmV; tmL = tmV; }       // never used when r == 0
     if (!ok) return SLIM_ERR_CUDA;
-    void* args[] = {&p, &tmV, &tmM, &tmR, &tmL};
+    void* args[] = {&p, &tmX, &tmV, &tmM, &tmR, &tmL};
     const dim3 grid(ctas), block(kDecodeThreads);
     cudaError_t e = nt == 1
         ? cudaLaunchCooperativeKernel((const void*)decode_kernel<1>, grid, block, args, pl.smem, st)
@@ -756,3 +816,9 @@ slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, 
 }
 
 }  // namespace slim
+
+#ifdef SLIM_DECODE_TRACE
+extern "C" int slim_debug_read_trace(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, slim::g_trace, sizeof(slim::g_trace));
+}
+#endif

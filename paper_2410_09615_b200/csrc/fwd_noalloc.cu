@@ -7,8 +7,7 @@
 namespace slim {
 
 // Scratch shared by every call of slim_linear_fwd_noalloc on a device: split-K
-// partial tiles plus, in its first SLIM_WORKSPACE_SYNC_BYTES, the grid-barrier
-// counters.  Each GPU that loads the library carries one copy until exit.
+// partial slots plus, in its first SLIM_WORKSPACE_SYNC_BYTES, the call counter.  Each GPU that loads the library carries one copy until exit.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[SLIM_NOALLOC_SCRATCH_BYTES];
 
 // In host code `g_noalloc_scratch` is only a handle for the runtime, not an
@@ -59,8 +58,11 @@ extern "C" slim_status_t slim_linear_fwd_noalloc(const void* X, int b, const uin
     slim_status_t st = scratch_address(&scratch);
     if (st != SLIM_OK) return st;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    // the array keeps whatever the previous call left: the barrier counters must start at zero
-    if (cudaMemsetAsync(scratch, 0, SLIM_WORKSPACE_SYNC_BYTES, stream) != cudaSuccess) return SLIM_ERR_CUDA;
+    // the array keeps whatever the previous call left (possibly of another shape, possibly cut
+    // short by a timeout): mark this call's hand-over slots empty and restart the call counter
+    if (cudaMemsetAsync(static_cast<char*>(scratch) + SLIM_WORKSPACE_SYNC_BYTES, 0xFF, need, stream) != cudaSuccess ||
+        cudaMemsetAsync(scratch, 0, SLIM_WORKSPACE_SYNC_BYTES, stream) != cudaSuccess)
+        return SLIM_ERR_CUDA;
     return launch_decode(static_cast<const __nv_bfloat16*>(X), b, vals, meta, s,
                          static_cast<const __nv_bfloat16*>(L), static_cast<const __nv_bfloat16*>(R), r, d_out,
                          d_in, static_cast<__nv_bfloat16*>(Y), scratch, status_dev, stream);

@@ -42,8 +42,10 @@ def run_case(d_in, d_out, r, b, seed, wseed=None, kernel=binding.KERNEL_AUTO, ro
     launches = binding.slim_last_launch_count()
     torch.cuda.synchronize()
     assert binding.read_status(status) == 0, f"device status {binding.read_status(status):#x}"
-    # the synchronisation words are left clean for the next call
-    assert int(ws[:binding.WORKSPACE_SYNC_BYTES].to(torch.int32).sum().item()) == 0
+    # the workspace is left ready for the next call: same inputs, same bits
+    Y2 = binding.slim_linear_fwd(X, vals, meta, s, L, R, workspace=ws, status=status, kernel=kernel)
+    torch.cuda.synchronize()
+    assert binding.read_status(status) == 0 and torch.equal(Y2.view(torch.int16), Y.view(torch.int16))
     y = inputs.bf16_bits_to_f64(binding.bits_from_bf16(Y))
     if rows is not None:
         y = y[np.asarray(rows)]

@@ -19,7 +19,7 @@ def test_noalloc_rejects_problems_beyond_its_scratch_on_the_host():
     build.build()
     lib = K.lib()
     fake = 4096          # aligned, never dereferenced: the call must fail before touching it
-    too_big = lib.slim_linear_fwd_noalloc(fake, 16, fake, fake, 1.0, fake, fake, 64, 32768, 65536, fake, None, None)
+    too_big = lib.slim_linear_fwd_noalloc(fake, 16, fake, fake, 1.0, fake, fake, 64, 65536, 28672, fake, None, None)
     assert too_big == K.SLIM_ERR_WORKSPACE
     assert lib.slim_linear_fwd_noalloc(fake, 17, fake, fake, 1.0, None, None, 0, 512, 512, fake, None,
                                        None) == K.SLIM_ERR_UNSUPPORTED_SHAPE
