@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libslim.so")
-SOURCES = ["api.cu", "pack.cu", "fwd_simple.cu", "fwd_decode.cu", "fwd_noalloc.cu"]
+SOURCES = ["api.cu", "pack.cu", "fwd_simple.cu", "fwd_decode.cu", "fwd_prefill.cu", "fwd_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math"]
 

@@ -44,6 +44,7 @@ static slim_status_t check_weight_shape(int d_out, int d_in) {
 
 static slim_kernel_t select_kernel(int b, int d_out, int d_in, int r) {
     if (b <= 16 && decode_supports(b, d_out, d_in, r)) return SLIM_KERNEL_DECODE;
+    if (b > 16 && prefill_supports(b, d_out, d_in, r)) return SLIM_KERNEL_PREFILL;
     return SLIM_KERNEL_SIMPLE;
 }
 
@@ -51,6 +52,8 @@ static size_t workspace_bytes(int b, int d_out, int d_in, int r) {
     size_t need = simple_workspace_bytes(b, d_out, d_in, r);
     const size_t d = decode_workspace_bytes(b, d_out, d_in, r);
     if (d > need) need = d;
+    const size_t pf = prefill_workspace_bytes(b, d_out, d_in, r);
+    if (pf > need) need = pf;
     need = (need + 255) / 256 * 256;
     return SLIM_WORKSPACE_SYNC_BYTES + need;
 }
@@ -135,6 +138,9 @@ slim_status_t slim_linear_fwd_ex(const void* X, int b, const uint8_t* vals, cons
     case SLIM_KERNEL_DECODE:
         if (b > 16 || !decode_supports(b, d_out, d_in, r)) return SLIM_ERR_UNSUPPORTED_SHAPE;
         return launch_decode(Xb, b, vals, meta, s, Lb, Rb, r, d_out, d_in, Yb, workspace, status_dev, stream);
+    case SLIM_KERNEL_PREFILL:
+        if (!prefill_supports(b, d_out, d_in, r)) return SLIM_ERR_UNSUPPORTED_SHAPE;
+        return launch_prefill(Xb, b, vals, meta, s, Lb, Rb, r, d_out, d_in, Yb, workspace, status_dev, stream);
     default:
         return SLIM_ERR_UNSUPPORTED_SHAPE;
     }

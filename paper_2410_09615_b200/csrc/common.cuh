@@ -46,4 +46,11 @@ slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, 
                             cudaStream_t st);
 int decode_query_residency(int nt);
 
+bool prefill_supports(int b, int d_out, int d_in, int r);
+size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r);
+slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
+                             float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
+                             int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
+                             cudaStream_t st);
+
 }  // namespace slim

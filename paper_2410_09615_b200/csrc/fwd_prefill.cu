@@ -1,0 +1,407 @@
+// Prefill-phase forward (many tokens): tcgen05 tensor cores with the accumulator
+// in tensor memory.
+//
+// One CTA computes a 128 (output rows) x 128 (tokens) tile of
+//     out[token][row] = scale * ( sum_k W[row][k] X[token][k]  +  sum_j A2[row][j] B2[token][j] )
+// in two chained phases that accumulate into the same TMEM tile:
+//   phase 1 (sparse): W is the packed int4 2:4 weight.  TMA brings 128 rows of value
+//       bytes and index bytes plus the X tile; four converter warps (one thread per
+//       weight row) expand nibbles to exact bf16 into the 128-byte-swizzled K-major
+//       layout the MMA reads, and write the 2:4 index words into tensor memory;
+//       one thread issues tcgen05.mma.sp (kind::f16, bf16 x bf16 -> fp32).
+//   phase 2 (dense): A2 and B2 are bf16 matrices brought by TMA as they are; the same
+//       thread issues tcgen05.mma into the same accumulator.
+// The layer forward is two launches of this kernel:
+//   T' = (X R^T) / s          phase 2 only  (A2 = R, B2 = X, scale 1/s), bf16 into the workspace
+//   Y  = s * (X Q^T + T' L^T) phase 1 then phase 2 (A2 = L, B2 = T', scale s)
+// so the adapter product and the scale are fused into the tile loop and the epilogue.
+//
+// Index words in tensor memory (one 32-bit column per MMA of 32 weight columns): lane
+// l holds 16 of the 32 columns (half (l / 8) % 2) of two rows, row l & ~8 in bits
+// 0-15 and row l | 8 in bits 16-31; the MMA addresses an even column pair and a
+// selector bit of the instruction descriptor picks the column.  A 32-bit word of the
+// packed index array is one row's 32 columns, so a converter thread swaps one
+// half-word with the thread eight rows away and stores the result.
+//
+// Pipeline: 4 stages of {A 16 KB, B 32 KB, value bytes 4 KB, index bytes 2 KB};
+// mbarriers: tma_full (TMA bytes landed), conv_done (converters finished a stage),
+// empty (tcgen05.commit: the MMAs that read the stage are complete), acc_full.
+// Every wait is bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on.
+#include <cuda.h>
+#include "common.cuh"
+
+namespace slim {
+
+constexpr int kPM = 128;            // output rows per CTA (MMA M)
+constexpr int kPN = 128;            // tokens per CTA (MMA N)
+constexpr int kPBK1 = 128;          // weight columns per stage in the sparse phase (4 MMAs of K = 32)
+constexpr int kPBK2 = 64;           // columns per stage in the dense phase (4 MMAs of K = 16)
+constexpr int kPStages = 4;
+constexpr int kPThreads = 192;      // warps 0-3 converters / epilogue, warp 4 TMA, warp 5 MMA
+constexpr int kATile = kPM * 128;               // 16 KB: 128 rows x 128 bytes
+constexpr int kBTile = kPN * 128;               // 16 KB: 128 tokens x 128 bytes
+constexpr int kValsTile = kPM * (kPBK1 / 4);    // 4 KB
+constexpr int kMetaTile = kPM * (kPBK1 / 8);    // 2 KB
+constexpr int kStageBytes = kATile + 2 * kBTile + kValsTile + kMetaTile;
+constexpr int kTmemCols = 256;      // accumulator: columns 0-127; index words: 128 + 4 * stage + mma
+constexpr int kTmemECol = 128;
+constexpr uint32_t kPSpinLimit = 1u << 21;
+constexpr size_t kPrefillSmem = 1024 + (size_t)kPStages * kStageBytes + 256;
+
+struct PrefillParams {
+    __nv_bfloat16* out;     // [tokens][ldo]
+    int ldo;
+    int m_total;            // valid output rows
+    int b;                  // valid tokens
+    int n1, n2;             // stages of the sparse and of the dense phase
+    float scale;
+    uint32_t* status;
+};
+
+namespace pf {
+
+__device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(s32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(s32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(s32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait.  The first wait of a CTA that expires raises `*abort_flag`; every later
+// wait of the CTA then gives up at once, so a broken pipeline costs one time-out, not many.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    const uint32_t addr = s32(bar);
+    for (uint32_t it = 0; it < kPSpinLimit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1u;
+    return false;
+}
+__device__ __forceinline__ void tma_tile(void* dst, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 :: "r"(s32(dst)), "l"(tmap), "r"(x), "r"(y), "r"(s32(bar)) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle,
+// 8-row groups 1024 bytes apart (descriptor version 1).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, both K-major.
+__host__ __device__ constexpr uint32_t idesc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_dense(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// A holds the two kept values of every group of four; e_tmem addresses the index words.
+__device__ __forceinline__ void mma_sparse(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t e_tmem,
+                                           uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+        :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(s32(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Two int4 codes of byte `T` of w -> exact bf16x2: nibble ^ 8 in the mantissa of 128.0
+// is 128 + (v + 8); subtracting 136 leaves v in [-8, 7].
+template <int T>
+__device__ __forceinline__ uint32_t nib2bf16(uint32_t w, uint32_t w_shr4) {
+    uint32_t x, y;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(x) : "r"(w), "r"(w_shr4), "n"(T * 0x1111 + 0x4400));
+    asm("lop3.b32 %0, %1, %2, %3, 0x6a;" : "=r"(y) : "r"(x), "r"(0x000F000Fu), "r"(0x43084308u));
+    __nv_bfloat162 v = *reinterpret_cast<__nv_bfloat162*>(&y);
+    const uint32_t bias_bits = 0x43084308u;
+    v = __hsub2(v, *reinterpret_cast<const __nv_bfloat162*>(&bias_bits));
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+}  // namespace pf
+
+__global__ void __launch_bounds__(kPThreads, 1)
+prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
+               const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmX,
+               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2)
+{
+    using namespace pf;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(stages + (size_t)kPStages * kStageBytes);
+    uint64_t* tma_full = bars;                       // [kPStages]
+    uint64_t* conv_done = bars + kPStages;           // [kPStages]
+    uint64_t* empty = bars + 2 * kPStages;           // [kPStages]
+    uint64_t* acc_full = bars + 3 * kPStages;        // [1]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kPStages + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kPM, n0 = blockIdx.y * kPN;
+    const int n_total = p.n1 + p.n2;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kPStages; ++i) { mbar_init(&tma_full[i], 1); mbar_init(&conv_done[i], kPM); mbar_init(&empty[i], 1); }
+        mbar_init(acc_full, 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+    bool ok = true;
+
+    if (warp == 4) {
+        // ============================ TMA producer ============================
+        // lane 0 runs the ring protocol; lanes 0-3 each request one tile of a stage
+        for (int it = 0; it < n_total; ++it) {
+            const int st = it % kPStages;
+            unsigned char* sbase = stages + (size_t)st * kStageBytes;
+            const bool sparse = it < p.n1;
+            if (lane == 0) {
+                if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
+                mbar_expect_tx(&tma_full[st], sparse ? (uint32_t)(kValsTile + kMetaTile + 2 * kBTile) : (uint32_t)(kATile + kBTile));
+            }
+            __syncwarp();
+            if (sparse) {
+                const int k = it * kPBK1;
+                if (lane == 0) tma_tile(sbase + kATile + 2 * kBTile, &tmV, k / 4, m0, &tma_full[st]);
+                else if (lane == 1) tma_tile(sbase + kATile + 2 * kBTile + kValsTile, &tmM, k / 8, m0, &tma_full[st]);
+                else if (lane == 2) tma_tile(sbase + kATile, &tmX, k, n0, &tma_full[st]);
+                else if (lane == 3) tma_tile(sbase + kATile + kBTile, &tmX, k + 64, n0, &tma_full[st]);
+            } else {
+                const int k = (it - p.n1) * kPBK2;
+                if (lane == 0) tma_tile(sbase, &tmA2, k, m0, &tma_full[st]);
+                else if (lane == 1) tma_tile(sbase + kATile, &tmB2, k, n0, &tma_full[st]);
+            }
+        }
+    } else if (warp == 5) {
+        // ============================ MMA issuer ============================
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16(kPM, kPN);
+            for (int it = 0; it < n_total; ++it) {
+                const int st = it % kPStages;
+                const uint32_t parity = (it / kPStages) & 1;
+                const bool sparse = it < p.n1;
+                ok = mbar_wait(sparse ? &conv_done[st] : &tma_full[st], parity, abort_flag) && ok;
+                fence_after_sync();
+                const uint32_t a_addr = s32(stages + (size_t)st * kStageBytes);
+                const uint32_t b_addr = a_addr + kATile;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
+                    if (sparse) {
+                        // A: 16 stored bf16 (32 bytes) per row and MMA; B: 32 columns (64 bytes)
+                        mma_sparse(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + (j >> 1) * kBTile + (j & 1) * 64),
+                                   tmem_base + kTmemECol + 4 * st + (j & ~1), idesc | (1u << 2) | (uint32_t)(j & 1), acc);
+                    } else {
+                        mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
+                    }
+                }
+                mma_commit(&empty[st]);          // the stage is free once these MMAs have read it
+            }
+            mma_commit(acc_full);
+        }
+    } else {
+        // ============================ converters, then epilogue ============================
+        const int row = threadIdx.x;                 // weight row inside the tile = TMEM lane
+        const int x = (row >> 3) & 1;
+        for (int it = 0; it < p.n1; ++it) {
+            const int st = it % kPStages;
+            unsigned char* sbase = stages + (size_t)st * kStageBytes;
+            ok = mbar_wait(&tma_full[st], (it / kPStages) & 1, abort_flag) && ok;
+            // ---- value bytes -> bf16 pairs, 16 bytes (one input word) at a time
+            const uint4* vrow = reinterpret_cast<const uint4*>(sbase + kATile + 2 * kBTile + row * (kPBK1 / 4));
+            unsigned char* arow = sbase + row * 128;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const uint4 v = vrow[half];
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t ws = w[c] >> 4;
+                    uint4 o;
+                    o.x = nib2bf16<0>(w[c], ws); o.y = nib2bf16<1>(w[c], ws);
+                    o.z = nib2bf16<2>(w[c], ws); o.w = nib2bf16<3>(w[c], ws);
+                    const int chunk = half * 4 + c;
+                    *reinterpret_cast<uint4*>(arow + (((chunk ^ row) & 7) << 4)) = o;
+                }
+            }
+            // ---- index words (layout in the file header)
+            const uint4 mv = *reinterpret_cast<const uint4*>(sbase + kATile + 2 * kBTile + kValsTile + row * (kPBK1 / 8));
+            const uint32_t mw[4] = {mv.x, mv.y, mv.z, mv.w};
+            uint32_t e[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t send = x ? (mw[j] & 0xFFFFu) : (mw[j] >> 16);
+                const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 8);
+                e[j] = x ? ((mw[j] & 0xFFFF0000u) | recv) : ((mw[j] & 0xFFFFu) | (recv << 16));
+            }
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + kTmemECol + 4 * st;
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
+                         :: "r"(taddr), "r"(e[0]), "r"(e[1]), "r"(e[2]), "r"(e[3]) : "memory");
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // A is read by the tensor core
+            fence_before_sync();
+            mbar_arrive(&conv_done[st]);
+        }
+        // ---- epilogue: thread = output row, TMEM columns = tokens
+        ok = mbar_wait(acc_full, 0, abort_flag) && ok;
+        fence_after_sync();
+        const int orow = m0 + row;
+#pragma unroll 1
+        for (int c0 = 0; c0 < kPN; c0 += 32) {
+            uint32_t r[32];
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + c0;
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                  "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                  "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                  "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                : "r"(taddr) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (orow < p.m_total) {
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const int token = n0 + c0 + c;
+                    if (token < p.b)
+                        p.out[(size_t)token * p.ldo + orow] = __float2bfloat16_rn(p.scale * __uint_as_float(r[c]));
+                }
+            }
+        }
+    }
+
+    if (!ok && lane == 0) flag_error(p.status, SLIM_ERR_TIMEOUT);
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        fence_after_sync();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*PfEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static PfEncodeTiledFn pf_encode_fn() {
+    static PfEncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PfEncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Row-major 2-D tensor [rows][row_elems]; box of box_rows x box_elems elements.
+static bool pf_map(CUtensorMap* map, const void* base, CUtensorMapDataType type, int esize, uint64_t row_elems,
+                   uint64_t rows, int box_elems, int box_rows, bool swizzle128) {
+    PfEncodeTiledFn fn = pf_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {row_elems, rows};
+    cuuint64_t strides[1] = {row_elems * (uint64_t)esize};
+    cuuint32_t box[2] = {(cuuint32_t)box_elems, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool prefill_supports(int b, int d_out, int d_in, int r) {
+    return b >= 1 && d_out % kPM == 0 && d_in % kPBK1 == 0 && r % 16 == 0 && r >= 0;
+}
+
+size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r) {
+    if (!prefill_supports(b, d_out, d_in, r)) return 0;
+    return ((size_t)b * (size_t)r * sizeof(__nv_bfloat16) + 255) / 256 * 256;
+}
+
+static bool g_prefill_attr_set[64];
+
+slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
+                             float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
+                             int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
+                             cudaStream_t st)
+{
+    slim_status_t err;
+    const DeviceInfo* di = device_info(&err);
+    if (!di) return err;
+    if (!prefill_supports(b, d_out, d_in, r)) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !g_prefill_attr_set[dev]) {
+        if (cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPrefillSmem) != cudaSuccess)
+            return SLIM_ERR_CUDA;
+        g_prefill_attr_set[dev] = true;
+    }
+    __nv_bfloat16* Tq = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + SLIM_WORKSPACE_SYNC_BYTES);
+    const float s_eff = s != 0.f ? s : 1.f;       // with s == 0 only the adapter term remains
+    CUtensorMap tmV, tmM, tmX, tmA2, tmB2;
+    bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPBK1 / 4, kPM, false) &&
+              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPBK1 / 8, kPM, false) &&
+              pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, kPN, true);
+    if (!ok) return SLIM_ERR_CUDA;
+    const dim3 block(kPThreads);
+    if (r > 0) {
+        // T' = (X R^T) / s : dense phase only, output rows = adapter index
+        ok = pf_map(&tmA2, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 64, kPM, true);
+        if (!ok) return SLIM_ERR_CUDA;
+        PrefillParams q;
+        q.out = Tq; q.ldo = r; q.m_total = r; q.b = b; q.n1 = 0; q.n2 = d_in / kPBK2; q.scale = 1.f / s_eff; q.status = status_dev;
+        const dim3 grid(ceil_div(r, kPM), ceil_div(b, kPN));
+        prefill_kernel<<<grid, block, kPrefillSmem, st>>>(q, tmV, tmM, tmX, tmA2, tmX);
+        count_launch(1);
+        if (cudaGetLastError() != cudaSuccess) return SLIM_ERR_CUDA;
+        ok = pf_map(&tmA2, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, 64, kPM, true) &&
+             pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, 64, kPN, true);
+        if (!ok) return SLIM_ERR_CUDA;
+    } else {
+        tmA2 = tmX; tmB2 = tmX;       // never used when r == 0
+    }
+    PrefillParams p;
+    p.out = Y; p.ldo = d_out; p.m_total = d_out; p.b = b;
+    p.n1 = s != 0.f ? d_in / kPBK1 : 0;
+    p.n2 = r > 0 ? ceil_div(r, kPBK2) : 0;
+    p.scale = s_eff; p.status = status_dev;
+    if (p.n1 + p.n2 == 0)             // s == 0 and no adapters: the result is zero
+        return cudaMemsetAsync(Y, 0, (size_t)b * d_out * 2, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+    const dim3 grid(d_out / kPM, ceil_div(b, kPN));
+    prefill_kernel<<<grid, block, kPrefillSmem, st>>>(p, tmV, tmM, tmX, tmA2, tmB2);
+    count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+}
+
+}  // namespace slim

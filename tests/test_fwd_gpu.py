@@ -52,12 +52,77 @@ def test_dispatcher_choices():
     assert K.slim_select_kernel(16, 4096, 11008, 416) == K.KERNEL_DECODE
     assert K.slim_select_kernel(8, 512, 512, 64) == K.KERNEL_DECODE
     assert K.slim_select_kernel(4, 64, 64, 16) != K.KERNEL_DECODE      # d_in not a multiple of 256
-    assert K.slim_select_kernel(17, 4096, 4096, 416) != K.KERNEL_DECODE
+    assert K.slim_select_kernel(17, 4096, 4096, 416) == K.KERNEL_PREFILL
+    assert K.slim_select_kernel(2048, 4096, 11008, 416) == K.KERNEL_PREFILL
+    assert K.slim_select_kernel(64, 48, 4096, 16) == K.KERNEL_SIMPLE        # d_out not a multiple of 128
 
 
 def test_shapes_outside_the_fast_kernels_still_work():
     assert_ok(run_case(64, 16, 16, 2, seed=31))          # d_in = 64: simple kernel
     assert_ok(run_case(320, 32, 0, 40, seed=32))         # b > 16, no adapters
+
+
+# ---- tcgen05 prefill kernel, small cases, all elements ----------------------
+PREFILL_SMALL = [  # d_in, d_out, r, b
+    (128, 128, 0, 17),       # one stage, no adapters
+    (256, 128, 16, 40),
+    (512, 256, 112, 200),    # ragged token tile, ragged rank, two row tiles
+    (1024, 384, 64, 128),    # more stages than the ring holds
+    (640, 128, 48, 8),       # a batch the dispatcher would give to the decode kernel
+    (2048, 512, 208, 300),
+]
+
+
+@pytest.mark.parametrize("d_in,d_out,r,b", PREFILL_SMALL)
+def test_small_prefill_kernel(d_in, d_out, r, b):
+    res = run_case(d_in, d_out, r, b, seed=13, kernel=K.KERNEL_PREFILL)
+    assert_ok(res)
+    assert res["launches"] == (2 if r else 1)
+
+
+def test_prefill_integer_inputs_are_exact():
+    rng = np.random.default_rng(15)
+    d_in, d_out, r, b = 256, 128, 16, 48
+    codes = rng.integers(-8, 8, size=(d_out, d_in)).astype(np.int8)
+    mask = inputs.top2_mask(rng.standard_normal((d_out, d_in)).astype(np.float32))
+    Xi = rng.integers(-1, 2, size=(b, d_in))
+    Li = rng.integers(-1, 2, size=(d_out, r))
+    Ri = (rng.random((r, d_in)) < 0.05).astype(np.int64) * rng.integers(-1, 2, size=(r, d_in))
+    vals, meta = K.slim_pack(to_dev(codes), to_dev(mask))
+    Y = K.slim_linear_fwd(K.bf16_from_bits(bf(Xi)), vals, meta, 1.0, K.bf16_from_bits(bf(Li)),
+                          K.bf16_from_bits(bf(Ri)), kernel=K.KERNEL_PREFILL)
+    exact = Xi @ (codes.astype(np.int64) * mask).T + (Xi @ Ri.T) @ Li.T
+    assert np.abs(exact).max() <= 256
+    got = inputs.bf16_bits_to_f64(K.bits_from_bf16(Y))
+    assert np.array_equal(got, exact.astype(np.float64))
+
+
+def test_prefill_one_hot_tokens_read_back_weight_columns():
+    rng = np.random.default_rng(16)
+    d_in, d_out, b = 512, 256, 64
+    codes = rng.integers(-8, 8, size=(d_out, d_in)).astype(np.int8)
+    mask = inputs.top2_mask(rng.standard_normal((d_out, d_in)).astype(np.float32))
+    vals, meta = K.slim_pack(to_dev(codes), to_dev(mask))
+    for base in (0, 61, 300):
+        ks = [(base + 7 * m) % d_in for m in range(b)]
+        X = np.zeros((b, d_in), np.float32)
+        X[np.arange(b), ks] = 1.0
+        Y = K.slim_linear_fwd(K.bf16_from_bits(bf(X)), vals, meta, 0.5, None, None, kernel=K.KERNEL_PREFILL)
+        got = inputs.bf16_bits_to_f64(K.bits_from_bf16(Y))
+        want = 0.5 * (codes.astype(np.float64) * mask)[:, ks].T
+        assert np.array_equal(got, want)
+
+
+def test_prefill_zero_scale_keeps_the_adapter_term():
+    ly = inputs.make_layer(256, 128, 32, 20, seed=17)
+    vals, meta = K.slim_pack(to_dev(ly.codes), to_dev(ly.mask))
+    X, L, R = K.bf16_from_bits(ly.X), K.bf16_from_bits(ly.L), K.bf16_from_bits(ly.R)
+    Y = K.slim_linear_fwd(X, vals, meta, 0.0, L, R, kernel=K.KERNEL_PREFILL)
+    ov, om = oracle.pack(ly.codes, ly.mask)
+    ref = oracle.linear_fwd(ly.X, ov, om, 0.0, ly.L, ly.R)
+    assert parity.compare(inputs.bf16_bits_to_f64(K.bits_from_bf16(Y)), ref)["ok"]
+    Y0 = K.slim_linear_fwd(X, vals, meta, 0.0, None, None, kernel=K.KERNEL_PREFILL)
+    assert float(Y0.float().abs().max()) == 0.0
 
 
 # ---- exact cases ------------------------------------------------------------
@@ -165,3 +230,22 @@ def test_full_size_decode_configs(d_in, d_out, r, b, seed, wseed):
     benchmark times (dispatcher's choice); all tokens compared."""
     assert K.slim_select_kernel(b, d_out, d_in, r) == K.KERNEL_DECODE
     assert_ok(run_case(d_in, d_out, r, b, seed, wseed))
+
+
+def prefill_cases(cfgs):
+    out = []
+    for cfg in cfgs:
+        for name, d_in, d_out, r, b, seed, wseed in inputs.config_cases(cfg):
+            if b > 16:
+                out.append(pytest.param(d_in, d_out, r, b, seed, wseed, id=f"cfg{cfg}-{name}-b{b}-r{r}"))
+    return out
+
+
+@pytest.mark.parametrize("d_in,d_out,r,b,seed,wseed", prefill_cases([2, 3, 4]))
+def test_full_size_prefill_configs(d_in, d_out, r, b, seed, wseed):
+    """2048- and 4096-token cases of configurations 2, 3 and 4 in the launch the
+    dispatcher picks; compared on sampled token rows (first, middle and last
+    rows of the edge tiles plus one seeded row in every other 128-token tile)."""
+    assert K.slim_select_kernel(b, d_out, d_in, r) == K.KERNEL_PREFILL
+    rows = inputs.sample_rows(b, tile=128, seed=seed, dense_edges=False)
+    assert_ok(run_case(d_in, d_out, r, b, seed, wseed, rows=rows))
