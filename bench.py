@@ -343,6 +343,7 @@ def run_ours(args):
 
     if rank == 0 and not args.skip_extras:
         line["per_case"] = per_case_table(K, lib, layers, ws, ws_bytes, status, stream, peak)
+        line["prefill"] = prefill_table(K, layers, stream)
         line["pack"] = time_pack(K, layers[1], stream)
     # ---- end to end through the host-buffer entry point
     line["e2e"] = time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, world, barrier)
@@ -406,6 +407,50 @@ def per_case_table(K, lib, layers, ws, ws_bytes, status, stream, peak):
                          "frac_measured": round(gbs / peak, 4), "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
                          "executed_TFLOPs": round(executed_flops(ly["d_in"], ly["d_out"], ly["r"], b) / (med * 1e-6) / 1e12, 2)})
         del copies
+    return rows
+
+
+def dense_tflops_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
+def prefill_table(K, layers, stream, tokens=2048):
+    """The same three layers at 2048 tokens (tcgen05 prefill kernel): us/call,
+    dense-equivalent TFLOP/s (the 2:4 product counted as if dense, adapters at
+    face value) and its fraction of the sparse bf16 peak, taken as twice the
+    measured dense bf16 peak."""
+    import torch
+    dense_peak, kind = dense_tflops_peak()
+    rows = []
+    for ly in layers:
+        X = K.bf16_from_bits(inputs.make_activations(tokens, ly["d_in"], 7))
+        Y = torch.empty((tokens, ly["d_out"]), dtype=torch.bfloat16, device=X.device)
+        ws = K.new_workspace(tokens, ly["d_out"], ly["d_in"], ly["r"])
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                K.slim_linear_fwd(X, ly["vals"], ly["meta"], ly["s"], ly["Ld"], ly["Rd"], Y=Y, workspace=ws)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = 20
+            e0.record(stream)
+            for _ in range(n):
+                K.slim_linear_fwd(X, ly["vals"], ly["meta"], ly["s"], ly["Ld"], ly["Rd"], Y=Y, workspace=ws)
+            e1.record(stream)
+            e1.synchronize()
+        us = 1e3 * e0.elapsed_time(e1) / n
+        dense_eq = 2.0 * tokens * ly["d_out"] * ly["d_in"] + 2.0 * tokens * ly["r"] * (ly["d_in"] + ly["d_out"])
+        tf = dense_eq / (us * 1e-6) / 1e12
+        rows.append({"layer": ly["name"], "d_in": ly["d_in"], "d_out": ly["d_out"], "r": ly["r"], "tokens": tokens,
+                     "kernel": K.KERNEL_NAMES[K.slim_select_kernel(tokens, ly["d_out"], ly["d_in"], ly["r"])],
+                     "us": round(us, 2), "dense_equiv_TFLOPs": round(tf, 1),
+                     "executed_TFLOPs": round(executed_flops(ly["d_in"], ly["d_out"], ly["r"], tokens) / (us * 1e-6) / 1e12, 1),
+                     "frac_of_sparse_peak": round(tf / (2 * dense_peak), 4), "sparse_peak_TFLOPs": 2 * dense_peak,
+                     "peak_kind": f"2 x dense bf16 of {kind}", "frac_of_nominal_4500": round(tf / 4500.0, 4)})
+        del X, Y, ws
     return rows
 
 

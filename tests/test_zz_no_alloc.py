@@ -51,7 +51,7 @@ def test_noalloc_matches_the_workspace_entry_point_twice(d_in, d_out, r, b):
         before = torch.cuda.memory_allocated()
         K.slim_linear_fwd_noalloc(X, vals, meta, ly.s, L, R, got, status=status)
         assert K.slim_last_launch_count() == 1
-        assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.memory_allocated() <= before     # torch may free earlier temporaries, never grow
         torch.cuda.synchronize()
         assert K.read_status(status) == 0
         res = parity.compare(inputs.bf16_bits_to_f64(K.bits_from_bf16(got)),
