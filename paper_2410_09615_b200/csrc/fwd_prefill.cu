@@ -1,12 +1,12 @@
 // Prefill-phase forward (many tokens): tcgen05 tensor cores with the accumulator
 // in tensor memory.
 //
-// One CTA computes a 128 (output rows) x 128 (tokens) tile of
+// One CTA computes a 128 (output rows) x N (tokens; N = 256, or 64 for small problems) tile of
 //     out[token][row] = scale * ( sum_k W[row][k] X[token][k]  +  sum_j A2[row][j] B2[token][j] )
 // in two chained phases that accumulate into the same TMEM tile:
 //   phase 1 (sparse): W is the packed int4 2:4 weight.  TMA brings 128 rows of value
-//       bytes and index bytes plus the X tile; four converter warps (one thread per
-//       weight row) expand nibbles to exact bf16 into the 128-byte-swizzled K-major
+//       bytes and index bytes plus the X tile; eight converter warps (two threads per
+//       weight row) expand nibbles to exact bf16 into the 64-byte-swizzled K-major
 //       layout the MMA reads, and write the 2:4 index words into tensor memory;
 //       one thread issues tcgen05.mma.sp (kind::f16, bf16 x bf16 -> fp32).
 //   phase 2 (dense): A2 and B2 are bf16 matrices brought by TMA as they are; the same
@@ -23,7 +23,9 @@
 // packed index array is one row's 32 columns, so a converter thread swaps one
 // half-word with the thread eight rows away and stores the result.
 //
-// Pipeline: 4 stages of {A 16 KB, B 32 KB, value bytes 4 KB, index bytes 2 KB};
+// Pipeline: 4 stages of {B N x 128 B, A 16 KB (8 KB used in phase 1), value bytes 2 KB,
+// index bytes 1 KB}; a stage is 64 weight columns (two sparse MMAs of K = 32, or four
+// dense MMAs of K = 16);
 // mbarriers: tma_full (TMA bytes landed), conv_done (converters finished a stage),
 // empty (tcgen05.commit: the MMAs that read the stage are complete), acc_full.
 // Every wait is bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on.
@@ -33,20 +35,22 @@
 namespace slim {
 
 constexpr int kPM = 128;            // output rows per CTA (MMA M)
-constexpr int kPN = 128;            // tokens per CTA (MMA N)
-constexpr int kPBK1 = 128;          // weight columns per stage in the sparse phase (4 MMAs of K = 32)
-constexpr int kPBK2 = 64;           // columns per stage in the dense phase (4 MMAs of K = 16)
+constexpr int kPBK = 64;            // columns per stage, both phases
 constexpr int kPStages = 4;
-constexpr int kPThreads = 192;      // warps 0-3 converters / epilogue, warp 4 TMA, warp 5 MMA
-constexpr int kATile = kPM * 128;               // 16 KB: 128 rows x 128 bytes
-constexpr int kBTile = kPN * 128;               // 16 KB: 128 tokens x 128 bytes
-constexpr int kValsTile = kPM * (kPBK1 / 4);    // 4 KB
-constexpr int kMetaTile = kPM * (kPBK1 / 8);    // 2 KB
-constexpr int kStageBytes = kATile + 2 * kBTile + kValsTile + kMetaTile;
-constexpr int kTmemCols = 256;      // accumulator: columns 0-127; index words: 128 + 4 * stage + mma
-constexpr int kTmemECol = 128;
+constexpr int kConvWarps = 8;       // warps 0-7 converters / epilogue, warp 8 TMA, warp 9 MMA
+constexpr int kPThreads = 32 * (kConvWarps + 2);
+constexpr int kATile = kPM * 128;               // 16 KB: 128 rows x 128 bytes (dense phase)
+constexpr int kValsTile = kPM * (kPBK / 4);     // 2 KB
+constexpr int kMetaTile = kPM * (kPBK / 8);     // 1 KB
 constexpr uint32_t kPSpinLimit = 1u << 21;
-constexpr size_t kPrefillSmem = 1024 + (size_t)kPStages * kStageBytes + 256;
+
+template <int N> struct PfCfg {
+    static constexpr int kBTile = N * 128;                                  // N tokens x 128 bytes
+    static constexpr int kStageBytes = kBTile + kATile + kValsTile + kMetaTile;
+    static constexpr int kECol = N;                                         // index words: N + 4 * stage + mma
+    static constexpr int kTmemCols = N >= 256 ? 512 : (N >= 128 ? 256 : 128);
+    static constexpr size_t kSmem = 1024 + (size_t)kPStages * kStageBytes + 256;
+};
 
 struct PrefillParams {
     __nv_bfloat16* out;     // [tokens][ldo]
@@ -99,6 +103,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
+// Same with 64-byte rows and 64-byte swizzle (8-row groups 512 bytes apart).
+__device__ __forceinline__ uint64_t smem_desc64(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(512 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)4 << 61);
+}
 // Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, both K-major.
 __host__ __device__ constexpr uint32_t idesc_bf16(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
@@ -141,13 +150,17 @@ __device__ __forceinline__ uint32_t nib2bf16(uint32_t w, uint32_t w_shr4) {
 
 }  // namespace pf
 
+template <int N>
 __global__ void __launch_bounds__(kPThreads, 1)
 prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmX,
                const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2)
 {
     using namespace pf;
+    using Cfg = PfCfg<N>;
+    constexpr int kBTile = Cfg::kBTile, kStageBytes = Cfg::kStageBytes, kECol = Cfg::kECol;
     extern __shared__ unsigned char smem_raw[];
+    // stage layout: B | A | value bytes | index bytes
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = reinterpret_cast<uint64_t*>(stages + (size_t)kPStages * kStageBytes);
     uint64_t* tma_full = bars;                       // [kPStages]
@@ -158,17 +171,17 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kPM, n0 = blockIdx.y * kPN;
+    const int m0 = blockIdx.x * kPM, n0 = blockIdx.y * N;
     const int n_total = p.n1 + p.n2;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kPStages; ++i) { mbar_init(&tma_full[i], 1); mbar_init(&conv_done[i], kPM); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < kPStages; ++i) { mbar_init(&tma_full[i], 1); mbar_init(&conv_done[i], 32 * kConvWarps); mbar_init(&empty[i], 1); }
         mbar_init(acc_full, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s32(tmem_slot)), "r"(kTmemCols) : "memory");
+    if (warp == kConvWarps + 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s32(tmem_slot)), "r"(Cfg::kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     fence_before_sync();
@@ -177,52 +190,52 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
     bool ok = true;
 
-    if (warp == 4) {
+    if (warp == kConvWarps) {
         // ============================ TMA producer ============================
-        // lane 0 runs the ring protocol; lanes 0-3 each request one tile of a stage
+        // lane 0 runs the ring protocol; lanes 0-2 each request one tile of a stage
         for (int it = 0; it < n_total; ++it) {
             const int st = it % kPStages;
             unsigned char* sbase = stages + (size_t)st * kStageBytes;
             const bool sparse = it < p.n1;
             if (lane == 0) {
                 if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
-                mbar_expect_tx(&tma_full[st], sparse ? (uint32_t)(kValsTile + kMetaTile + 2 * kBTile) : (uint32_t)(kATile + kBTile));
+                mbar_expect_tx(&tma_full[st], sparse ? (uint32_t)(kValsTile + kMetaTile + kBTile) : (uint32_t)(kATile + kBTile));
             }
             __syncwarp();
             if (sparse) {
-                const int k = it * kPBK1;
-                if (lane == 0) tma_tile(sbase + kATile + 2 * kBTile, &tmV, k / 4, m0, &tma_full[st]);
-                else if (lane == 1) tma_tile(sbase + kATile + 2 * kBTile + kValsTile, &tmM, k / 8, m0, &tma_full[st]);
-                else if (lane == 2) tma_tile(sbase + kATile, &tmX, k, n0, &tma_full[st]);
-                else if (lane == 3) tma_tile(sbase + kATile + kBTile, &tmX, k + 64, n0, &tma_full[st]);
+                const int k = it * kPBK;
+                if (lane == 0) tma_tile(sbase, &tmX, k, n0, &tma_full[st]);
+                else if (lane == 1) tma_tile(sbase + kBTile + kATile, &tmV, k / 4, m0, &tma_full[st]);
+                else if (lane == 2) tma_tile(sbase + kBTile + kATile + kValsTile, &tmM, k / 8, m0, &tma_full[st]);
             } else {
-                const int k = (it - p.n1) * kPBK2;
-                if (lane == 0) tma_tile(sbase, &tmA2, k, m0, &tma_full[st]);
-                else if (lane == 1) tma_tile(sbase + kATile, &tmB2, k, n0, &tma_full[st]);
+                const int k = (it - p.n1) * kPBK;
+                if (lane == 0) tma_tile(sbase, &tmB2, k, n0, &tma_full[st]);
+                else if (lane == 1) tma_tile(sbase + kBTile, &tmA2, k, m0, &tma_full[st]);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kConvWarps + 1) {
         // ============================ MMA issuer ============================
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16(kPM, kPN);
+            constexpr uint32_t idesc = idesc_bf16(kPM, N);
             for (int it = 0; it < n_total; ++it) {
                 const int st = it % kPStages;
                 const uint32_t parity = (it / kPStages) & 1;
                 const bool sparse = it < p.n1;
                 ok = mbar_wait(sparse ? &conv_done[st] : &tma_full[st], parity, abort_flag) && ok;
                 fence_after_sync();
-                const uint32_t a_addr = s32(stages + (size_t)st * kStageBytes);
-                const uint32_t b_addr = a_addr + kATile;
+                const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
+                const uint32_t a_addr = b_addr + kBTile;
+                if (sparse) {
+                    // per MMA: A 16 stored bf16 (32 bytes of a 64-byte row), B 32 columns (64 bytes)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
-                    if (sparse) {
-                        // A: 16 stored bf16 (32 bytes) per row and MMA; B: 32 columns (64 bytes)
-                        mma_sparse(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + (j >> 1) * kBTile + (j & 1) * 64),
-                                   tmem_base + kTmemECol + 4 * st + (j & ~1), idesc | (1u << 2) | (uint32_t)(j & 1), acc);
-                    } else {
-                        mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
-                    }
+                    for (int j = 0; j < 2; ++j)
+                        mma_sparse(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
+                                   tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, (it > 0 || j > 0) ? 1u : 0u);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc,
+                                  (it > 0 || j > 0) ? 1u : 0u);
                 }
                 mma_commit(&empty[st]);          // the stage is free once these MMAs have read it
             }
@@ -230,55 +243,47 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
         }
     } else {
         // ============================ converters, then epilogue ============================
-        const int row = threadIdx.x;                 // weight row inside the tile = TMEM lane
+        const int row = threadIdx.x & 127;           // weight row inside the tile = TMEM lane
+        const int half = threadIdx.x >> 7;           // which 32 of the stage's 64 columns this thread expands
         const int x = (row >> 3) & 1;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         for (int it = 0; it < p.n1; ++it) {
             const int st = it % kPStages;
             unsigned char* sbase = stages + (size_t)st * kStageBytes;
             ok = mbar_wait(&tma_full[st], (it / kPStages) & 1, abort_flag) && ok;
-            // ---- value bytes -> bf16 pairs, 16 bytes (one input word) at a time
-            const uint4* vrow = reinterpret_cast<const uint4*>(sbase + kATile + 2 * kBTile + row * (kPBK1 / 4));
-            unsigned char* arow = sbase + row * 128;
+            // ---- 8 value bytes -> 16 bf16: two 16-byte chunks of the row (64-byte rows, 64-byte swizzle)
+            const uint2 v = *reinterpret_cast<const uint2*>(sbase + kBTile + kATile + row * (kPBK / 4) + 8 * half);
+            unsigned char* arow = sbase + kBTile + row * 64;
+            const uint32_t w[2] = {v.x, v.y};
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const uint4 v = vrow[half];
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t ws = w[c] >> 4;
-                    uint4 o;
-                    o.x = nib2bf16<0>(w[c], ws); o.y = nib2bf16<1>(w[c], ws);
-                    o.z = nib2bf16<2>(w[c], ws); o.w = nib2bf16<3>(w[c], ws);
-                    const int chunk = half * 4 + c;
-                    *reinterpret_cast<uint4*>(arow + (((chunk ^ row) & 7) << 4)) = o;
-                }
+            for (int c = 0; c < 2; ++c) {
+                const uint32_t ws = w[c] >> 4;
+                uint4 o;
+                o.x = nib2bf16<0>(w[c], ws); o.y = nib2bf16<1>(w[c], ws);
+                o.z = nib2bf16<2>(w[c], ws); o.w = nib2bf16<3>(w[c], ws);
+                const int chunk = half * 2 + c;
+                *reinterpret_cast<uint4*>(arow + (((chunk ^ (row >> 1)) & 3) << 4)) = o;
             }
-            // ---- index words (layout in the file header)
-            const uint4 mv = *reinterpret_cast<const uint4*>(sbase + kATile + 2 * kBTile + kValsTile + row * (kPBK1 / 8));
-            const uint32_t mw[4] = {mv.x, mv.y, mv.z, mv.w};
-            uint32_t e[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t send = x ? (mw[j] & 0xFFFFu) : (mw[j] >> 16);
-                const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 8);
-                e[j] = x ? ((mw[j] & 0xFFFF0000u) | recv) : ((mw[j] & 0xFFFFu) | (recv << 16));
-            }
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + kTmemECol + 4 * st;
-            asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
-                         :: "r"(taddr), "r"(e[0]), "r"(e[1]), "r"(e[2]), "r"(e[3]) : "memory");
+            // ---- index word of MMA `half` (layout in the file header)
+            const uint32_t mw = *reinterpret_cast<const uint32_t*>(sbase + kBTile + kATile + kValsTile + row * (kPBK / 8) + 4 * half);
+            const uint32_t send = x ? (mw & 0xFFFFu) : (mw >> 16);
+            const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 8);
+            const uint32_t e = x ? ((mw & 0xFFFF0000u) | recv) : ((mw & 0xFFFFu) | (recv << 16));
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};"
+                         :: "r"(tmem_base + lane_base + kECol + 4 * st + half), "r"(e) : "memory");
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // A is read by the tensor core
             fence_before_sync();
             mbar_arrive(&conv_done[st]);
         }
-        // ---- epilogue: thread = output row, TMEM columns = tokens
+        // ---- epilogue: thread = output row, TMEM columns = tokens; the two halves split the columns
         ok = mbar_wait(acc_full, 0, abort_flag) && ok;
         fence_after_sync();
         const int orow = m0 + row;
 #pragma unroll 1
-        for (int c0 = 0; c0 < kPN; c0 += 32) {
+        for (int c0 = half * (N / 2); c0 < (half + 1) * (N / 2); c0 += 32) {
             uint32_t r[32];
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + c0;
+            const uint32_t taddr = tmem_base + lane_base + c0;
             asm volatile(
                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -303,9 +308,9 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     if (!ok && lane == 0) flag_error(p.status, SLIM_ERR_TIMEOUT);
     fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kConvWarps + 1) {
         fence_after_sync();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(Cfg::kTmemCols) : "memory");
     }
 }
 
@@ -341,7 +346,7 @@ static bool pf_map(CUtensorMap* map, const void* base, CUtensorMapDataType type,
 }
 
 bool prefill_supports(int b, int d_out, int d_in, int r) {
-    return b >= 1 && d_out % kPM == 0 && d_in % kPBK1 == 0 && r % 16 == 0 && r >= 0;
+    return b >= 1 && d_out % kPM == 0 && d_in % kPBK == 0 && r % 16 == 0 && r >= 0;
 }
 
 size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r) {
@@ -350,6 +355,16 @@ size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r) {
 }
 
 static bool g_prefill_attr_set[64];
+
+template <int N>
+static slim_status_t launch_tile_kernel(const PrefillParams& q, int m_rows, const CUtensorMap& tmV, const CUtensorMap& tmM,
+                                        const CUtensorMap& tmX, const CUtensorMap& tmA2, const CUtensorMap& tmB2,
+                                        cudaStream_t st) {
+    const dim3 grid(ceil_div(m_rows, kPM), ceil_div(q.b, N)), block(kPThreads);
+    prefill_kernel<N><<<grid, block, PfCfg<N>::kSmem, st>>>(q, tmV, tmM, tmX, tmA2, tmB2);
+    count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+}
 
 slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
                              float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
@@ -363,45 +378,46 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !g_prefill_attr_set[dev]) {
-        if (cudaFuncSetAttribute(prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPrefillSmem) != cudaSuccess)
+        if (cudaFuncSetAttribute(prefill_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256>::kSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<64>::kSmem) != cudaSuccess)
             return SLIM_ERR_CUDA;
         g_prefill_attr_set[dev] = true;
     }
     __nv_bfloat16* Tq = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + SLIM_WORKSPACE_SYNC_BYTES);
     const float s_eff = s != 0.f ? s : 1.f;       // with s == 0 only the adapter term remains
-    CUtensorMap tmV, tmM, tmX, tmA2, tmB2;
-    bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPBK1 / 4, kPM, false) &&
-              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPBK1 / 8, kPM, false) &&
-              pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, kPN, true);
+    // token tile: 256 when that still gives every SM a tile, else 64
+    const bool wide = (long long)(d_out / kPM) * ceil_div(b, 256) >= di->sm_count;
+    const int n_main = wide ? 256 : 64;
+    const int n_pre = 64;                         // the T' product has few row tiles: narrow token tiles fill the machine
+    CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;
+    bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPBK / 4, kPM, false) &&
+              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPBK / 8, kPM, false) &&
+              pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, n_main, true);
     if (!ok) return SLIM_ERR_CUDA;
-    const dim3 block(kPThreads);
     if (r > 0) {
         // T' = (X R^T) / s : dense phase only, output rows = adapter index
-        ok = pf_map(&tmA2, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 64, kPM, true);
+        ok = pf_map(&tmA2, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 64, kPM, true) &&
+             pf_map(&tmXpre, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, n_pre, true);
         if (!ok) return SLIM_ERR_CUDA;
         PrefillParams q;
-        q.out = Tq; q.ldo = r; q.m_total = r; q.b = b; q.n1 = 0; q.n2 = d_in / kPBK2; q.scale = 1.f / s_eff; q.status = status_dev;
-        const dim3 grid(ceil_div(r, kPM), ceil_div(b, kPN));
-        prefill_kernel<<<grid, block, kPrefillSmem, st>>>(q, tmV, tmM, tmX, tmA2, tmX);
-        count_launch(1);
-        if (cudaGetLastError() != cudaSuccess) return SLIM_ERR_CUDA;
+        q.out = Tq; q.ldo = r; q.m_total = r; q.b = b; q.n1 = 0; q.n2 = d_in / kPBK; q.scale = 1.f / s_eff; q.status = status_dev;
+        slim_status_t rc = launch_tile_kernel<64>(q, r, tmV, tmM, tmXpre, tmA2, tmXpre, st);
+        if (rc != SLIM_OK) return rc;
         ok = pf_map(&tmA2, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, 64, kPM, true) &&
-             pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, 64, kPN, true);
+             pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, 64, n_main, true);
         if (!ok) return SLIM_ERR_CUDA;
     } else {
         tmA2 = tmX; tmB2 = tmX;       // never used when r == 0
     }
     PrefillParams p;
     p.out = Y; p.ldo = d_out; p.m_total = d_out; p.b = b;
-    p.n1 = s != 0.f ? d_in / kPBK1 : 0;
-    p.n2 = r > 0 ? ceil_div(r, kPBK2) : 0;
+    p.n1 = s != 0.f ? d_in / kPBK : 0;
+    p.n2 = r > 0 ? ceil_div(r, kPBK) : 0;
     p.scale = s_eff; p.status = status_dev;
     if (p.n1 + p.n2 == 0)             // s == 0 and no adapters: the result is zero
         return cudaMemsetAsync(Y, 0, (size_t)b * d_out * 2, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
-    const dim3 grid(d_out / kPM, ceil_div(b, kPN));
-    prefill_kernel<<<grid, block, kPrefillSmem, st>>>(p, tmV, tmM, tmX, tmA2, tmB2);
-    count_launch(1);
-    return cudaGetLastError() == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+    return wide ? launch_tile_kernel<256>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st)
+                : launch_tile_kernel<64>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
 }
 
 }  // namespace slim
