@@ -24,7 +24,7 @@
 // half-word with the thread eight rows away and stores the result.
 //
 // Pipeline: 4 stages of {B N x 128 B, A 16 KB (8 KB used in phase 1), value bytes 2 KB,
-// index bytes 1 KB}; a stage is 64 weight columns (two sparse MMAs of K = 32, or four
+// index bytes 2 KB (16 per row, of which a stage uses 8)}; a stage is 64 weight columns (two sparse MMAs of K = 32, or four
 // dense MMAs of K = 16);
 // mbarriers: tma_full (TMA bytes landed), conv_done (converters finished a stage),
 // empty (tcgen05.commit: the MMAs that read the stage are complete), acc_full.
@@ -41,7 +41,7 @@ constexpr int kConvWarps = 8;       // warps 0-7 converters / epilogue, warp 8 T
 constexpr int kPThreads = 32 * (kConvWarps + 2);
 constexpr int kATile = kPM * 128;               // 16 KB: 128 rows x 128 bytes (dense phase)
 constexpr int kValsTile = kPM * (kPBK / 4);     // 2 KB
-constexpr int kMetaTile = kPM * (kPBK / 8);     // 1 KB
+constexpr int kMetaTile = kPM * 16;             // 2 KB: a TMA row is at least 16 bytes = two stages of index bytes
 constexpr uint32_t kPSpinLimit = 1u << 21;
 
 template <int N> struct PfCfg {
@@ -206,7 +206,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 const int k = it * kPBK;
                 if (lane == 0) tma_tile(sbase, &tmX, k, n0, &tma_full[st]);
                 else if (lane == 1) tma_tile(sbase + kBTile + kATile, &tmV, k / 4, m0, &tma_full[st]);
-                else if (lane == 2) tma_tile(sbase + kBTile + kATile + kValsTile, &tmM, k / 8, m0, &tma_full[st]);
+                else if (lane == 2) tma_tile(sbase + kBTile + kATile + kValsTile, &tmM, (k / 8) & ~15, m0, &tma_full[st]);
             } else {
                 const int k = (it - p.n1) * kPBK;
                 if (lane == 0) tma_tile(sbase, &tmB2, k, n0, &tma_full[st]);
@@ -265,7 +265,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 *reinterpret_cast<uint4*>(arow + (((chunk ^ (row >> 1)) & 3) << 4)) = o;
             }
             // ---- index word of MMA `half` (layout in the file header)
-            const uint32_t mw = *reinterpret_cast<const uint32_t*>(sbase + kBTile + kATile + kValsTile + row * (kPBK / 8) + 4 * half);
+            const uint32_t mw = *reinterpret_cast<const uint32_t*>(sbase + kBTile + kATile + kValsTile + row * 16 + 8 * (it & 1) + 4 * half);
             const uint32_t send = x ? (mw & 0xFFFFu) : (mw >> 16);
             const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 8);
             const uint32_t e = x ? ((mw & 0xFFFF0000u) | recv) : ((mw & 0xFFFFu) | (recv << 16));
@@ -391,7 +391,7 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     const int n_pre = 64;                         // the T' product has few row tiles: narrow token tiles fill the machine
     CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;
     bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPBK / 4, kPM, false) &&
-              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPBK / 8, kPM, false) &&
+              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, 16, kPM, false) &&
               pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, n_main, true);
     if (!ok) return SLIM_ERR_CUDA;
     if (r > 0) {
