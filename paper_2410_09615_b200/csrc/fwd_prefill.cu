@@ -23,11 +23,15 @@
 // packed index array is one row's 32 columns, so a converter thread swaps one
 // half-word with the thread eight rows away and stores the result.
 //
-// Pipeline: 4 stages of {B N x 128 B, A 16 KB (8 KB used in phase 1), value bytes 2 KB,
-// index bytes 2 KB (16 per row, of which a stage uses 8)}; a stage is 64 weight columns (two sparse MMAs of K = 32, or four
-// dense MMAs of K = 16);
-// mbarriers: tma_full (TMA bytes landed), conv_done (converters finished a stage),
-// empty (tcgen05.commit: the MMAs that read the stage are complete), acc_full.
+// Pipeline.  4 stages of {B: N tokens x 128 bytes, A: 16 KB (8 KB used in phase 1)}; a
+// stage is 64 weight columns (two sparse MMAs of K = 32, or four dense MMAs of K = 16).
+// The packed value and index bytes travel separately, 256 columns (4 stages) per TMA tile,
+// through a 2-slot ring of their own.  A thread is held ~160 ns by every TMA request it
+// starts, so requests are spread over three producer warps: token tiles of even stages,
+// token tiles of odd stages, packed tiles and A2 tiles.
+// mbarriers: b_full / a2_full / pk_full (TMA bytes landed), conv_done (converters
+// finished a stage), empty / pk_empty (tcgen05.commit: the MMAs that read the stage are
+// complete; converters done with a packed slot), acc_full.
 // Every wait is bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on.
 #include <cuda.h>
 #include "common.cuh"
@@ -37,19 +41,23 @@ namespace slim {
 constexpr int kPM = 128;            // output rows per CTA (MMA M)
 constexpr int kPBK = 64;            // columns per stage, both phases
 constexpr int kPStages = 4;
-constexpr int kConvWarps = 8;       // warps 0-7 converters / epilogue, warp 8 TMA, warp 9 MMA
-constexpr int kPThreads = 32 * (kConvWarps + 2);
+constexpr int kPkStages = 4;        // stages covered by one packed tile (256 weight columns)
+constexpr int kPkSlots = 2;
+constexpr int kConvWarps = 8;       // warps 0-7 converters / epilogue
+constexpr int kWarpXEven = 8, kWarpMma = 9, kWarpXOdd = 10, kWarpPk = 11;
+constexpr int kPThreads = 32 * 12;
 constexpr int kATile = kPM * 128;               // 16 KB: 128 rows x 128 bytes (dense phase)
-constexpr int kValsTile = kPM * (kPBK / 4);     // 2 KB
-constexpr int kMetaTile = kPM * 16;             // 2 KB: a TMA row is at least 16 bytes = two stages of index bytes
+constexpr int kValsTile = kPM * (kPkStages * kPBK / 4);     // 8 KB: 64 value bytes per row
+constexpr int kMetaTile = kPM * (kPkStages * kPBK / 8);     // 4 KB: 32 index bytes per row
+constexpr int kPkSlotBytes = kValsTile + kMetaTile;
 constexpr uint32_t kPSpinLimit = 1u << 21;
 
 template <int N> struct PfCfg {
     static constexpr int kBTile = N * 128;                                  // N tokens x 128 bytes
-    static constexpr int kStageBytes = kBTile + kATile + kValsTile + kMetaTile;
+    static constexpr int kStageBytes = kBTile + kATile;
     static constexpr int kECol = N;                                         // index words: N + 4 * stage + mma
     static constexpr int kTmemCols = N >= 256 ? 512 : (N >= 128 ? 256 : 128);
-    static constexpr size_t kSmem = 1024 + (size_t)kPStages * kStageBytes + 256;
+    static constexpr size_t kSmem = 1024 + (size_t)kPStages * kStageBytes + kPkSlots * kPkSlotBytes + 512;
 };
 
 struct PrefillParams {
@@ -61,6 +69,16 @@ struct PrefillParams {
     float scale;
     uint32_t* status;
 };
+
+// Optional timeline: built with -DSLIM_PREFILL_TRACE, one thread per warp role of the first
+// CTAs records the global timer around its waits for the first 48 stages.
+#ifdef SLIM_PREFILL_TRACE
+__device__ unsigned long long g_ptrace[8][6][48];
+#define PSTAMP(role, it) do { if (blockIdx.x + gridDim.x * blockIdx.y < 8 && (it) < 48) { unsigned long long t_; \
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_ptrace[blockIdx.x + gridDim.x * blockIdx.y][role][it] = t_; } } while (0)
+#else
+#define PSTAMP(role, it) do { } while (0)
+#endif
 
 namespace pf {
 
@@ -160,14 +178,18 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     using Cfg = PfCfg<N>;
     constexpr int kBTile = Cfg::kBTile, kStageBytes = Cfg::kStageBytes, kECol = Cfg::kECol;
     extern __shared__ unsigned char smem_raw[];
-    // stage layout: B | A | value bytes | index bytes
+    // layout: stages {B | A} | packed slots {value bytes | index bytes} | barriers
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(stages + (size_t)kPStages * kStageBytes);
-    uint64_t* tma_full = bars;                       // [kPStages]
-    uint64_t* conv_done = bars + kPStages;           // [kPStages]
-    uint64_t* empty = bars + 2 * kPStages;           // [kPStages]
-    uint64_t* acc_full = bars + 3 * kPStages;        // [1]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kPStages + 1);
+    unsigned char* packed = stages + (size_t)kPStages * kStageBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(packed + kPkSlots * kPkSlotBytes);
+    uint64_t* b_full = bars;                         // [kPStages] token tile landed
+    uint64_t* a2_full = bars + kPStages;             // [kPStages] dense-phase A tile landed
+    uint64_t* conv_done = bars + 2 * kPStages;       // [kPStages]
+    uint64_t* empty = bars + 3 * kPStages;           // [kPStages]
+    uint64_t* pk_full = bars + 4 * kPStages;         // [kPkSlots]
+    uint64_t* pk_empty = pk_full + kPkSlots;         // [kPkSlots]
+    uint64_t* acc_full = pk_empty + kPkSlots;        // [1]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -175,12 +197,16 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     const int n_total = p.n1 + p.n2;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kPStages; ++i) { mbar_init(&tma_full[i], 1); mbar_init(&conv_done[i], 32 * kConvWarps); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < kPStages; ++i) {
+            mbar_init(&b_full[i], 1); mbar_init(&a2_full[i], 1);
+            mbar_init(&conv_done[i], 32 * kConvWarps); mbar_init(&empty[i], 1);
+        }
+        for (int i = 0; i < kPkSlots; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], 32 * kConvWarps); }
         mbar_init(acc_full, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kConvWarps + 1) {
+    if (warp == kWarpMma) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s32(tmem_slot)), "r"(Cfg::kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -190,30 +216,42 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
     bool ok = true;
 
-    if (warp == kConvWarps) {
-        // ============================ TMA producer ============================
-        // lane 0 runs the ring protocol; lanes 0-2 each request one tile of a stage
-        for (int it = 0; it < n_total; ++it) {
-            const int st = it % kPStages;
-            unsigned char* sbase = stages + (size_t)st * kStageBytes;
-            const bool sparse = it < p.n1;
-            if (lane == 0) {
+    if (warp == kWarpXEven || warp == kWarpXOdd) {
+        // ============================ token-tile producers ============================
+        if (lane == 0) {
+            for (int it = warp == kWarpXEven ? 0 : 1; it < n_total; it += 2) {
+                const int st = it % kPStages;
+                const bool sparse = it < p.n1;
                 if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
-                mbar_expect_tx(&tma_full[st], sparse ? (uint32_t)(kValsTile + kMetaTile + kBTile) : (uint32_t)(kATile + kBTile));
-            }
-            __syncwarp();
-            if (sparse) {
-                const int k = it * kPBK;
-                if (lane == 0) tma_tile(sbase, &tmX, k, n0, &tma_full[st]);
-                else if (lane == 1) tma_tile(sbase + kBTile + kATile, &tmV, k / 4, m0, &tma_full[st]);
-                else if (lane == 2) tma_tile(sbase + kBTile + kATile + kValsTile, &tmM, (k / 8) & ~15, m0, &tma_full[st]);
-            } else {
-                const int k = (it - p.n1) * kPBK;
-                if (lane == 0) tma_tile(sbase, &tmB2, k, n0, &tma_full[st]);
-                else if (lane == 1) tma_tile(sbase + kBTile, &tmA2, k, m0, &tma_full[st]);
+                mbar_expect_tx(&b_full[st], (uint32_t)kBTile);
+                tma_tile(stages + (size_t)st * kStageBytes, sparse ? &tmX : &tmB2,
+                         sparse ? it * kPBK : (it - p.n1) * kPBK, n0, &b_full[st]);
+                PSTAMP(0, it);
             }
         }
-    } else if (warp == kConvWarps + 1) {
+    } else if (warp == kWarpPk) {
+        // ============================ packed-tile and A2 producer ============================
+        // lanes 0 and 1 request the value-byte and the index-byte tile with one instruction
+        const int n_groups = ceil_div(p.n1, kPkStages);
+        for (int gi = 0; gi < n_groups; ++gi) {
+            const int slot = gi % kPkSlots;
+            if (lane == 0) {
+                if (gi >= kPkSlots) ok = mbar_wait(&pk_empty[slot], ((gi / kPkSlots) & 1) ^ 1, abort_flag) && ok;
+                mbar_expect_tx(&pk_full[slot], (uint32_t)kPkSlotBytes);
+            }
+            __syncwarp();
+            unsigned char* dst = packed + slot * kPkSlotBytes + (lane == 0 ? 0 : kValsTile);
+            if (lane < 2) tma_tile(dst, lane == 0 ? &tmV : &tmM, gi * (lane == 0 ? 64 : 32), m0, &pk_full[slot]);
+        }
+        if (lane == 0) {
+            for (int it = p.n1; it < n_total; ++it) {
+                const int st = it % kPStages;
+                if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
+                mbar_expect_tx(&a2_full[st], (uint32_t)kATile);
+                tma_tile(stages + (size_t)st * kStageBytes + kBTile, &tmA2, (it - p.n1) * kPBK, m0, &a2_full[st]);
+            }
+        }
+    } else if (warp == kWarpMma) {
         // ============================ MMA issuer ============================
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16(kPM, N);
@@ -221,8 +259,16 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 const int st = it % kPStages;
                 const uint32_t parity = (it / kPStages) & 1;
                 const bool sparse = it < p.n1;
-                ok = mbar_wait(sparse ? &conv_done[st] : &tma_full[st], parity, abort_flag) && ok;
+                ok = mbar_wait(&b_full[st], parity, abort_flag) && ok;
+                if (sparse) {
+                    ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
+                } else {
+                    // a2_full[st] is armed by dense stages only: its phase counts those
+                    const int first = p.n1 + (st - p.n1 % kPStages + kPStages) % kPStages;
+                    ok = mbar_wait(&a2_full[st], (uint32_t)(((it - first) / kPStages) & 1), abort_flag) && ok;
+                }
                 fence_after_sync();
+                PSTAMP(3, it);
                 const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
                 const uint32_t a_addr = b_addr + kBTile;
                 if (sparse) {
@@ -238,6 +284,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                                   (it > 0 || j > 0) ? 1u : 0u);
                 }
                 mma_commit(&empty[st]);          // the stage is free once these MMAs have read it
+                PSTAMP(4, it);
             }
             mma_commit(acc_full);
         }
@@ -249,11 +296,15 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         for (int it = 0; it < p.n1; ++it) {
             const int st = it % kPStages;
-            unsigned char* sbase = stages + (size_t)st * kStageBytes;
-            ok = mbar_wait(&tma_full[st], (it / kPStages) & 1, abort_flag) && ok;
+            const int gi = it / kPkStages, q = it % kPkStages, slot = gi % kPkSlots;
+            const unsigned char* pk = packed + slot * kPkSlotBytes;
+            if (q == 0) ok = mbar_wait(&pk_full[slot], (gi / kPkSlots) & 1, abort_flag) && ok;
+            // the MMAs of the previous use of this stage must be done with its A tile and index words
+            if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
+            if (threadIdx.x == 0) PSTAMP(1, it);
             // ---- 8 value bytes -> 16 bf16: two 16-byte chunks of the row (64-byte rows, 64-byte swizzle)
-            const uint2 v = *reinterpret_cast<const uint2*>(sbase + kBTile + kATile + row * (kPBK / 4) + 8 * half);
-            unsigned char* arow = sbase + kBTile + row * 64;
+            const uint2 v = *reinterpret_cast<const uint2*>(pk + row * 64 + q * 16 + 8 * half);
+            unsigned char* arow = stages + (size_t)st * kStageBytes + kBTile + row * 64;
             const uint32_t w[2] = {v.x, v.y};
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
@@ -265,7 +316,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 *reinterpret_cast<uint4*>(arow + (((chunk ^ (row >> 1)) & 3) << 4)) = o;
             }
             // ---- index word of MMA `half` (layout in the file header)
-            const uint32_t mw = *reinterpret_cast<const uint32_t*>(sbase + kBTile + kATile + kValsTile + row * 16 + 8 * (it & 1) + 4 * half);
+            const uint32_t mw = *reinterpret_cast<const uint32_t*>(pk + kValsTile + row * 32 + q * 8 + 4 * half);
             const uint32_t send = x ? (mw & 0xFFFFu) : (mw >> 16);
             const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 8);
             const uint32_t e = x ? ((mw & 0xFFFF0000u) | recv) : ((mw & 0xFFFFu) | (recv << 16));
@@ -275,6 +326,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // A is read by the tensor core
             fence_before_sync();
             mbar_arrive(&conv_done[st]);
+            if (q == kPkStages - 1 || it == p.n1 - 1) mbar_arrive(&pk_empty[slot]);
+            if (threadIdx.x == 0) PSTAMP(2, it);
         }
         // ---- epilogue: thread = output row, TMEM columns = tokens; the two halves split the columns
         ok = mbar_wait(acc_full, 0, abort_flag) && ok;
@@ -308,7 +361,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     if (!ok && lane == 0) flag_error(p.status, SLIM_ERR_TIMEOUT);
     fence_before_sync();
     __syncthreads();
-    if (warp == kConvWarps + 1) {
+    if (warp == kWarpMma) {
         fence_after_sync();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(Cfg::kTmemCols) : "memory");
     }
@@ -390,8 +443,8 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     const int n_main = wide ? 256 : 64;
     const int n_pre = 64;                         // the T' product has few row tiles: narrow token tiles fill the machine
     CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;
-    bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPBK / 4, kPM, false) &&
-              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, 16, kPM, false) &&
+    bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPkStages * kPBK / 4, kPM, false) &&
+              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPkStages * kPBK / 8, kPM, false) &&
               pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, n_main, true);
     if (!ok) return SLIM_ERR_CUDA;
     if (r > 0) {
@@ -421,3 +474,9 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
 }
 
 }  // namespace slim
+
+#ifdef SLIM_PREFILL_TRACE
+extern "C" int slim_debug_read_ptrace(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, slim::g_ptrace, sizeof(slim::g_ptrace));
+}
+#endif
