@@ -28,8 +28,8 @@
 // The packed value and index bytes travel separately, 256 columns (4 stages) per TMA tile,
 // through a 2-slot ring of their own.  A thread is held ~160 ns by every TMA request it
 // starts, so requests are spread over three producer warps: token tiles of even stages,
-// token tiles of odd stages, packed tiles and A2 tiles.
-// mbarriers: b_full / a2_full / pk_full (TMA bytes landed), conv_done (converters
+// token tiles of odd stages (each with the A2 tile in phase 2), packed tiles.
+// mbarriers: b_full / pk_full (TMA bytes landed), conv_done (converters
 // finished a stage), empty / pk_empty (tcgen05.commit: the MMAs that read the stage are
 // complete; converters done with a packed slot), acc_full.
 // Every wait is bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on.
@@ -182,11 +182,10 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char* packed = stages + (size_t)kPStages * kStageBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(packed + kPkSlots * kPkSlotBytes);
-    uint64_t* b_full = bars;                         // [kPStages] token tile landed
-    uint64_t* a2_full = bars + kPStages;             // [kPStages] dense-phase A tile landed
-    uint64_t* conv_done = bars + 2 * kPStages;       // [kPStages]
-    uint64_t* empty = bars + 3 * kPStages;           // [kPStages]
-    uint64_t* pk_full = bars + 4 * kPStages;         // [kPkSlots]
+    uint64_t* b_full = bars;                         // [kPStages] token tile (and A2 tile) landed
+    uint64_t* conv_done = bars + kPStages;           // [kPStages]
+    uint64_t* empty = bars + 2 * kPStages;           // [kPStages]
+    uint64_t* pk_full = bars + 3 * kPStages;         // [kPkSlots]
     uint64_t* pk_empty = pk_full + kPkSlots;         // [kPkSlots]
     uint64_t* acc_full = pk_empty + kPkSlots;        // [1]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
@@ -198,7 +197,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kPStages; ++i) {
-            mbar_init(&b_full[i], 1); mbar_init(&a2_full[i], 1);
+            mbar_init(&b_full[i], 1);
             mbar_init(&conv_done[i], 32 * kConvWarps); mbar_init(&empty[i], 1);
         }
         for (int i = 0; i < kPkSlots; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], 32 * kConvWarps); }
@@ -218,19 +217,27 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
 
     if (warp == kWarpXEven || warp == kWarpXOdd) {
         // ============================ token-tile producers ============================
-        if (lane == 0) {
-            for (int it = warp == kWarpXEven ? 0 : 1; it < n_total; it += 2) {
-                const int st = it % kPStages;
-                const bool sparse = it < p.n1;
+        // Each of the two warps walks every second stage in order (a waiter that skipped uses of
+        // a barrier would mistake an old phase for the one it needs).  Sparse stage: lane 0
+        // requests the token tile.  Dense stage: lanes 0 and 1 request the token tile and the A2
+        // tile with one instruction.
+        for (int it = warp == kWarpXEven ? 0 : 1; it < n_total; it += 2) {
+            const int st = it % kPStages;
+            const bool sparse = it < p.n1;
+            if (lane == 0) {
                 if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
-                mbar_expect_tx(&b_full[st], (uint32_t)kBTile);
-                tma_tile(stages + (size_t)st * kStageBytes, sparse ? &tmX : &tmB2,
-                         sparse ? it * kPBK : (it - p.n1) * kPBK, n0, &b_full[st]);
-                PSTAMP(0, it);
+                mbar_expect_tx(&b_full[st], (uint32_t)(sparse ? kBTile : kBTile + kATile));
             }
+            __syncwarp();
+            unsigned char* sbase = stages + (size_t)st * kStageBytes;
+            const int k = sparse ? it * kPBK : (it - p.n1) * kPBK;
+            if (lane == 0 || (lane == 1 && !sparse))
+                tma_tile(lane == 0 ? sbase : sbase + kBTile, lane == 1 ? &tmA2 : (sparse ? &tmX : &tmB2), k,
+                         lane == 0 ? n0 : m0, &b_full[st]);
+            if (lane == 0) PSTAMP(0, it);
         }
     } else if (warp == kWarpPk) {
-        // ============================ packed-tile and A2 producer ============================
+        // ============================ packed-tile producer ============================
         // lanes 0 and 1 request the value-byte and the index-byte tile with one instruction
         const int n_groups = ceil_div(p.n1, kPkStages);
         for (int gi = 0; gi < n_groups; ++gi) {
@@ -243,14 +250,6 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             unsigned char* dst = packed + slot * kPkSlotBytes + (lane == 0 ? 0 : kValsTile);
             if (lane < 2) tma_tile(dst, lane == 0 ? &tmV : &tmM, gi * (lane == 0 ? 64 : 32), m0, &pk_full[slot]);
         }
-        if (lane == 0) {
-            for (int it = p.n1; it < n_total; ++it) {
-                const int st = it % kPStages;
-                if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
-                mbar_expect_tx(&a2_full[st], (uint32_t)kATile);
-                tma_tile(stages + (size_t)st * kStageBytes + kBTile, &tmA2, (it - p.n1) * kPBK, m0, &a2_full[st]);
-            }
-        }
     } else if (warp == kWarpMma) {
         // ============================ MMA issuer ============================
         if (lane == 0) {
@@ -260,13 +259,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 const uint32_t parity = (it / kPStages) & 1;
                 const bool sparse = it < p.n1;
                 ok = mbar_wait(&b_full[st], parity, abort_flag) && ok;
-                if (sparse) {
-                    ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
-                } else {
-                    // a2_full[st] is armed by dense stages only: its phase counts those
-                    const int first = p.n1 + (st - p.n1 % kPStages + kPStages) % kPStages;
-                    ok = mbar_wait(&a2_full[st], (uint32_t)(((it - first) / kPStages) & 1), abort_flag) && ok;
-                }
+                if (sparse) ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
                 fence_after_sync();
                 PSTAMP(3, it);
                 const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
