@@ -231,9 +231,12 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             __syncwarp();
             unsigned char* sbase = stages + (size_t)st * kStageBytes;
             const int k = sparse ? it * kPBK : (it - p.n1) * kPBK;
-            if (lane == 0 || (lane == 1 && !sparse))
-                tma_tile(lane == 0 ? sbase : sbase + kBTile, lane == 1 ? &tmA2 : (sparse ? &tmX : &tmB2), k,
-                         lane == 0 ? n0 : m0, &b_full[st]);
+            // the token tile travels as N / 64 boxes of 64 tokens (smaller boxes land sooner), one per lane
+            constexpr int kXBoxes = N / 64;
+            if (lane < kXBoxes || (lane == kXBoxes && !sparse))
+                tma_tile(lane < kXBoxes ? sbase + lane * (64 * 128) : sbase + kBTile,
+                         lane == kXBoxes ? &tmA2 : (sparse ? &tmX : &tmB2), k,
+                         lane < kXBoxes ? n0 + 64 * lane : m0, &b_full[st]);
             if (lane == 0) PSTAMP(0, it);
         }
     } else if (warp == kWarpPk) {
@@ -438,19 +441,19 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;
     bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPkStages * kPBK / 4, kPM, false) &&
               pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPkStages * kPBK / 8, kPM, false) &&
-              pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, n_main, true);
+              pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, 64, true);
     if (!ok) return SLIM_ERR_CUDA;
     if (r > 0) {
         // T' = (X R^T) / s : dense phase only, output rows = adapter index
         ok = pf_map(&tmA2, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 64, kPM, true) &&
-             pf_map(&tmXpre, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, n_pre, true);
+             pf_map(&tmXpre, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, 64, true);
         if (!ok) return SLIM_ERR_CUDA;
         PrefillParams q;
         q.out = Tq; q.ldo = r; q.m_total = r; q.b = b; q.n1 = 0; q.n2 = d_in / kPBK; q.scale = 1.f / s_eff; q.status = status_dev;
         slim_status_t rc = launch_tile_kernel<64>(q, r, tmV, tmM, tmXpre, tmA2, tmXpre, st);
         if (rc != SLIM_OK) return rc;
         ok = pf_map(&tmA2, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, 64, kPM, true) &&
-             pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, 64, n_main, true);
+             pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, 64, 64, true);
         if (!ok) return SLIM_ERR_CUDA;
     } else {
         tmA2 = tmX; tmB2 = tmX;       // never used when r == 0
