@@ -40,7 +40,6 @@ namespace slim {
 
 constexpr int kPM = 128;            // output rows per CTA (MMA M)
 constexpr int kPBK = 64;            // columns per stage, both phases
-constexpr int kPStages = 4;
 constexpr int kPkStages = 4;        // stages covered by one packed tile (256 weight columns)
 constexpr int kPkSlots = 2;
 constexpr int kConvWarps = 8;       // warps 0-7 converters / epilogue
@@ -52,12 +51,18 @@ constexpr int kMetaTile = kPM * (kPkStages * kPBK / 8);     // 4 KB: 32 index by
 constexpr int kPkSlotBytes = kValsTile + kMetaTile;
 constexpr uint32_t kPSpinLimit = 1u << 21;
 
-template <int N> struct PfCfg {
-    static constexpr int kBTile = N * 128;                                  // N tokens x 128 bytes
+// TWO = a pair of CTAs (cluster of 2 along the row tiles) shares one token tile: each CTA
+// loads half of it and one cta_group::2 MMA of shape 256 x N, issued by the even CTA,
+// drives both tensor cores.  Halves the token-tile traffic per CTA and leaves room for
+// more stages.
+template <int N, bool TWO> struct PfCfg {
+    static constexpr int kBRows = TWO ? N / 2 : N;                          // token rows this CTA loads
+    static constexpr int kBTile = kBRows * 128;
+    static constexpr int kStages = TWO ? 6 : 4;
     static constexpr int kStageBytes = kBTile + kATile;
     static constexpr int kECol = N;                                         // index words: N + 4 * stage + mma
     static constexpr int kTmemCols = N >= 256 ? 512 : (N >= 128 ? 256 : 128);
-    static constexpr size_t kSmem = 1024 + (size_t)kPStages * kStageBytes + kPkSlots * kPkSlotBytes + 512;
+    static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + kPkSlots * kPkSlotBytes + 512;
 };
 
 struct PrefillParams {
@@ -150,6 +155,58 @@ __device__ __forceinline__ void mma_sparse(uint32_t d_tmem, uint64_t a_desc, uin
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(s32(bar)) : "memory");
 }
+// ---- CTA-pair variants
+__device__ __forceinline__ void mma_dense2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_sparse2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t e_tmem,
+                                            uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+        :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Address of the same shared-memory object in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t peer_addr(const void* p, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(s32(p)), "r"(rank));
+    return r;
+}
+// Completion of this thread's earlier MMAs arrives on a barrier given by cluster address.
+__device__ __forceinline__ void mma_commit2(uint32_t cluster_bar_addr) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(cluster_bar_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" :: "r"(cluster_bar_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    const uint32_t addr = s32(bar);
+    for (uint32_t it = 0; it < kPSpinLimit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1u;
+    return false;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
 __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -168,15 +225,15 @@ __device__ __forceinline__ uint32_t nib2bf16(uint32_t w, uint32_t w_shr4) {
 
 }  // namespace pf
 
-template <int N>
+template <int N, bool TWO>
 __global__ void __launch_bounds__(kPThreads, 1)
 prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmX,
                const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2)
 {
     using namespace pf;
-    using Cfg = PfCfg<N>;
-    constexpr int kBTile = Cfg::kBTile, kStageBytes = Cfg::kStageBytes, kECol = Cfg::kECol;
+    using Cfg = PfCfg<N, TWO>;
+    constexpr int kBTile = Cfg::kBTile, kStageBytes = Cfg::kStageBytes, kECol = Cfg::kECol, kPStages = Cfg::kStages;
     extern __shared__ unsigned char smem_raw[];
     // layout: stages {B | A} | packed slots {value bytes | index bytes} | barriers
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -188,26 +245,35 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     uint64_t* pk_full = bars + 3 * kPStages;         // [kPkSlots]
     uint64_t* pk_empty = pk_full + kPkSlots;         // [kPkSlots]
     uint64_t* acc_full = pk_empty + kPkSlots;        // [1]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+    uint64_t* peer_ready = acc_full + 1;             // [kPStages] pair only: the odd CTA's stage is ready
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(peer_ready + kPStages);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = TWO ? cluster_rank() : 0u;           // 0 = the CTA that issues the pair's MMAs
     const int m0 = blockIdx.x * kPM, n0 = blockIdx.y * N;
+    const int nb0 = n0 + (int)rank * Cfg::kBRows;                // first token row this CTA loads
     const int n_total = p.n1 + p.n2;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kPStages; ++i) {
             mbar_init(&b_full[i], 1);
-            mbar_init(&conv_done[i], 32 * kConvWarps); mbar_init(&empty[i], 1);
+            mbar_init(&conv_done[i], 32 * kConvWarps); mbar_init(&empty[i], 1); mbar_init(&peer_ready[i], 1);
         }
         for (int i = 0; i < kPkSlots; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], 32 * kConvWarps); }
         mbar_init(acc_full, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (TWO) cluster_sync_all();                    // both CTAs' barriers exist before anything crosses
     if (warp == kWarpMma) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s32(tmem_slot)), "r"(Cfg::kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (TWO) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s32(tmem_slot)), "r"(Cfg::kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(s32(tmem_slot)), "r"(Cfg::kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     fence_before_sync();
     __syncthreads();
@@ -232,11 +298,11 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             unsigned char* sbase = stages + (size_t)st * kStageBytes;
             const int k = sparse ? it * kPBK : (it - p.n1) * kPBK;
             // the token tile travels as N / 64 boxes of 64 tokens (smaller boxes land sooner), one per lane
-            constexpr int kXBoxes = N / 64;
+            constexpr int kXBoxes = Cfg::kBRows / 64;
             if (lane < kXBoxes || (lane == kXBoxes && !sparse))
                 tma_tile(lane < kXBoxes ? sbase + lane * (64 * 128) : sbase + kBTile,
                          lane == kXBoxes ? &tmA2 : (sparse ? &tmX : &tmB2), k,
-                         lane < kXBoxes ? n0 + 64 * lane : m0, &b_full[st]);
+                         lane < kXBoxes ? nb0 + 64 * lane : m0, &b_full[st]);
             if (lane == 0) PSTAMP(0, it);
         }
     } else if (warp == kWarpPk) {
@@ -255,14 +321,25 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
         }
     } else if (warp == kWarpMma) {
         // ============================ MMA issuer ============================
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16(kPM, N);
+        if (lane == 0 && TWO && rank != 0) {
+            // odd CTA of a pair: tell the even CTA when this CTA's half of a stage is ready
+            for (int it = 0; it < n_total; ++it) {
+                const int st = it % kPStages;
+                const uint32_t parity = (it / kPStages) & 1;
+                ok = mbar_wait(&b_full[st], parity, abort_flag) && ok;
+                if (it < p.n1) ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
+                fence_before_sync();
+                mbar_arrive_cluster(peer_addr(&peer_ready[st], 0));
+            }
+        } else if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16(TWO ? 2 * kPM : kPM, N);
             for (int it = 0; it < n_total; ++it) {
                 const int st = it % kPStages;
                 const uint32_t parity = (it / kPStages) & 1;
                 const bool sparse = it < p.n1;
                 ok = mbar_wait(&b_full[st], parity, abort_flag) && ok;
                 if (sparse) ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
+                if (TWO) ok = mbar_wait_cluster(&peer_ready[st], parity, abort_flag) && ok;
                 fence_after_sync();
                 PSTAMP(3, it);
                 const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
@@ -270,19 +347,28 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 if (sparse) {
                     // per MMA: A 16 stored bf16 (32 bytes of a 64-byte row), B 32 columns (64 bytes)
 #pragma unroll
-                    for (int j = 0; j < 2; ++j)
-                        mma_sparse(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
-                                   tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, (it > 0 || j > 0) ? 1u : 0u);
+                    for (int j = 0; j < 2; ++j) {
+                        const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
+                        if (TWO) mma_sparse2(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
+                                             tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
+                        else     mma_sparse(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
+                                            tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
+                    }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc,
-                                  (it > 0 || j > 0) ? 1u : 0u);
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
+                        if (TWO) mma_dense2(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
+                        else     mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
+                    }
                 }
-                mma_commit(&empty[st]);          // the stage is free once these MMAs have read it
+                // the stage is free (in both CTAs of a pair) once these MMAs have read it
+                if (TWO) { mma_commit2(peer_addr(&empty[st], 0)); mma_commit2(peer_addr(&empty[st], 1)); }
+                else mma_commit(&empty[st]);
                 PSTAMP(4, it);
             }
-            mma_commit(acc_full);
+            if (TWO) { mma_commit2(peer_addr(acc_full, 0)); mma_commit2(peer_addr(acc_full, 1)); }
+            else mma_commit(acc_full);
         }
     } else {
         // ============================ converters, then epilogue ============================
@@ -357,9 +443,11 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     if (!ok && lane == 0) flag_error(p.status, SLIM_ERR_TIMEOUT);
     fence_before_sync();
     __syncthreads();
+    if (TWO) cluster_sync_all();                    // neither CTA leaves while the other may still read its shared memory
     if (warp == kWarpMma) {
         fence_after_sync();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(Cfg::kTmemCols) : "memory");
+        if (TWO) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(Cfg::kTmemCols) : "memory");
+        else     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(Cfg::kTmemCols) : "memory");
     }
 }
 
@@ -405,14 +493,22 @@ size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r) {
 
 static bool g_prefill_attr_set[64];
 
-template <int N>
+template <int N, bool TWO>
 static slim_status_t launch_tile_kernel(const PrefillParams& q, int m_rows, const CUtensorMap& tmV, const CUtensorMap& tmM,
                                         const CUtensorMap& tmX, const CUtensorMap& tmA2, const CUtensorMap& tmB2,
                                         cudaStream_t st) {
-    const dim3 grid(ceil_div(m_rows, kPM), ceil_div(q.b, N)), block(kPThreads);
-    prefill_kernel<N><<<grid, block, PfCfg<N>::kSmem, st>>>(q, tmV, tmM, tmX, tmA2, tmB2);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ceil_div(m_rows, kPM), ceil_div(q.b, N));
+    cfg.blockDim = dim3(kPThreads);
+    cfg.dynamicSmemBytes = PfCfg<N, TWO>::kSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = TWO ? 2 : 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_kernel<N, TWO>, q, tmV, tmM, tmX, tmA2, tmB2);
     count_launch(1);
-    return cudaGetLastError() == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+    return e == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
 }
 
 slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
@@ -427,8 +523,9 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !g_prefill_attr_set[dev]) {
-        if (cudaFuncSetAttribute(prefill_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256>::kSmem) != cudaSuccess ||
-            cudaFuncSetAttribute(prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<64>::kSmem) != cudaSuccess)
+        if (cudaFuncSetAttribute(prefill_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256, true>::kSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256, false>::kSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<64, false>::kSmem) != cudaSuccess)
             return SLIM_ERR_CUDA;
         g_prefill_attr_set[dev] = true;
     }
@@ -450,7 +547,7 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
         if (!ok) return SLIM_ERR_CUDA;
         PrefillParams q;
         q.out = Tq; q.ldo = r; q.m_total = r; q.b = b; q.n1 = 0; q.n2 = d_in / kPBK; q.scale = 1.f / s_eff; q.status = status_dev;
-        slim_status_t rc = launch_tile_kernel<64>(q, r, tmV, tmM, tmXpre, tmA2, tmXpre, st);
+        slim_status_t rc = launch_tile_kernel<64, false>(q, r, tmV, tmM, tmXpre, tmA2, tmXpre, st);
         if (rc != SLIM_OK) return rc;
         ok = pf_map(&tmA2, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, 64, kPM, true) &&
              pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, 64, 64, true);
@@ -465,8 +562,10 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     p.scale = s_eff; p.status = status_dev;
     if (p.n1 + p.n2 == 0)             // s == 0 and no adapters: the result is zero
         return cudaMemsetAsync(Y, 0, (size_t)b * d_out * 2, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
-    return wide ? launch_tile_kernel<256>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st)
-                : launch_tile_kernel<64>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
+    if (!wide) return launch_tile_kernel<64, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
+    // pairs of CTAs need an even number of row tiles
+    return (d_out / kPM) % 2 == 0 ? launch_tile_kernel<256, true>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st)
+                                  : launch_tile_kernel<256, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
 }
 
 }  // namespace slim
