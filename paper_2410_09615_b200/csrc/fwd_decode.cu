@@ -346,18 +346,20 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
         // ---- the CTA's slice of the activations: 4 tiles of 64 columns per block, rows >= b read as zero
         if (sh.grp >= 0) {
             if (lane == 0) mbar_arrive_expect_tx(x_bar, (uint32_t)(sh.nb * 4 * x_sub));
-            __syncwarp();
             if (lane < sh.nb * 4) tma_tile(xs + lane * x_sub, &tmX, sh.blk_begin * 256 + 64 * lane, 0, x_bar);
         }
-        // Returns the slot (all lanes) once it is free and its full barrier is armed.
+        // Returns the slot once it is free; lane 0 arms its full barrier.  The whole warp waits:
+        // a single waiting lane followed by a warp barrier costs some hundred nanoseconds per
+        // tile.  (A tile may land before lane 0 has armed the barrier; the phase cannot
+        // complete before that arrival.)
+        int slot_i = 0;
+        uint32_t phase = 0;
         auto acquire = [&](uint32_t bytes) -> int {
-            const int slot = it % n_slots;
-            if (lane == 0) {
-                if (it >= (uint32_t)n_slots) ok = mbar_wait(&empty_bar[slot], ((it / n_slots) & 1) ^ 1) && ok;
-                mbar_arrive_expect_tx(&full_bar[slot], bytes);
-            }
-            __syncwarp();
+            const int slot = slot_i;
+            if (it >= (uint32_t)n_slots) ok = mbar_wait(&empty_bar[slot], phase ^ 1) && ok;
+            if (lane == 0) mbar_arrive_expect_tx(&full_bar[slot], bytes);
             ++it;
+            if (++slot_i == n_slots) { slot_i = 0; phase ^= 1; }
             return slot;
         };
         // ---- R chunks: 16 rows x (256 or 512) columns of bf16 = 4 or 8 tiles of 64 columns

@@ -41,7 +41,6 @@ namespace slim {
 constexpr int kPM = 128;            // output rows per CTA (MMA M)
 constexpr int kPBK = 64;            // columns per stage, both phases
 constexpr int kPkStages = 4;        // stages covered by one packed tile (256 weight columns)
-constexpr int kPkSlots = 2;
 constexpr int kConvWarps = 8;       // warps 0-7 converters / epilogue
 constexpr int kWarpXEven = 8, kWarpMma = 9, kWarpXOdd = 10, kWarpPk = 11;
 constexpr int kPThreads = 32 * 12;
@@ -58,11 +57,13 @@ constexpr uint32_t kPSpinLimit = 1u << 21;
 template <int N, bool TWO> struct PfCfg {
     static constexpr int kBRows = TWO ? N / 2 : N;                          // token rows this CTA loads
     static constexpr int kBTile = kBRows * 128;
-    static constexpr int kStages = TWO ? 6 : 4;
+    static constexpr int kStages = TWO ? 5 : 4;
+    // Packed tiles come from HBM (latency of a microsecond or two): the ring holds what fits.
+    static constexpr int kPkSlots = TWO ? 4 : (N >= 256 ? 2 : 8);
     static constexpr int kStageBytes = kBTile + kATile;
     static constexpr int kECol = N;                                         // index words: N + 4 * stage + mma
     static constexpr int kTmemCols = N >= 256 ? 512 : (N >= 128 ? 256 : 128);
-    static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + kPkSlots * kPkSlotBytes + 512;
+    static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + kPkSlots * kPkSlotBytes + 1024;
 };
 
 struct PrefillParams {
@@ -207,6 +208,11 @@ __device__ __forceinline__ uint32_t cluster_rank() {
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -234,6 +240,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     using namespace pf;
     using Cfg = PfCfg<N, TWO>;
     constexpr int kBTile = Cfg::kBTile, kStageBytes = Cfg::kStageBytes, kECol = Cfg::kECol, kPStages = Cfg::kStages;
+    constexpr int kPkSlots = Cfg::kPkSlots;
     extern __shared__ unsigned char smem_raw[];
     // layout: stages {B | A} | packed slots {value bytes | index bytes} | barriers
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -254,13 +261,19 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     const int m0 = blockIdx.x * kPM, n0 = blockIdx.y * N;
     const int nb0 = n0 + (int)rank * Cfg::kBRows;                // first token row this CTA loads
     const int n_total = p.n1 + p.n2;
+    // CTAs that share token rows start their walk over the weight columns at different places,
+    // so that at any moment they ask the L2 for different lines of X rather than all for the same
+    // ones.  The walk is rotated by whole 256-column groups (a pair of CTAs rotates together).
+    const int n_groups = ceil_div(p.n1, kPkStages);
+    const int rot_g = (p.n1 % kPkStages == 0 && n_groups > 0)
+                          ? (int)(((blockIdx.x >> (TWO ? 1 : 0)) + 3u * blockIdx.y) % (unsigned)n_groups) : 0;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kPStages; ++i) {
             mbar_init(&b_full[i], 1);
-            mbar_init(&conv_done[i], 32 * kConvWarps); mbar_init(&empty[i], 1); mbar_init(&peer_ready[i], 1);
+            mbar_init(&conv_done[i], kConvWarps); mbar_init(&empty[i], 1); mbar_init(&peer_ready[i], 1);
         }
-        for (int i = 0; i < kPkSlots; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], 32 * kConvWarps); }
+        for (int i = 0; i < kPkSlots; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], kConvWarps); }
         mbar_init(acc_full, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -290,38 +303,36 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
         for (int it = warp == kWarpXEven ? 0 : 1; it < n_total; it += 2) {
             const int st = it % kPStages;
             const bool sparse = it < p.n1;
-            if (lane == 0) {
-                if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
-                mbar_expect_tx(&b_full[st], (uint32_t)(sparse ? kBTile : kBTile + kATile));
-            }
-            __syncwarp();
+            // The whole warp waits (no lane is left behind at a warp barrier while another
+            // spins: that costs some hundred nanoseconds per stage); lane 0 arms the barrier.
+            if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
+            if (lane == 0) mbar_expect_tx(&b_full[st], (uint32_t)(sparse ? kBTile : kBTile + kATile));
             unsigned char* sbase = stages + (size_t)st * kStageBytes;
-            const int k = sparse ? it * kPBK : (it - p.n1) * kPBK;
-            // the token tile travels as N / 64 boxes of 64 tokens (smaller boxes land sooner), one per lane
-            constexpr int kXBoxes = Cfg::kBRows / 64;
-            if (lane < kXBoxes || (lane == kXBoxes && !sparse))
-                tma_tile(lane < kXBoxes ? sbase + lane * (64 * 128) : sbase + kBTile,
-                         lane == kXBoxes ? &tmA2 : (sparse ? &tmX : &tmB2), k,
-                         lane < kXBoxes ? nb0 + 64 * lane : m0, &b_full[st]);
+            int kb = sparse ? it + rot_g * kPkStages : it - p.n1;
+            if (sparse && kb >= p.n1) kb -= p.n1;
+            const int k = kb * kPBK;
+            // lane 0: the token tile (one box); lane 1, dense stages only: the A2 tile
+            if (lane == 0 || (lane == 1 && !sparse))
+                tma_tile(lane == 0 ? sbase : sbase + kBTile, lane == 1 ? &tmA2 : (sparse ? &tmX : &tmB2), k,
+                         lane == 0 ? nb0 : m0, &b_full[st]);
             if (lane == 0) PSTAMP(0, it);
         }
     } else if (warp == kWarpPk) {
         // ============================ packed-tile producer ============================
         // lanes 0 and 1 request the value-byte and the index-byte tile with one instruction
-        const int n_groups = ceil_div(p.n1, kPkStages);
         for (int gi = 0; gi < n_groups; ++gi) {
             const int slot = gi % kPkSlots;
-            if (lane == 0) {
-                if (gi >= kPkSlots) ok = mbar_wait(&pk_empty[slot], ((gi / kPkSlots) & 1) ^ 1, abort_flag) && ok;
-                mbar_expect_tx(&pk_full[slot], (uint32_t)kPkSlotBytes);
-            }
-            __syncwarp();
+            const int g = gi + rot_g < n_groups ? gi + rot_g : gi + rot_g - n_groups;
+            if (gi >= kPkSlots) ok = mbar_wait(&pk_empty[slot], ((gi / kPkSlots) & 1) ^ 1, abort_flag) && ok;
+            if (lane == 0) mbar_expect_tx(&pk_full[slot], (uint32_t)kPkSlotBytes);
             unsigned char* dst = packed + slot * kPkSlotBytes + (lane == 0 ? 0 : kValsTile);
-            if (lane < 2) tma_tile(dst, lane == 0 ? &tmV : &tmM, gi * (lane == 0 ? 64 : 32), m0, &pk_full[slot]);
+            if (lane < 2) tma_tile(dst, lane == 0 ? &tmV : &tmM, g * (lane == 0 ? 64 : 32), m0, &pk_full[slot]);
         }
     } else if (warp == kWarpMma) {
         // ============================ MMA issuer ============================
-        if (lane == 0 && TWO && rank != 0) {
+        // The whole warp walks the stages and waits together; one elected lane issues.  (A loop
+        // run by a single lane of a diverged warp issues the tensor-core instructions far slower.)
+        if (TWO && rank != 0) {
             // odd CTA of a pair: tell the even CTA when this CTA's half of a stage is ready
             for (int it = 0; it < n_total; ++it) {
                 const int st = it % kPStages;
@@ -329,9 +340,13 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 ok = mbar_wait(&b_full[st], parity, abort_flag) && ok;
                 if (it < p.n1) ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
                 fence_before_sync();
-                mbar_arrive_cluster(peer_addr(&peer_ready[st], 0));
+                if (elect_one()) {
+                    mbar_arrive_cluster(peer_addr(&peer_ready[st], 0));
+                    PSTAMP(5, it);
+                }
+                __syncwarp();
             }
-        } else if (lane == 0) {
+        } else {
             constexpr uint32_t idesc = idesc_bf16(TWO ? 2 * kPM : kPM, N);
             for (int it = 0; it < n_total; ++it) {
                 const int st = it % kPStages;
@@ -341,34 +356,40 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 if (sparse) ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
                 if (TWO) ok = mbar_wait_cluster(&peer_ready[st], parity, abort_flag) && ok;
                 fence_after_sync();
-                PSTAMP(3, it);
                 const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
                 const uint32_t a_addr = b_addr + kBTile;
-                if (sparse) {
-                    // per MMA: A 16 stored bf16 (32 bytes of a 64-byte row), B 32 columns (64 bytes)
+                if (elect_one()) {
+                    PSTAMP(3, it);
+                    if (sparse) {
+                        // per MMA: A 16 stored bf16 (32 bytes of a 64-byte row), B 32 columns (64 bytes)
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
-                        if (TWO) mma_sparse2(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
-                                             tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
-                        else     mma_sparse(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
-                                            tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
-                    }
-                } else {
+                        for (int j = 0; j < 2; ++j) {
+                            const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
+                            if (TWO) mma_sparse2(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
+                                                 tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
+                            else     mma_sparse(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
+                                                tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
+                        }
+                    } else {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
-                        if (TWO) mma_dense2(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
-                        else     mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
+                            if (TWO) mma_dense2(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
+                            else     mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
+                        }
                     }
+                    // the stage is free (in both CTAs of a pair) once these MMAs have read it
+                    if (TWO) { mma_commit2(peer_addr(&empty[st], 0)); mma_commit2(peer_addr(&empty[st], 1)); }
+                    else mma_commit(&empty[st]);
+                    PSTAMP(4, it);
                 }
-                // the stage is free (in both CTAs of a pair) once these MMAs have read it
-                if (TWO) { mma_commit2(peer_addr(&empty[st], 0)); mma_commit2(peer_addr(&empty[st], 1)); }
-                else mma_commit(&empty[st]);
-                PSTAMP(4, it);
+                __syncwarp();
             }
-            if (TWO) { mma_commit2(peer_addr(acc_full, 0)); mma_commit2(peer_addr(acc_full, 1)); }
-            else mma_commit(acc_full);
+            if (elect_one()) {
+                if (TWO) { mma_commit2(peer_addr(acc_full, 0)); mma_commit2(peer_addr(acc_full, 1)); }
+                else mma_commit(acc_full);
+            }
+            __syncwarp();
         }
     } else {
         // ============================ converters, then epilogue ============================
@@ -407,8 +428,12 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // A is read by the tensor core
             fence_before_sync();
-            mbar_arrive(&conv_done[st]);
-            if (q == kPkStages - 1 || it == p.n1 - 1) mbar_arrive(&pk_empty[slot]);
+            // one arrival per warp: arrivals on one barrier are served one after another
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&conv_done[st]);
+                if (q == kPkStages - 1 || it == p.n1 - 1) mbar_arrive(&pk_empty[slot]);
+            }
             if (threadIdx.x == 0) PSTAMP(2, it);
         }
         // ---- epilogue: thread = output row, TMEM columns = tokens; the two halves split the columns
@@ -533,12 +558,13 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     const float s_eff = s != 0.f ? s : 1.f;       // with s == 0 only the adapter term remains
     // token tile: 256 when that still gives every SM a tile, else 64
     const bool wide = (long long)(d_out / kPM) * ceil_div(b, 256) >= di->sm_count;
-    const int n_main = wide ? 256 : 64;
     const int n_pre = 64;                         // the T' product has few row tiles: narrow token tiles fill the machine
+    const bool pair = false && wide && (d_out / kPM) % 2 == 0;     // pairs of CTAs need an even number of row tiles
+    const int xbox = wide ? (pair ? 128 : 256) : 64;      // token rows one CTA loads per stage = one TMA box
     CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;
     bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPkStages * kPBK / 4, kPM, false) &&
               pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPkStages * kPBK / 8, kPM, false) &&
-              pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, 64, true);
+              pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, xbox, true);
     if (!ok) return SLIM_ERR_CUDA;
     if (r > 0) {
         // T' = (X R^T) / s : dense phase only, output rows = adapter index
@@ -550,7 +576,7 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
         slim_status_t rc = launch_tile_kernel<64, false>(q, r, tmV, tmM, tmXpre, tmA2, tmXpre, st);
         if (rc != SLIM_OK) return rc;
         ok = pf_map(&tmA2, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, 64, kPM, true) &&
-             pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, 64, 64, true);
+             pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, 64, xbox, true);
         if (!ok) return SLIM_ERR_CUDA;
     } else {
         tmA2 = tmX; tmB2 = tmX;       // never used when r == 0
@@ -563,8 +589,7 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     if (p.n1 + p.n2 == 0)             // s == 0 and no adapters: the result is zero
         return cudaMemsetAsync(Y, 0, (size_t)b * d_out * 2, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
     if (!wide) return launch_tile_kernel<64, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
-    // pairs of CTAs need an even number of row tiles
-    return (d_out / kPM) % 2 == 0 ? launch_tile_kernel<256, true>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st)
+    return pair ? launch_tile_kernel<256, true>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st)
                                   : launch_tile_kernel<256, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
 }
 
