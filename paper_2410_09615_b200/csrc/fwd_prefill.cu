@@ -57,10 +57,14 @@ constexpr uint32_t kPSpinLimit = 1u << 21;
 template <int N, bool TWO> struct PfCfg {
     static constexpr int kBRows = TWO ? N / 2 : N;                          // token rows this CTA loads
     static constexpr int kBTile = kBRows * 128;
-    static constexpr int kStages = TWO ? 5 : 4;
+    // A region of a stage: the expanded weight tile needs 8 KB; the pair kernel's dense stages are
+    // 32 columns wide so that their A2 tile fits there too and more stages fit in shared memory.
+    static constexpr int kARegion = TWO ? kATile / 2 : kATile;
+    static constexpr int kDK = TWO ? 32 : 64;                               // columns of a dense stage
+    static constexpr int kStages = TWO ? 7 : 4;
     // Packed tiles come from HBM (latency of a microsecond or two): the ring holds what fits.
     static constexpr int kPkSlots = TWO ? 4 : (N >= 256 ? 2 : 8);
-    static constexpr int kStageBytes = kBTile + kATile;
+    static constexpr int kStageBytes = kBTile + kARegion;
     static constexpr int kECol = N;                                         // index words: N + 4 * stage + mma
     static constexpr int kTmemCols = N >= 256 ? 512 : (N >= 128 ? 256 : 128);
     static constexpr size_t kSmem = 1024 + (size_t)kStages * kStageBytes + kPkSlots * kPkSlotBytes + 1024;
@@ -182,6 +186,10 @@ __device__ __forceinline__ uint32_t peer_addr(const void* p, uint32_t rank) {
 __device__ __forceinline__ void mma_commit2(uint32_t cluster_bar_addr) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(cluster_bar_addr) : "memory");
 }
+// Arrival on a barrier of another CTA of the cluster, ordered like a CTA-local arrival.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" :: "r"(cluster_bar_addr) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" :: "r"(cluster_bar_addr) : "memory");
 }
@@ -240,7 +248,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     using namespace pf;
     using Cfg = PfCfg<N, TWO>;
     constexpr int kBTile = Cfg::kBTile, kStageBytes = Cfg::kStageBytes, kECol = Cfg::kECol, kPStages = Cfg::kStages;
-    constexpr int kPkSlots = Cfg::kPkSlots;
+    constexpr int kPkSlots = Cfg::kPkSlots, kDK = Cfg::kDK;
     extern __shared__ unsigned char smem_raw[];
     // layout: stages {B | A} | packed slots {value bytes | index bytes} | barriers
     unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -271,7 +279,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     if (threadIdx.x == 0) {
         for (int i = 0; i < kPStages; ++i) {
             mbar_init(&b_full[i], 1);
-            mbar_init(&conv_done[i], kConvWarps); mbar_init(&empty[i], 1); mbar_init(&peer_ready[i], 1);
+            mbar_init(&conv_done[i], TWO ? kConvWarps : kConvWarps / 2); mbar_init(&empty[i], 1); mbar_init(&peer_ready[i], 1);
         }
         for (int i = 0; i < kPkSlots; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], kConvWarps); }
         mbar_init(acc_full, 1);
@@ -306,11 +314,12 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             // The whole warp waits (no lane is left behind at a warp barrier while another
             // spins: that costs some hundred nanoseconds per stage); lane 0 arms the barrier.
             if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
-            if (lane == 0) mbar_expect_tx(&b_full[st], (uint32_t)(sparse ? kBTile : kBTile + kATile));
+            // dense stage: kDK columns of the token rows and of the A2 rows
+            if (lane == 0) mbar_expect_tx(&b_full[st], (uint32_t)(sparse ? kBTile : (Cfg::kBRows + kPM) * kDK * 2));
             unsigned char* sbase = stages + (size_t)st * kStageBytes;
             int kb = sparse ? it + rot_g * kPkStages : it - p.n1;
             if (sparse && kb >= p.n1) kb -= p.n1;
-            const int k = kb * kPBK;
+            const int k = sparse ? kb * kPBK : kb * kDK;
             // lane 0: the token tile (one box); lane 1, dense stages only: the A2 tile
             if (lane == 0 || (lane == 1 && !sparse))
                 tma_tile(lane == 0 ? sbase : sbase + kBTile, lane == 1 ? &tmA2 : (sparse ? &tmX : &tmB2), k,
@@ -330,21 +339,20 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
         }
     } else if (warp == kWarpMma) {
         // ============================ MMA issuer ============================
-        // The whole warp walks the stages and waits together; one elected lane issues.  (A loop
-        // run by a single lane of a diverged warp issues the tensor-core instructions far slower.)
+        // The whole warp walks the stages and waits together; one elected lane issues (a loop run
+        // by a single lane of a diverged warp issues the tensor-core instructions more slowly).
         if (TWO && rank != 0) {
-            // odd CTA of a pair: tell the even CTA when this CTA's half of a stage is ready
-            for (int it = 0; it < n_total; ++it) {
-                const int st = it % kPStages;
-                const uint32_t parity = (it / kPStages) & 1;
-                ok = mbar_wait(&b_full[st], parity, abort_flag) && ok;
-                if (it < p.n1) ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
-                fence_before_sync();
-                if (elect_one()) {
-                    mbar_arrive_cluster(peer_addr(&peer_ready[st], 0));
+            // Odd CTA of a pair: tell the even CTA when this CTA's token rows (and A2 rows) of a
+            // stage have landed.  The data stay in this CTA's shared memory and are read by this
+            // SM's tensor core, so an arrival ordered after the landing within this CTA is enough;
+            // a cluster-scope release costs some 300 cycles per stage.
+            if (lane == 0) {
+                for (int it = 0; it < n_total; ++it) {
+                    const int st = it % kPStages;
+                    ok = mbar_wait(&b_full[st], (it / kPStages) & 1, abort_flag) && ok;
+                    mbar_arrive_remote(peer_addr(&peer_ready[st], 0));
                     PSTAMP(5, it);
                 }
-                __syncwarp();
             }
         } else {
             constexpr uint32_t idesc = idesc_bf16(TWO ? 2 * kPM : kPM, N);
@@ -353,88 +361,100 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 const uint32_t parity = (it / kPStages) & 1;
                 const bool sparse = it < p.n1;
                 ok = mbar_wait(&b_full[st], parity, abort_flag) && ok;
-                if (sparse) ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
-                if (TWO) ok = mbar_wait_cluster(&peer_ready[st], parity, abort_flag) && ok;
+                if (TWO) {          // arrivals from the other CTA: its converters, its loads
+                    if (sparse) ok = mbar_wait_cluster(&conv_done[st], parity, abort_flag) && ok;
+                    ok = mbar_wait_cluster(&peer_ready[st], parity, abort_flag) && ok;
+                } else if (sparse) {
+                    ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
+                }
                 fence_after_sync();
                 const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
                 const uint32_t a_addr = b_addr + kBTile;
-                if (elect_one()) {
-                    PSTAMP(3, it);
-                    if (sparse) {
-                        // per MMA: A 16 stored bf16 (32 bytes of a 64-byte row), B 32 columns (64 bytes)
+                if (!elect_one()) continue;
+                PSTAMP(3, it);
+                if (sparse) {
+                    // per MMA: A 16 stored bf16 (32 bytes of a 64-byte row), B 32 columns (64 bytes)
 #pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
-                            if (TWO) mma_sparse2(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
-                                                 tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
-                            else     mma_sparse(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
-                                                tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
-                            if (TWO) mma_dense2(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
-                            else     mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
-                        }
+                    for (int j = 0; j < 2; ++j) {
+                        const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
+                        if (TWO) mma_sparse2(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
+                                             tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
+                        else     mma_sparse(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc(b_addr + 64 * j),
+                                            tmem_base + kECol + 4 * st, idesc | (1u << 2) | (uint32_t)j, acc);
                     }
-                    // the stage is free (in both CTAs of a pair) once these MMAs have read it
-                    if (TWO) { mma_commit2(peer_addr(&empty[st], 0)); mma_commit2(peer_addr(&empty[st], 1)); }
-                    else mma_commit(&empty[st]);
-                    PSTAMP(4, it);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kDK / 16; ++j) {
+                        const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
+                        // pair kernel: 32-column stages, 64-byte rows with the 64-byte swizzle
+                        if (TWO) mma_dense2(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc64(b_addr + 32 * j), idesc, acc);
+                        else     mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
+                    }
                 }
-                __syncwarp();
+                // the stage is free (in both CTAs of a pair) once these MMAs have read it
+                if (TWO) { mma_commit2(peer_addr(&empty[st], 0)); mma_commit2(peer_addr(&empty[st], 1)); }
+                else mma_commit(&empty[st]);
+                PSTAMP(4, it);
             }
             if (elect_one()) {
                 if (TWO) { mma_commit2(peer_addr(acc_full, 0)); mma_commit2(peer_addr(acc_full, 1)); }
                 else mma_commit(acc_full);
             }
-            __syncwarp();
         }
     } else {
         // ============================ converters, then epilogue ============================
+        // Two groups of four warps take every second stage each, so that the latency chain of one
+        // stage (load, expand, store, index words into TMEM, fences, arrival) overlaps the next
+        // stage's.  Within a group a thread owns one weight row of the tile.
         const int row = threadIdx.x & 127;           // weight row inside the tile = TMEM lane
-        const int half = threadIdx.x >> 7;           // which 32 of the stage's 64 columns this thread expands
+        const int half = threadIdx.x >> 7;           // converter group; in the epilogue, which half of the columns
         const int x = (row >> 3) & 1;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        for (int it = 0; it < p.n1; ++it) {
+        for (int it = half; it < p.n1; it += 2) {
             const int st = it % kPStages;
             const int gi = it / kPkStages, q = it % kPkStages, slot = gi % kPkSlots;
             const unsigned char* pk = packed + slot * kPkSlotBytes;
-            if (q == 0) ok = mbar_wait(&pk_full[slot], (gi / kPkSlots) & 1, abort_flag) && ok;
+            ok = mbar_wait(&pk_full[slot], (gi / kPkSlots) & 1, abort_flag) && ok;
             // the MMAs of the previous use of this stage must be done with its A tile and index words
             if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
-            if (threadIdx.x == 0) PSTAMP(1, it);
-            // ---- 8 value bytes -> 16 bf16: two 16-byte chunks of the row (64-byte rows, 64-byte swizzle)
-            const uint2 v = *reinterpret_cast<const uint2*>(pk + row * 64 + q * 16 + 8 * half);
+            if ((threadIdx.x & 127) == 0) PSTAMP(1, it);
+            // ---- 16 value bytes -> 32 bf16: the row's four 16-byte chunks (64-byte rows, 64-byte swizzle)
+            const uint4 v = *reinterpret_cast<const uint4*>(pk + row * 64 + q * 16);
+            const uint2 mw2 = *reinterpret_cast<const uint2*>(pk + kValsTile + row * 32 + q * 8);
             unsigned char* arow = stages + (size_t)st * kStageBytes + kBTile + row * 64;
-            const uint32_t w[2] = {v.x, v.y};
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < 4; ++c) {
                 const uint32_t ws = w[c] >> 4;
                 uint4 o;
                 o.x = nib2bf16<0>(w[c], ws); o.y = nib2bf16<1>(w[c], ws);
                 o.z = nib2bf16<2>(w[c], ws); o.w = nib2bf16<3>(w[c], ws);
-                const int chunk = half * 2 + c;
-                *reinterpret_cast<uint4*>(arow + (((chunk ^ (row >> 1)) & 3) << 4)) = o;
+                *reinterpret_cast<uint4*>(arow + (((c ^ (row >> 1)) & 3) << 4)) = o;
             }
-            // ---- index word of MMA `half` (layout in the file header)
-            const uint32_t mw = *reinterpret_cast<const uint32_t*>(pk + kValsTile + row * 32 + q * 8 + 4 * half);
-            const uint32_t send = x ? (mw & 0xFFFFu) : (mw >> 16);
-            const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 8);
-            const uint32_t e = x ? ((mw & 0xFFFF0000u) | recv) : ((mw & 0xFFFFu) | (recv << 16));
-            asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};"
-                         :: "r"(tmem_base + lane_base + kECol + 4 * st + half), "r"(e) : "memory");
+            // ---- index words of the stage's two MMAs (layout in the file header)
+            uint32_t e[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t mw = h ? mw2.y : mw2.x;
+                const uint32_t send = x ? (mw & 0xFFFFu) : (mw >> 16);
+                const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 8);
+                e[h] = x ? ((mw & 0xFFFF0000u) | recv) : ((mw & 0xFFFFu) | (recv << 16));
+            }
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};"
+                         :: "r"(tmem_base + lane_base + kECol + 4 * st), "r"(e[0]), "r"(e[1]) : "memory");
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // A is read by the tensor core
             fence_before_sync();
             // one arrival per warp: arrivals on one barrier are served one after another
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&conv_done[st]);
-                if (q == kPkStages - 1 || it == p.n1 - 1) mbar_arrive(&pk_empty[slot]);
+                // a pair's MMAs are issued by the even CTA: both CTAs' converters report there
+                if (TWO && rank != 0) mbar_arrive_remote(peer_addr(&conv_done[st], 0));
+                else mbar_arrive(&conv_done[st]);
+                // this group's last stage of the packed tile
+                if (q >= 2 || it + 2 >= p.n1) mbar_arrive(&pk_empty[slot]);
             }
-            if (threadIdx.x == 0) PSTAMP(2, it);
+            if ((threadIdx.x & 127) == 0) PSTAMP(2, it);
         }
         // ---- epilogue: thread = output row, TMEM columns = tokens; the two halves split the columns
         ok = mbar_wait(acc_full, 0, abort_flag) && ok;
@@ -495,7 +515,7 @@ static PfEncodeTiledFn pf_encode_fn() {
 
 // Row-major 2-D tensor [rows][row_elems]; box of box_rows x box_elems elements.
 static bool pf_map(CUtensorMap* map, const void* base, CUtensorMapDataType type, int esize, uint64_t row_elems,
-                   uint64_t rows, int box_elems, int box_rows, bool swizzle128) {
+                   uint64_t rows, int box_elems, int box_rows, int swizzle_bytes) {
     PfEncodeTiledFn fn = pf_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {row_elems, rows};
@@ -503,7 +523,7 @@ static bool pf_map(CUtensorMap* map, const void* base, CUtensorMapDataType type,
     cuuint32_t box[2] = {(cuuint32_t)box_elems, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -559,24 +579,28 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     // token tile: 256 when that still gives every SM a tile, else 64
     const bool wide = (long long)(d_out / kPM) * ceil_div(b, 256) >= di->sm_count;
     const int n_pre = 64;                         // the T' product has few row tiles: narrow token tiles fill the machine
-    const bool pair = false && wide && (d_out / kPM) % 2 == 0;     // pairs of CTAs need an even number of row tiles
+    // The CTA-pair kernel (prefill_kernel<256, true>) is correct but measures slower than one CTA
+    // per tile (about 500 ns per stage against 420), so it is not dispatched.
+    const bool pair = false;
     const int xbox = wide ? (pair ? 128 : 256) : 64;      // token rows one CTA loads per stage = one TMA box
+    const int dk = pair ? PfCfg<256, true>::kDK : PfCfg<256, false>::kDK;   // columns of a dense stage
     CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;
-    bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPkStages * kPBK / 4, kPM, false) &&
-              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPkStages * kPBK / 8, kPM, false) &&
-              pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, xbox, true);
+    bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPkStages * kPBK / 4, kPM, 0) &&
+              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPkStages * kPBK / 8, kPM, 0) &&
+              pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, xbox, 128);
     if (!ok) return SLIM_ERR_CUDA;
     if (r > 0) {
         // T' = (X R^T) / s : dense phase only, output rows = adapter index
-        ok = pf_map(&tmA2, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 64, kPM, true) &&
-             pf_map(&tmXpre, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, 64, true);
+        ok = pf_map(&tmA2, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 64, kPM, 128) &&
+             pf_map(&tmXpre, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, 64, 128);
         if (!ok) return SLIM_ERR_CUDA;
         PrefillParams q;
         q.out = Tq; q.ldo = r; q.m_total = r; q.b = b; q.n1 = 0; q.n2 = d_in / kPBK; q.scale = 1.f / s_eff; q.status = status_dev;
         slim_status_t rc = launch_tile_kernel<64, false>(q, r, tmV, tmM, tmXpre, tmA2, tmXpre, st);
         if (rc != SLIM_OK) return rc;
-        ok = pf_map(&tmA2, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, 64, kPM, true) &&
-             pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, 64, xbox, true);
+        // dense stages of the main kernel: 64 columns (128-byte rows), or 32 (64-byte rows) in the pair kernel
+        ok = pf_map(&tmA2, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, dk, kPM, dk == 64 ? 128 : 64) &&
+             pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, dk, xbox, dk == 64 ? 128 : 64);
         if (!ok) return SLIM_ERR_CUDA;
     } else {
         tmA2 = tmX; tmB2 = tmX;       // never used when r == 0
@@ -584,7 +608,7 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     PrefillParams p;
     p.out = Y; p.ldo = d_out; p.m_total = d_out; p.b = b;
     p.n1 = s != 0.f ? d_in / kPBK : 0;
-    p.n2 = r > 0 ? ceil_div(r, kPBK) : 0;
+    p.n2 = r > 0 ? ceil_div(r, dk) : 0;
     p.scale = s_eff; p.status = status_dev;
     if (p.n1 + p.n2 == 0)             // s == 0 and no adapters: the result is zero
         return cudaMemsetAsync(Y, 0, (size_t)b * d_out * 2, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
