@@ -54,16 +54,19 @@ constexpr uint32_t kPSpinLimit = 1u << 21;
 // loads half of it and one cta_group::2 MMA of shape 256 x N, issued by the even CTA,
 // drives both tensor cores.  Halves the token-tile traffic per CTA and leaves room for
 // more stages.
-template <int N, bool TWO> struct PfCfg {
+// PRE = the dense-only launch (T' product): no packed tiles, so the room goes to more stages.
+template <int N, bool TWO, bool PRE = false> struct PfCfg {
     static constexpr int kBRows = TWO ? N / 2 : N;                          // token rows this CTA loads
     static constexpr int kBTile = kBRows * 128;
-    // A region of a stage: the expanded weight tile needs 8 KB; the pair kernel's dense stages are
-    // 32 columns wide so that their A2 tile fits there too and more stages fit in shared memory.
-    static constexpr int kARegion = TWO ? kATile / 2 : kATile;
-    static constexpr int kDK = TWO ? 32 : 64;                               // columns of a dense stage
-    static constexpr int kStages = TWO ? 7 : 4;
+    // A region of a stage: the expanded weight tile needs 8 KB.  The main kernels' dense stages are
+    // 32 columns wide so that their A2 tile fits there too: a smaller stage means more stages in
+    // flight, and the loop is bound by the latency of the token tile.  The dense-only launch
+    // has no expanded tiles and keeps 64-column stages.
+    static constexpr int kARegion = PRE ? kATile : kATile / 2;
+    static constexpr int kDK = PRE ? 64 : 32;                               // columns of a dense stage
+    static constexpr int kStages = PRE ? (N >= 256 ? 4 : 8) : (TWO ? 7 : (N >= 256 ? 5 : 8));
     // Packed tiles come from HBM (latency of a microsecond or two): the ring holds what fits.
-    static constexpr int kPkSlots = TWO ? 4 : (N >= 256 ? 2 : 8);
+    static constexpr int kPkSlots = PRE ? 1 : (TWO ? 4 : (N >= 256 ? 2 : 7));
     static constexpr int kStageBytes = kBTile + kARegion;
     static constexpr int kECol = N;                                         // index words: N + 4 * stage + mma
     static constexpr int kTmemCols = N >= 256 ? 512 : (N >= 128 ? 256 : 128);
@@ -78,13 +81,20 @@ struct PrefillParams {
     int n1, n2;             // stages of the sparse and of the dense phase
     float scale;
     uint32_t* status;
+    // dense-only launch split along K over blockIdx.z: slice z covers `k_per` stages from z * k_per and
+    // writes its fp32 partial tile to part[z][token][ldo] (part == nullptr: one slice, bf16 to out)
+    float* part;
+    int k_per;
 };
 
 // Optional timeline: built with -DSLIM_PREFILL_TRACE, one thread per warp role of the first
 // CTAs records the global timer around its waits for the first 48 stages.
 #ifdef SLIM_PREFILL_TRACE
+#ifndef SLIM_PTRACE_PRE
+#define SLIM_PTRACE_PRE 0          // 1: stamp the dense-only launch instead of the main one
+#endif
 __device__ unsigned long long g_ptrace[8][6][48];
-#define PSTAMP(role, it) do { if (blockIdx.x + gridDim.x * blockIdx.y < 8 && (it) < 48) { unsigned long long t_; \
+#define PSTAMP(role, it) do { if (PRE == (SLIM_PTRACE_PRE != 0) && blockIdx.z == 0 && blockIdx.x + gridDim.x * blockIdx.y < 8 && (it) < 48) { unsigned long long t_; \
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_ptrace[blockIdx.x + gridDim.x * blockIdx.y][role][it] = t_; } } while (0)
 #else
 #define PSTAMP(role, it) do { } while (0)
@@ -237,16 +247,30 @@ __device__ __forceinline__ uint32_t nib2bf16(uint32_t w, uint32_t w_shr4) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// 32 consecutive 32-bit columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 }  // namespace pf
 
-template <int N, bool TWO>
+template <int N, bool TWO, bool PRE = false>
 __global__ void __launch_bounds__(kPThreads, 1)
 prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmX,
                const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2)
 {
     using namespace pf;
-    using Cfg = PfCfg<N, TWO>;
+    using Cfg = PfCfg<N, TWO, PRE>;
     constexpr int kBTile = Cfg::kBTile, kStageBytes = Cfg::kStageBytes, kECol = Cfg::kECol, kPStages = Cfg::kStages;
     constexpr int kPkSlots = Cfg::kPkSlots, kDK = Cfg::kDK;
     extern __shared__ unsigned char smem_raw[];
@@ -268,7 +292,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     const uint32_t rank = TWO ? cluster_rank() : 0u;           // 0 = the CTA that issues the pair's MMAs
     const int m0 = blockIdx.x * kPM, n0 = blockIdx.y * N;
     const int nb0 = n0 + (int)rank * Cfg::kBRows;                // first token row this CTA loads
-    const int n_total = p.n1 + p.n2;
+    const int k_first = PRE && p.part ? (int)blockIdx.z * p.k_per : 0;      // first dense stage of this K slice
+    const int n_total = PRE && p.part ? min(p.k_per, p.n2 - k_first) : p.n1 + p.n2;
     // CTAs that share token rows start their walk over the weight columns at different places,
     // so that at any moment they ask the L2 for different lines of X rather than all for the same
     // ones.  The walk is rotated by whole 256-column groups (a pair of CTAs rotates together).
@@ -276,6 +301,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     const int rot_g = (p.n1 % kPkStages == 0 && n_groups > 0)
                           ? (int)(((blockIdx.x >> (TWO ? 1 : 0)) + 3u * blockIdx.y) % (unsigned)n_groups) : 0;
 
+    if (threadIdx.x == 0) PSTAMP(5, 44);
     if (threadIdx.x == 0) {
         for (int i = 0; i < kPStages; ++i) {
             mbar_init(&b_full[i], 1);
@@ -301,6 +327,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
     bool ok = true;
+    if (threadIdx.x == 0) PSTAMP(5, 45);
 
     if (warp == kWarpXEven || warp == kWarpXOdd) {
         // ============================ token-tile producers ============================
@@ -317,7 +344,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             // dense stage: kDK columns of the token rows and of the A2 rows
             if (lane == 0) mbar_expect_tx(&b_full[st], (uint32_t)(sparse ? kBTile : (Cfg::kBRows + kPM) * kDK * 2));
             unsigned char* sbase = stages + (size_t)st * kStageBytes;
-            int kb = sparse ? it + rot_g * kPkStages : it - p.n1;
+            int kb = sparse ? it + rot_g * kPkStages : it - p.n1 + k_first;
             if (sparse && kb >= p.n1) kb -= p.n1;
             const int k = sparse ? kb * kPBK : kb * kDK;
             // lane 0: the token tile (one box); lane 1, dense stages only: the A2 tile
@@ -339,8 +366,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
         }
     } else if (warp == kWarpMma) {
         // ============================ MMA issuer ============================
-        // The whole warp walks the stages and waits together; one elected lane issues (a loop run
-        // by a single lane of a diverged warp issues the tensor-core instructions more slowly).
+        // One elected lane walks the stages and issues.
         if (TWO && rank != 0) {
             // Odd CTA of a pair: tell the even CTA when this CTA's token rows (and A2 rows) of a
             // stage have landed.  The data stay in this CTA's shared memory and are read by this
@@ -354,7 +380,7 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                     PSTAMP(5, it);
                 }
             }
-        } else {
+        } else if (elect_one()) {
             constexpr uint32_t idesc = idesc_bf16(TWO ? 2 * kPM : kPM, N);
             for (int it = 0; it < n_total; ++it) {
                 const int st = it % kPStages;
@@ -370,7 +396,6 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 fence_after_sync();
                 const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
                 const uint32_t a_addr = b_addr + kBTile;
-                if (!elect_one()) continue;
                 PSTAMP(3, it);
                 if (sparse) {
                     // per MMA: A 16 stored bf16 (32 bytes of a 64-byte row), B 32 columns (64 bytes)
@@ -386,9 +411,10 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
 #pragma unroll
                     for (int j = 0; j < kDK / 16; ++j) {
                         const uint32_t acc = (it > 0 || j > 0) ? 1u : 0u;
-                        // pair kernel: 32-column stages, 64-byte rows with the 64-byte swizzle
-                        if (TWO) mma_dense2(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc64(b_addr + 32 * j), idesc, acc);
-                        else     mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
+                        // 32-column stages: 64-byte rows with the 64-byte swizzle; 64-column stages: 128-byte rows
+                        if (TWO)            mma_dense2(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc64(b_addr + 32 * j), idesc, acc);
+                        else if (kDK == 32) mma_dense(tmem_base, smem_desc64(a_addr + 32 * j), smem_desc64(b_addr + 32 * j), idesc, acc);
+                        else                mma_dense(tmem_base, smem_desc(a_addr + 32 * j), smem_desc(b_addr + 32 * j), idesc, acc);
                     }
                 }
                 // the stage is free (in both CTAs of a pair) once these MMAs have read it
@@ -396,10 +422,8 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 else mma_commit(&empty[st]);
                 PSTAMP(4, it);
             }
-            if (elect_one()) {
-                if (TWO) { mma_commit2(peer_addr(acc_full, 0)); mma_commit2(peer_addr(acc_full, 1)); }
-                else mma_commit(acc_full);
-            }
+            if (TWO) { mma_commit2(peer_addr(acc_full, 0)); mma_commit2(peer_addr(acc_full, 1)); }
+            else mma_commit(acc_full);
         }
     } else {
         // ============================ converters, then epilogue ============================
@@ -459,32 +483,26 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
         // ---- epilogue: thread = output row, TMEM columns = tokens; the two halves split the columns
         ok = mbar_wait(acc_full, 0, abort_flag) && ok;
         fence_after_sync();
+        if (threadIdx.x == 0) PSTAMP(5, 46);
         const int orow = m0 + row;
 #pragma unroll 1
         for (int c0 = half * (N / 2); c0 < (half + 1) * (N / 2); c0 += 32) {
             uint32_t r[32];
-            const uint32_t taddr = tmem_base + lane_base + c0;
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                  "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                  "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                  "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                : "r"(taddr) : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            tmem_ld32(tmem_base + lane_base + c0, r);
             if (orow < p.m_total) {
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
                     const int token = n0 + c0 + c;
-                    if (token < p.b)
-                        p.out[(size_t)token * p.ldo + orow] = __float2bfloat16_rn(p.scale * __uint_as_float(r[c]));
+                    if (token < p.b) {
+                        if (PRE && p.part) p.part[((size_t)blockIdx.z * p.b + token) * p.ldo + orow] = __uint_as_float(r[c]);
+                        else p.out[(size_t)token * p.ldo + orow] = __float2bfloat16_rn(p.scale * __uint_as_float(r[c]));
+                    }
                 }
             }
         }
     }
 
+    if (threadIdx.x == 0) PSTAMP(5, 47);
     if (!ok && lane == 0) flag_error(p.status, SLIM_ERR_TIMEOUT);
     fence_before_sync();
     __syncthreads();
@@ -496,7 +514,43 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
     }
 }
 
+// Sum of the K slices' partial tiles, scaled and rounded to bf16 (fixed order: deterministic).
+__global__ void pre_reduce_kernel(const float* __restrict__ part, int slices, size_t n, float scale, __nv_bfloat16* __restrict__ out)
+{
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= n) return;
+    float4 acc = *reinterpret_cast<const float4*>(part + i);
+    for (int z = 1; z < slices; ++z) {
+        const float4 v = *reinterpret_cast<const float4*>(part + (size_t)z * n + i);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    __nv_bfloat162 lo = __floats2bfloat162_rn(scale * acc.x, scale * acc.y), hi = __floats2bfloat162_rn(scale * acc.z, scale * acc.w);
+    uint2 o; o.x = *reinterpret_cast<uint32_t*>(&lo); o.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(out + i) = o;
+}
+
 // ------------------------------------------------------------------ host side
+// Shape of the dense-only launch T' = X R^T: token tile, K slices, stages per slice.  The product
+// has few tiles (r / 128 x tokens / tile), so K is split until they about fill the machine.
+struct PrePlan { int n_tok; int slices; int k_per; };
+static PrePlan pre_plan(int b, int d_in, int r, int sm_count) {
+    PrePlan pl;
+    pl.n_tok = b >= 192 ? 256 : 64;
+    const int tiles = ceil_div(r, kPM) * ceil_div(b, pl.n_tok);
+    const int n2 = d_in / kPBK;
+    int ks = sm_count / (tiles > 0 ? tiles : 1);
+    ks = ks < 1 ? 1 : (ks > 8 ? 8 : ks);
+    if (ks > n2) ks = n2 > 0 ? n2 : 1;
+    pl.k_per = ceil_div(n2, ks);
+    pl.slices = ceil_div(n2, pl.k_per);          // every slice has at least one stage
+    return pl;
+}
+static int pre_sm_count() {
+    slim_status_t err = SLIM_OK;
+    const DeviceInfo* di = device_info(&err);
+    return di && di->sm_count > 0 ? di->sm_count : 148;
+}
+
 typedef CUresult (*PfEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -533,25 +587,28 @@ bool prefill_supports(int b, int d_out, int d_in, int r) {
 
 size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r) {
     if (!prefill_supports(b, d_out, d_in, r)) return 0;
-    return ((size_t)b * (size_t)r * sizeof(__nv_bfloat16) + 255) / 256 * 256;
+    const size_t tq = ((size_t)b * (size_t)r * sizeof(__nv_bfloat16) + 255) / 256 * 256;
+    if (r == 0) return tq;
+    const PrePlan pl = pre_plan(b, d_in, r, pre_sm_count());
+    return tq + (pl.slices > 1 ? (size_t)pl.slices * b * r * sizeof(float) : 0);
 }
 
 static bool g_prefill_attr_set[64];
 
-template <int N, bool TWO>
+template <int N, bool TWO, bool PRE = false>
 static slim_status_t launch_tile_kernel(const PrefillParams& q, int m_rows, const CUtensorMap& tmV, const CUtensorMap& tmM,
                                         const CUtensorMap& tmX, const CUtensorMap& tmA2, const CUtensorMap& tmB2,
-                                        cudaStream_t st) {
+                                        cudaStream_t st, int slices = 1) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ceil_div(m_rows, kPM), ceil_div(q.b, N));
+    cfg.gridDim = dim3(ceil_div(m_rows, kPM), ceil_div(q.b, N), slices);
     cfg.blockDim = dim3(kPThreads);
-    cfg.dynamicSmemBytes = PfCfg<N, TWO>::kSmem;
+    cfg.dynamicSmemBytes = PfCfg<N, TWO, PRE>::kSmem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = TWO ? 2 : 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_kernel<N, TWO>, q, tmV, tmM, tmX, tmA2, tmB2);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_kernel<N, TWO, PRE>, q, tmV, tmM, tmX, tmA2, tmB2);
     count_launch(1);
     return e == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
 }
@@ -570,7 +627,9 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     if (dev >= 0 && dev < 64 && !g_prefill_attr_set[dev]) {
         if (cudaFuncSetAttribute(prefill_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256, true>::kSmem) != cudaSuccess ||
             cudaFuncSetAttribute(prefill_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256, false>::kSmem) != cudaSuccess ||
-            cudaFuncSetAttribute(prefill_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<64, false>::kSmem) != cudaSuccess)
+            cudaFuncSetAttribute(prefill_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<64, false>::kSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_kernel<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<64, false, true>::kSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_kernel<256, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256, false, true>::kSmem) != cudaSuccess)
             return SLIM_ERR_CUDA;
         g_prefill_attr_set[dev] = true;
     }
@@ -583,7 +642,7 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     // per tile (about 500 ns per stage against 420), so it is not dispatched.
     const bool pair = false;
     const int xbox = wide ? (pair ? 128 : 256) : 64;      // token rows one CTA loads per stage = one TMA box
-    const int dk = pair ? PfCfg<256, true>::kDK : PfCfg<256, false>::kDK;   // columns of a dense stage
+    const int dk = PfCfg<256, false>::kDK;                // columns of a dense stage of the main kernels
     CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;
     bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPkStages * kPBK / 4, kPM, 0) &&
               pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPkStages * kPBK / 8, kPM, 0) &&
@@ -591,13 +650,24 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     if (!ok) return SLIM_ERR_CUDA;
     if (r > 0) {
         // T' = (X R^T) / s : dense phase only, output rows = adapter index
+        const PrePlan pl = pre_plan(b, d_in, r, di->sm_count);
         ok = pf_map(&tmA2, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 64, kPM, 128) &&
-             pf_map(&tmXpre, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, 64, 128);
+             pf_map(&tmXpre, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, pl.n_tok, 128);
         if (!ok) return SLIM_ERR_CUDA;
         PrefillParams q;
         q.out = Tq; q.ldo = r; q.m_total = r; q.b = b; q.n1 = 0; q.n2 = d_in / kPBK; q.scale = 1.f / s_eff; q.status = status_dev;
-        slim_status_t rc = launch_tile_kernel<64, false>(q, r, tmV, tmM, tmXpre, tmA2, tmXpre, st);
+        q.k_per = pl.k_per;
+        // partial tiles of the K slices follow T' in the workspace
+        q.part = pl.slices > 1 ? reinterpret_cast<float*>(reinterpret_cast<char*>(Tq) + ((size_t)b * r * sizeof(__nv_bfloat16) + 255) / 256 * 256) : nullptr;
+        slim_status_t rc = pl.n_tok == 256 ? launch_tile_kernel<256, false, true>(q, r, tmV, tmM, tmXpre, tmA2, tmXpre, st, pl.slices)
+                                           : launch_tile_kernel<64, false, true>(q, r, tmV, tmM, tmXpre, tmA2, tmXpre, st, pl.slices);
         if (rc != SLIM_OK) return rc;
+        if (q.part) {
+            const size_t n = (size_t)b * r;
+            pre_reduce_kernel<<<(unsigned)((n / 4 + 255) / 256), 256, 0, st>>>(q.part, pl.slices, n, q.scale, Tq);
+            count_launch(1);
+            if (cudaGetLastError() != cudaSuccess) return SLIM_ERR_CUDA;
+        }
         // dense stages of the main kernel: 64 columns (128-byte rows), or 32 (64-byte rows) in the pair kernel
         ok = pf_map(&tmA2, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, dk, kPM, dk == 64 ? 128 : 64) &&
              pf_map(&tmB2, Tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)b, dk, xbox, dk == 64 ? 128 : 64);
@@ -609,7 +679,7 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     p.out = Y; p.ldo = d_out; p.m_total = d_out; p.b = b;
     p.n1 = s != 0.f ? d_in / kPBK : 0;
     p.n2 = r > 0 ? ceil_div(r, dk) : 0;
-    p.scale = s_eff; p.status = status_dev;
+    p.scale = s_eff; p.status = status_dev; p.part = nullptr; p.k_per = 0;
     if (p.n1 + p.n2 == 0)             // s == 0 and no adapters: the result is zero
         return cudaMemsetAsync(Y, 0, (size_t)b * d_out * 2, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
     if (!wide) return launch_tile_kernel<64, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);

@@ -77,7 +77,8 @@ PREFILL_SMALL = [  # d_in, d_out, r, b
 def test_small_prefill_kernel(d_in, d_out, r, b):
     res = run_case(d_in, d_out, r, b, seed=13, kernel=K.KERNEL_PREFILL)
     assert_ok(res)
-    assert res["launches"] == (2 if r else 1)
+    # main launch; with adapters also the T' launch and, when that one is split along K, its reduction
+    assert res["launches"] in ((2, 3) if r else (1,))
 
 
 def test_prefill_integer_inputs_are_exact():
