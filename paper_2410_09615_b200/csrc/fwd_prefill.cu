@@ -443,8 +443,10 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
             if ((threadIdx.x & 127) == 0) PSTAMP(1, it);
             // ---- 16 value bytes -> 32 bf16: the row's four 16-byte chunks (64-byte rows, 64-byte swizzle)
-            const uint4 v = *reinterpret_cast<const uint4*>(pk + row * 64 + q * 16);
-            const uint2 mw2 = *reinterpret_cast<const uint2*>(pk + kValsTile + row * 32 + q * 8);
+            // the packed tiles are stored with the 64-byte (values) and 32-byte (indices) TMA swizzles so
+            // that a warp's row-strided reads spread over the banks
+            const uint4 v = *reinterpret_cast<const uint4*>(pk + row * 64 + (((q ^ (row >> 1)) & 3) << 4));
+            const uint2 mw2 = *reinterpret_cast<const uint2*>(pk + kValsTile + row * 32 + ((((q >> 1) ^ (row >> 2)) & 1) << 4) + (q & 1) * 8);
             unsigned char* arow = stages + (size_t)st * kStageBytes + kBTile + row * 64;
             const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -577,7 +579,7 @@ static bool pf_map(CUtensorMap* map, const void* base, CUtensorMapDataType type,
     cuuint32_t box[2] = {(cuuint32_t)box_elems, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -644,8 +646,8 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     const int xbox = wide ? (pair ? 128 : 256) : 64;      // token rows one CTA loads per stage = one TMA box
     const int dk = PfCfg<256, false>::kDK;                // columns of a dense stage of the main kernels
     CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;
-    bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPkStages * kPBK / 4, kPM, 0) &&
-              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPkStages * kPBK / 8, kPM, 0) &&
+    bool ok = pf_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, kPkStages * kPBK / 4, kPM, 64) &&
+              pf_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, kPkStages * kPBK / 8, kPM, 32) &&
               pf_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, xbox, 128);
     if (!ok) return SLIM_ERR_CUDA;
     if (r > 0) {
