@@ -5,14 +5,17 @@
 //     out[token][row] = scale * ( sum_k W[row][k] X[token][k]  +  sum_j A2[row][j] B2[token][j] )
 // in two chained phases that accumulate into the same TMEM tile:
 //   phase 1 (sparse): W is the packed int4 2:4 weight.  TMA brings 128 rows of value
-//       bytes and index bytes plus the X tile; eight converter warps (two threads per
-//       weight row) expand nibbles to exact bf16 into the 64-byte-swizzled K-major
-//       layout the MMA reads, and write the 2:4 index words into tensor memory;
-//       one thread issues tcgen05.mma.sp (kind::f16, bf16 x bf16 -> fp32).
+//       bytes and index bytes plus the X tile; eight converter warps (two groups on
+//       alternate stages, one thread per weight row) expand nibbles to exact bf16 into the
+//       64-byte-swizzled K-major layout the MMA reads, and write the 2:4 index words into
+//       tensor memory; one thread issues tcgen05.mma.sp (kind::f16, bf16 x bf16 -> fp32).
 //   phase 2 (dense): A2 and B2 are bf16 matrices brought by TMA as they are; the same
 //       thread issues tcgen05.mma into the same accumulator.
-// The layer forward is two launches of this kernel:
-//   T' = (X R^T) / s          phase 2 only  (A2 = R, B2 = X, scale 1/s), bf16 into the workspace
+// The layer forward is two or three launches:
+//   T' = (X R^T) / s          phase 2 only (A2 = R, B2 = X, scale 1/s), bf16 into the workspace.
+//                             The product has few tiles, so K is split over blockIdx.z; the
+//                             slices write fp32 partial tiles and a small kernel adds them in a
+//                             fixed order (one slice: bf16 directly, no second launch).
 //   Y  = s * (X Q^T + T' L^T) phase 1 then phase 2 (A2 = L, B2 = T', scale s)
 // so the adapter product and the scale are fused into the tile loop and the epilogue.
 //
@@ -23,15 +26,21 @@
 // packed index array is one row's 32 columns, so a converter thread swaps one
 // half-word with the thread eight rows away and stores the result.
 //
-// Pipeline.  4 stages of {B: N tokens x 128 bytes, A: 16 KB (8 KB used in phase 1)}; a
-// stage is 64 weight columns (two sparse MMAs of K = 32, or four dense MMAs of K = 16).
-// The packed value and index bytes travel separately, 256 columns (4 stages) per TMA tile,
-// through a 2-slot ring of their own.  A thread is held ~160 ns by every TMA request it
-// starts, so requests are spread over three producer warps: token tiles of even stages,
-// token tiles of odd stages (each with the A2 tile in phase 2), packed tiles.
-// mbarriers: b_full / pk_full (TMA bytes landed), conv_done (converters
-// finished a stage), empty / pk_empty (tcgen05.commit: the MMAs that read the stage are
-// complete; converters done with a packed slot), acc_full.
+// Pipeline.  A ring of stages {B: token rows x 128 bytes, A: 8 KB (16 KB in the dense-only
+// launch)}; a sparse stage is 64 weight columns (two MMAs of K = 32), a dense stage 32 columns
+// (two MMAs of K = 16; 64 columns in the dense-only launch).  The packed value and index bytes
+// travel separately, 256 columns (4 stages) per TMA tile, through a ring of their own.
+// Warps: 0-7 converters, then epilogue; 8 and 10 token tiles of even / odd stages (with the A2
+// tile in phase 2); 9 MMA issue; 11 packed tiles.
+// mbarriers: b_full / pk_full (TMA bytes landed), conv_done (converters finished a stage),
+// empty / pk_empty (tcgen05.commit: the MMAs that read the stage are complete; converters
+// done with a packed slot), acc_full.
+// Measured on B200 and built into the loops below: a barrier operation is served per thread
+// (a warp-wide try_wait or 32 arrivals cost 32 times one), a lane left at a warp barrier
+// while another lane of its warp spins costs some hundred nanoseconds per iteration, and one
+// MMA costs at least the 128 cycles its 128-row A operand takes to load, whatever N.
+// With one CTA per tile the loop is bound by shared-memory bandwidth: per stage TMA writes
+// 35 KB, the tensor core reads 40 KB, the converters move 11 KB.
 // Every wait is bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on.
 #include <cuda.h>
 #include "common.cuh"
