@@ -593,7 +593,8 @@ static bool pf_map(CUtensorMap* map, const void* base, CUtensorMapDataType type,
 }
 
 bool prefill_supports(int b, int d_out, int d_in, int r) {
-    return b >= 1 && d_out % kPM == 0 && d_in % kPBK == 0 && r % 16 == 0 && r >= 0;
+    // d_in % 128: the rows of the index-byte array (d_in / 8 bytes) must be a multiple of 16 bytes for TMA
+    return b >= 1 && d_out % kPM == 0 && d_in % 128 == 0 && r % 16 == 0 && r >= 0;
 }
 
 size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r) {

@@ -55,11 +55,13 @@ def test_dispatcher_choices():
     assert K.slim_select_kernel(17, 4096, 4096, 416) == K.KERNEL_PREFILL
     assert K.slim_select_kernel(2048, 4096, 11008, 416) == K.KERNEL_PREFILL
     assert K.slim_select_kernel(64, 48, 4096, 16) == K.KERNEL_SIMPLE        # d_out not a multiple of 128
+    assert K.slim_select_kernel(50, 128, 704, 32) == K.KERNEL_SIMPLE        # d_in not a multiple of 128
 
 
 def test_shapes_outside_the_fast_kernels_still_work():
     assert_ok(run_case(64, 16, 16, 2, seed=31))          # d_in = 64: simple kernel
     assert_ok(run_case(320, 32, 0, 40, seed=32))         # b > 16, no adapters
+    assert_ok(run_case(704, 128, 32, 50, seed=33))       # b > 16, d_in % 128 != 0: not the prefill kernel
 
 
 # ---- tcgen05 prefill kernel, small cases, all elements ----------------------
@@ -70,6 +72,8 @@ PREFILL_SMALL = [  # d_in, d_out, r, b
     (1024, 384, 64, 128),    # more stages than the ring holds
     (640, 128, 48, 8),       # a batch the dispatcher would give to the decode kernel
     (2048, 512, 208, 300),
+    (1408, 128, 32, 50),     # 22 stages: the K slices of the T' launch are uneven
+    (384, 256, 16, 600),     # more token tiles than stages per slice
 ]
 
 
