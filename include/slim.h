@@ -68,7 +68,9 @@ typedef enum {
     SLIM_KERNEL_AUTO = 0,    /* by batch size: decode for b <= 16, prefill above */
     SLIM_KERNEL_SIMPLE = 1,  /* CUDA-core kernel, any legal shape; correctness anchor */
     SLIM_KERNEL_DECODE = 2,  /* streaming sparse tensor-core kernel for small batches */
-    SLIM_KERNEL_PREFILL = 3  /* tcgen05 sparse tensor-core kernel for many tokens */
+    SLIM_KERNEL_PREFILL = 3, /* tcgen05 sparse tensor-core kernel for many tokens */
+    SLIM_KERNEL_PREFILL_PAIR = 4 /* the same with two CTAs per 256-row tile (cta_group::2); never chosen
+                                    by the dispatcher; needs an even number of 128-row tiles */
 } slim_kernel_t;
 
 /*

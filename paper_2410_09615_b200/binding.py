@@ -18,8 +18,8 @@ LIB_PATH = os.path.join(_HERE, "libslim.so")
 
 (SLIM_OK, SLIM_ERR_INVALID_ARG, SLIM_ERR_UNSUPPORTED_SHAPE, SLIM_ERR_BAD_MASK, SLIM_ERR_CODE_RANGE,
  SLIM_ERR_WORKSPACE, SLIM_ERR_CUDA, SLIM_ERR_TIMEOUT, SLIM_ERR_ARCH) = range(9)
-KERNEL_AUTO, KERNEL_SIMPLE, KERNEL_DECODE, KERNEL_PREFILL = range(4)
-KERNEL_NAMES = {KERNEL_AUTO: "auto", KERNEL_SIMPLE: "simple", KERNEL_DECODE: "decode", KERNEL_PREFILL: "prefill"}
+KERNEL_AUTO, KERNEL_SIMPLE, KERNEL_DECODE, KERNEL_PREFILL, KERNEL_PREFILL_PAIR = range(5)
+KERNEL_NAMES = {KERNEL_AUTO: "auto", KERNEL_SIMPLE: "simple", KERNEL_DECODE: "decode", KERNEL_PREFILL: "prefill", KERNEL_PREFILL_PAIR: "prefill_pair"}
 WORKSPACE_SYNC_BYTES = 256
 NOALLOC_SCRATCH_BYTES = 16 << 20
 

@@ -141,6 +141,9 @@ slim_status_t slim_linear_fwd_ex(const void* X, int b, const uint8_t* vals, cons
     case SLIM_KERNEL_PREFILL:
         if (!prefill_supports(b, d_out, d_in, r)) return SLIM_ERR_UNSUPPORTED_SHAPE;
         return launch_prefill(Xb, b, vals, meta, s, Lb, Rb, r, d_out, d_in, Yb, workspace, status_dev, stream);
+    case SLIM_KERNEL_PREFILL_PAIR:
+        if (!prefill_supports(b, d_out, d_in, r)) return SLIM_ERR_UNSUPPORTED_SHAPE;
+        return launch_prefill(Xb, b, vals, meta, s, Lb, Rb, r, d_out, d_in, Yb, workspace, status_dev, stream, true);
     default:
         return SLIM_ERR_UNSUPPORTED_SHAPE;
     }

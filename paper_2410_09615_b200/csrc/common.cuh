@@ -51,6 +51,6 @@ size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r);
 slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
                              float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
                              int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
-                             cudaStream_t st);
+                             cudaStream_t st, bool force_pair = false);
 
 }  // namespace slim

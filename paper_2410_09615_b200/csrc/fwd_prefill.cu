@@ -628,7 +628,7 @@ static slim_status_t launch_tile_kernel(const PrefillParams& q, int m_rows, cons
 slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
                              float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
                              int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
-                             cudaStream_t st)
+                             cudaStream_t st, bool force_pair)
 {
     slim_status_t err;
     const DeviceInfo* di = device_info(&err);
@@ -648,11 +648,12 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     __nv_bfloat16* Tq = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + SLIM_WORKSPACE_SYNC_BYTES);
     const float s_eff = s != 0.f ? s : 1.f;       // with s == 0 only the adapter term remains
     // token tile: 256 when that still gives every SM a tile, else 64
-    const bool wide = (long long)(d_out / kPM) * ceil_div(b, 256) >= di->sm_count;
+    const bool wide = force_pair || (long long)(d_out / kPM) * ceil_div(b, 256) >= di->sm_count;
     const int n_pre = 64;                         // the T' product has few row tiles: narrow token tiles fill the machine
-    // The CTA-pair kernel (prefill_kernel<256, true>) is correct but measures slower than one CTA
-    // per tile (about 500 ns per stage against 420), so it is not dispatched.
-    const bool pair = false;
+    // The CTA-pair kernel (prefill_kernel<256, true>) measures no faster than one CTA per tile, so
+    // it runs only when asked for by name.
+    if (force_pair && (d_out / kPM) % 2 != 0) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    const bool pair = force_pair;
     const int xbox = wide ? (pair ? 128 : 256) : 64;      // token rows one CTA loads per stage = one TMA box
     const int dk = PfCfg<256, false>::kDK;                // columns of a dense stage of the main kernels
     CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;

@@ -85,6 +85,24 @@ def test_small_prefill_kernel(d_in, d_out, r, b):
     assert res["launches"] in ((2, 3) if r else (1,))
 
 
+PREFILL_PAIR = [  # d_in, d_out, r, b: even numbers of 128-row tiles
+    (256, 256, 16, 40),
+    (1024, 512, 112, 300),   # ragged token tile and rank, more stages than the ring holds
+    (2048, 256, 0, 520),     # no adapters, three token tiles
+    (1408, 256, 48, 50),     # uneven K slices of the T' launch, ragged 32-column adapter stages
+]
+
+
+@pytest.mark.parametrize("d_in,d_out,r,b", PREFILL_PAIR)
+def test_small_prefill_pair_kernel(d_in, d_out, r, b):
+    assert_ok(run_case(d_in, d_out, r, b, seed=14, kernel=K.KERNEL_PREFILL_PAIR))
+
+
+def test_prefill_pair_needs_an_even_number_of_row_tiles():
+    with pytest.raises(K.SlimError):
+        run_case(256, 384, 16, 40, seed=14, kernel=K.KERNEL_PREFILL_PAIR)
+
+
 def test_prefill_integer_inputs_are_exact():
     rng = np.random.default_rng(15)
     d_in, d_out, r, b = 256, 128, 16, 48
