@@ -227,6 +227,31 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
     *abort_flag = 1u;
     return false;
 }
+// One try_wait, no loop.  `cluster`: acquire at cluster scope (arrivals came from the other CTA).
+__device__ __forceinline__ uint32_t mbar_try(uint64_t* bar, uint32_t parity, bool cluster) {
+    uint32_t done;
+    if (cluster)
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(s32(bar)), "r"(parity) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(s32(bar)), "r"(parity) : "memory");
+    return done;
+}
+// Bounded wait for several barriers at once.  A try_wait takes about 200 cycles to answer even when
+// the phase is long complete, so waits that follow each other are asked together, not in turn.
+__device__ __forceinline__ bool mbar_wait_all(uint64_t* b0, uint32_t p0, bool c0, uint64_t* b1, uint32_t p1, bool c1,
+                                              uint64_t* b2, uint32_t p2, bool c2, volatile uint32_t* abort_flag) {
+    for (uint32_t it = 0; it < kPSpinLimit; ++it) {
+        const uint32_t d0 = b0 ? mbar_try(b0, p0, c0) : 1u;
+        const uint32_t d1 = b1 ? mbar_try(b1, p1, c1) : 1u;
+        const uint32_t d2 = b2 ? mbar_try(b2, p2, c2) : 1u;
+        if (d0 & d1 & d2) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1u;
+    return false;
+}
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -395,13 +420,9 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
                 const int st = it % kPStages;
                 const uint32_t parity = (it / kPStages) & 1;
                 const bool sparse = it < p.n1;
-                ok = mbar_wait(&b_full[st], parity, abort_flag) && ok;
-                if (TWO) {          // arrivals from the other CTA: its converters, its loads
-                    if (sparse) ok = mbar_wait_cluster(&conv_done[st], parity, abort_flag) && ok;
-                    ok = mbar_wait_cluster(&peer_ready[st], parity, abort_flag) && ok;
-                } else if (sparse) {
-                    ok = mbar_wait(&conv_done[st], parity, abort_flag) && ok;
-                }
+                // token tile landed; converters done (in a pair: both CTAs', reported here); the other CTA's loads landed
+                ok = mbar_wait_all(&b_full[st], parity, false, sparse ? &conv_done[st] : nullptr, parity, TWO,
+                                   TWO ? &peer_ready[st] : nullptr, parity, true, abort_flag) && ok;
                 fence_after_sync();
                 const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
                 const uint32_t a_addr = b_addr + kBTile;
@@ -447,9 +468,10 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             const int st = it % kPStages;
             const int gi = it / kPkStages, q = it % kPkStages, slot = gi % kPkSlots;
             const unsigned char* pk = packed + slot * kPkSlotBytes;
-            ok = mbar_wait(&pk_full[slot], (gi / kPkSlots) & 1, abort_flag) && ok;
-            // the MMAs of the previous use of this stage must be done with its A tile and index words
-            if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
+            // the packed tile has landed, and the MMAs of the previous use of this stage are done with
+            // its A tile and index words
+            ok = mbar_wait_all(&pk_full[slot], (gi / kPkSlots) & 1, false, it >= kPStages ? &empty[st] : nullptr,
+                               ((it / kPStages) & 1) ^ 1, false, nullptr, 0, false, abort_flag) && ok;
             if ((threadIdx.x & 127) == 0) PSTAMP(1, it);
             // ---- 16 value bytes -> 32 bf16: the row's four 16-byte chunks (64-byte rows, 64-byte swizzle)
             // the packed tiles are stored with the 64-byte (values) and 32-byte (indices) TMA swizzles so
