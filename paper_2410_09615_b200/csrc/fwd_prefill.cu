@@ -416,25 +416,14 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             }
         } else if (elect_one()) {
             constexpr uint32_t idesc = idesc_bf16(TWO ? 2 * kPM : kPM, N);
-            uint32_t pre = 0;       // the coming stage was found ready by an early probe
             for (int it = 0; it < n_total; ++it) {
                 const int st = it % kPStages;
                 const uint32_t parity = (it / kPStages) & 1;
                 const bool sparse = it < p.n1;
                 // token tile landed; converters done (in a pair: both CTAs', reported here); the other CTA's loads landed
-                if (!pre)
-                    ok = mbar_wait_all(&b_full[st], parity, false, sparse ? &conv_done[st] : nullptr, parity, TWO,
-                                       TWO ? &peer_ready[st] : nullptr, parity, true, abort_flag) && ok;
+                ok = mbar_wait_all(&b_full[st], parity, false, sparse ? &conv_done[st] : nullptr, parity, TWO,
+                                   TWO ? &peer_ready[st] : nullptr, parity, true, abort_flag) && ok;
                 fence_after_sync();
-                // ask about the next stage now: the answer comes back while this stage's MMAs are issued
-                pre = 0;
-                if (it + 1 < n_total) {
-                    const int st1 = (it + 1) % kPStages;
-                    const uint32_t par1 = ((it + 1) / kPStages) & 1;
-                    pre = mbar_try(&b_full[st1], par1, false);
-                    if (it + 1 < p.n1) pre &= mbar_try(&conv_done[st1], par1, TWO);
-                    if (TWO) pre &= mbar_try(&peer_ready[st1], par1, true);
-                }
                 const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
                 const uint32_t a_addr = b_addr + kBTile;
                 PSTAMP(3, it);
