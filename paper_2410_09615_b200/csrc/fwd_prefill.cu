@@ -238,6 +238,17 @@ __device__ __forceinline__ uint32_t mbar_try(uint64_t* bar, uint32_t parity, boo
                      : "=r"(done) : "r"(s32(bar)), "r"(parity) : "memory");
     return done;
 }
+// The same question without waiting (try_wait holds the thread for a while when the answer is no).
+__device__ __forceinline__ uint32_t mbar_test(uint64_t* bar, uint32_t parity, bool cluster) {
+    uint32_t done;
+    if (cluster)
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(s32(bar)), "r"(parity) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(s32(bar)), "r"(parity) : "memory");
+    return done;
+}
 // Bounded wait for several barriers at once.  A try_wait takes about 200 cycles to answer even when
 // the phase is long complete, so waits that follow each other are asked together, not in turn.
 __device__ __forceinline__ bool mbar_wait_all(uint64_t* b0, uint32_t p0, bool c0, uint64_t* b1, uint32_t p1, bool c1,
@@ -416,14 +427,26 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             }
         } else if (elect_one()) {
             constexpr uint32_t idesc = idesc_bf16(TWO ? 2 * kPM : kPM, N);
+            uint32_t pre = 0;       // the coming stage was found ready by an early test
             for (int it = 0; it < n_total; ++it) {
                 const int st = it % kPStages;
                 const uint32_t parity = (it / kPStages) & 1;
                 const bool sparse = it < p.n1;
                 // token tile landed; converters done (in a pair: both CTAs', reported here); the other CTA's loads landed
-                ok = mbar_wait_all(&b_full[st], parity, false, sparse ? &conv_done[st] : nullptr, parity, TWO,
-                                   TWO ? &peer_ready[st] : nullptr, parity, true, abort_flag) && ok;
+                if (!pre)
+                    ok = mbar_wait_all(&b_full[st], parity, false, sparse ? &conv_done[st] : nullptr, parity, TWO,
+                                       TWO ? &peer_ready[st] : nullptr, parity, true, abort_flag) && ok;
                 fence_after_sync();
+                // ask about the next stage now, without waiting: the answer comes back while this stage's
+                // MMAs are issued, and in steady state it is yes
+                pre = 0;
+                if (it + 1 < n_total) {
+                    const int st1 = (it + 1) % kPStages;
+                    const uint32_t par1 = ((it + 1) / kPStages) & 1;
+                    pre = mbar_test(&b_full[st1], par1, false);
+                    if (it + 1 < p.n1) pre &= mbar_test(&conv_done[st1], par1, TWO);
+                    if (TWO) pre &= mbar_test(&peer_ready[st1], par1, true);
+                }
                 const uint32_t b_addr = s32(stages + (size_t)st * kStageBytes);
                 const uint32_t a_addr = b_addr + kBTile;
                 PSTAMP(3, it);
