@@ -36,11 +36,13 @@
 // empty / pk_empty (tcgen05.commit: the MMAs that read the stage are complete; converters
 // done with a packed slot), acc_full.
 // Measured on B200 and built into the loops below: a barrier operation is served per thread
-// (a warp-wide try_wait or 32 arrivals cost 32 times one), a lane left at a warp barrier
-// while another lane of its warp spins costs some hundred nanoseconds per iteration, and one
-// MMA costs at least the 128 cycles its 128-row A operand takes to load, whatever N.
-// With one CTA per tile the loop is bound by shared-memory bandwidth: per stage TMA writes
-// 35 KB, the tensor core reads 40 KB, the converters move 11 KB.
+// (a warp-wide try_wait or 32 arrivals cost 32 times one); the answer of a try_wait takes about
+// 200 cycles even when the phase is long complete, so waits that follow each other are asked
+// together; a lane left at a warp barrier while another lane of its warp spins costs some hundred
+// nanoseconds per iteration; one MMA costs at least the 128 cycles its 128-row A operand takes to
+// load, whatever N.  With one CTA per tile a stage takes about 320 ns: its slot's next token tile
+// is requested ~600 ns after the MMAs that free the slot were issued and lands ~900 ns later, over
+// the 5 stages that fit in shared memory.
 // Every wait is bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on.
 #include <cuda.h>
 #include "common.cuh"
