@@ -249,6 +249,10 @@ __device__ __forceinline__ Share make_share(const DecodeParams& p, int cta) {
 }
 
 // Sum the consumer warps' partial tiles (fragment order) through shared memory.
+// Cross-warp sums go through a ring of buffers in shared memory: a buffer is written again only
+// two consumer barriers after it was read (the weight phase uses two buffers per barrier).
+constexpr int kRedBufs = 4;
+
 template <int NT>
 __device__ __forceinline__ float block_tile_sum(float* red, const float (&acc)[NT][4], bool active, int n_active) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -263,6 +267,28 @@ __device__ __forceinline__ float block_tile_sum(float* red, const float (&acc)[N
     float sum = 0.f;
     if (threadIdx.x < frag)
         for (int w = 0; w < n_active; ++w) sum += red[w * frag + threadIdx.x];
+    return sum;
+}
+
+// The same for two tiles with one barrier: a barrier and its skew cost as much as a tile's MMAs.
+template <int NT>
+__device__ __forceinline__ float2 block_tile_sum2(float* red0, float* red1, const float (&acc0)[NT][4],
+                                                  const float (&acc1)[NT][4], bool active, int n_active) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int frag = NT * 128;
+    if (active) {
+#pragma unroll
+        for (int h = 0; h < NT; ++h)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                red0[warp * frag + (h * 4 + q) * 32 + lane] = acc0[h][q];
+                red1[warp * frag + (h * 4 + q) * 32 + lane] = acc1[h][q];
+            }
+    }
+    consumer_sync();
+    float2 sum = make_float2(0.f, 0.f);
+    if (threadIdx.x < frag)
+        for (int w = 0; w < n_active; ++w) { sum.x += red0[w * frag + threadIdx.x]; sum.y += red1[w * frag + threadIdx.x]; }
     return sum;
 }
 
@@ -319,7 +345,7 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
     unsigned char* xs = ring + (size_t)p.n_slots * kSlotBytes;
     __nv_bfloat16* Ts = reinterpret_cast<__nv_bfloat16*>(xs + 32 * x_sub);
     float* red_base = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(Ts) + (size_t)NT * 8 * p.r_pad * 2);
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(red_base + 2 * kConsumerWarps * frag);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(red_base + kRedBufs * kConsumerWarps * frag);
     uint64_t* empty_bar = full_bar + kMaxSlots;
     uint64_t* x_bar = empty_bar + kMaxSlots;
 
@@ -447,7 +473,7 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
     };
     auto next_red = [&]() -> float* {
         float* r = red_base + red_buf * kConsumerWarps * frag;
-        red_buf ^= 1;
+        red_buf = (red_buf + 1) & (kRedBufs - 1);
         return r;
     };
     // the number of this call on this workspace (read before any CTA of the call can have left)
@@ -531,52 +557,66 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
         const uint32_t byte_sel = (uint32_t)t * 0x1111u + 0x4400u;   // bytes {t, t, 4+t, 4+t}
         const uint32_t meta_sel = (t & 1) ? 0x7632u : 0x5410u;
         STAMP(4);
-        for (int tile = sh.w_begin; tile < sh.w_begin + sh.w_count; ++tile) {
-            const unsigned char* base = wait_full();
-            if (tile == sh.w_begin) STAMP(5);
-            if (tile == sh.w_begin + 1) STAMP(6);
-            float acc[NT][4];
+        // Tiles go two at a time: both are multiplied, then one cross-warp sum serves both.
+        const int w_end = sh.w_begin + sh.w_count;
+        for (int tile = sh.w_begin; tile < w_end; tile += 2) {
+            const bool two = tile + 1 < w_end;
+            float acc2[2][NT][4];
 #pragma unroll
-            for (int h = 0; h < NT; ++h)
+            for (int u = 0; u < 2; ++u)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
-            if (w_active) {
-                // value bytes of block `warp`: tile warp/2, bytes 64 (warp % 2) .. +64 of the row;
-                // index bytes: tile 4 + warp/4, bytes 32 (warp % 4) .. +32
-                const unsigned char* vsub = base + (warp >> 1) * kSubTile;
-                const unsigned char* msub = base + (4 + (warp >> 2)) * kSubTile;
-                const int vo = (warp & 1) * 64, mo = (warp & 3) * 32 + 16 * (t >> 1);
-                uint4 v0[4], v1[4];
+                for (int h = 0; h < NT; ++h)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    v0[i] = lds128(vsub + swz(g, vo + 16 * i));
-                    v1[i] = lds128(vsub + swz(g + 8, vo + 16 * i));
-                }
-                // index words of steps 0-3 come from threads 0,1 of a quad, of steps 4-7 from threads 2,3
-                const uint4 m0 = lds128(msub + swz(g, mo));
-                const uint4 m1 = lds128(msub + swz(g + 8, mo));
+                    for (int e = 0; e < 4; ++e) acc2[u][h][e] = 0.f;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    uint32_t a[4];
-                    a[0] = decode_group(word_of(v0[j >> 1], (2 * j) & 3), byte_sel);
-                    a[1] = decode_group(word_of(v1[j >> 1], (2 * j) & 3), byte_sel);
-                    a[2] = decode_group(word_of(v0[j >> 1], (2 * j + 1) & 3), byte_sel);
-                    a[3] = decode_group(word_of(v1[j >> 1], (2 * j + 1) & 3), byte_sel);
-                    // metadata word: low half = row g, high half = row g+8, 16 columns each
-                    uint32_t e;
-                    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(e)
-                        : "r"(word_of(m0, j & 3)), "r"(word_of(m1, j & 3)), "r"(meta_sel));
+            for (int u = 0; u < 2; ++u) {
+                if (u == 1 && !two) break;
+                float (&acc)[NT][4] = acc2[u];
+                const unsigned char* base = wait_full();
+                if (tile + u == sh.w_begin) STAMP(5);
+                if (tile + u == sh.w_begin + 1) STAMP(6);
+                if (w_active) {
+                    // value bytes of block `warp`: tile warp/2, bytes 64 (warp % 2) .. +64 of the row;
+                    // index bytes: tile 4 + warp/4, bytes 32 (warp % 4) .. +32
+                    const unsigned char* vsub = base + (warp >> 1) * kSubTile;
+                    const unsigned char* msub = base + (4 + (warp >> 2)) * kSubTile;
+                    const int vo = (warp & 1) * 64, mo = (warp & 3) * 32 + 16 * (t >> 1);
+                    uint4 v0[4], v1[4];
 #pragma unroll
-                    for (int h = 0; h < NT; ++h) {
-                        if (j < 4) mma_sp_16832<0>(acc[h], a, xf[j][h], e);
-                        else       mma_sp_16832<1>(acc[h], a, xf[j][h], e);
+                    for (int i = 0; i < 4; ++i) {
+                        v0[i] = lds128(vsub + swz(g, vo + 16 * i));
+                        v1[i] = lds128(vsub + swz(g + 8, vo + 16 * i));
+                    }
+                    // index words of steps 0-3 come from threads 0,1 of a quad, of steps 4-7 from threads 2,3
+                    const uint4 m0 = lds128(msub + swz(g, mo));
+                    const uint4 m1 = lds128(msub + swz(g + 8, mo));
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        uint32_t a[4];
+                        a[0] = decode_group(word_of(v0[j >> 1], (2 * j) & 3), byte_sel);
+                        a[1] = decode_group(word_of(v1[j >> 1], (2 * j) & 3), byte_sel);
+                        a[2] = decode_group(word_of(v0[j >> 1], (2 * j + 1) & 3), byte_sel);
+                        a[3] = decode_group(word_of(v1[j >> 1], (2 * j + 1) & 3), byte_sel);
+                        // metadata word: low half = row g, high half = row g+8, 16 columns each
+                        uint32_t e;
+                        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(e)
+                            : "r"(word_of(m0, j & 3)), "r"(word_of(m1, j & 3)), "r"(meta_sel));
+#pragma unroll
+                        for (int h = 0; h < NT; ++h) {
+                            if (j < 4) mma_sp_16832<0>(acc[h], a, xf[j][h], e);
+                            else       mma_sp_16832<1>(acc[h], a, xf[j][h], e);
+                        }
                     }
                 }
+                release();
             }
-            release();
-            const float sum = block_tile_sum<NT>(next_red(), acc, w_active, sh.nb);
-            if (threadIdx.x < frag)
-                st_gpu(p.Ppart + ((size_t)sh.ks * tilesW + tile) * frag + threadIdx.x, slot_bits(sum));
+            float* r0 = next_red();
+            float* r1 = next_red();
+            const float2 sum = block_tile_sum2<NT>(r0, r1, acc2[0], acc2[1], w_active, sh.nb);
+            if (threadIdx.x < frag) {
+                st_gpu(p.Ppart + ((size_t)sh.ks * tilesW + tile) * frag + threadIdx.x, slot_bits(sum.x));
+                if (two) st_gpu(p.Ppart + ((size_t)sh.ks * tilesW + tile + 1) * frag + threadIdx.x, slot_bits(sum.y));
+            }
         }
     }
 
@@ -700,7 +740,7 @@ static bool make_plan(int b, int d_out, int d_in, int r, int ctas, DecodePlan* p
     pl->r_pad = pad_rank(r);
     const size_t frag = (size_t)pl->nt * 128 * sizeof(float);
     const size_t fixed = 1024 /* alignment slack */ + 32 * (size_t)pl->nt * 8 * 128 /* X slice */ +
-                         (size_t)pl->nt * 8 * pl->r_pad * 2 + 2 * kConsumerWarps * frag + (2 * kMaxSlots + 2) * 8 + 64;
+                         (size_t)pl->nt * 8 * pl->r_pad * 2 + kRedBufs * kConsumerWarps * frag + (2 * kMaxSlots + 2) * 8 + 64;
     if (fixed + 3 * (size_t)kSlotBytes > kSmemBudget) return false;
     int n = (int)((kSmemBudget - fixed) / kSlotBytes);
     pl->n_slots = n > kMaxSlots ? kMaxSlots : n;
