@@ -369,11 +369,6 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
         // ============================ producer warp ============================
         uint32_t it = 0;
         bool ok = true;
-        // ---- the CTA's slice of the activations: 4 tiles of 64 columns per block, rows >= b read as zero
-        if (sh.grp >= 0) {
-            if (lane == 0) mbar_arrive_expect_tx(x_bar, (uint32_t)(sh.nb * 4 * x_sub));
-            if (lane < sh.nb * 4) tma_tile(xs + lane * x_sub, &tmX, sh.blk_begin * 256 + 64 * lane, 0, x_bar);
-        }
         // Returns the slot once it is free; lane 0 arms its full barrier.  The whole warp waits:
         // a single waiting lane followed by a warp barrier costs some hundred nanoseconds per
         // tile.  (A tile may land before lane 0 has armed the barrier; the phase cannot
@@ -480,6 +475,13 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
     uint32_t call = 0;
     if (p.r > 0) call = (uint32_t)(ld_gpu64(p.departures) / (unsigned)n_ctas) + 1u;
 
+    // The CTA's slice of the activations: 4 tiles of 64 columns per block, rows >= b read as zero.
+    // Consumer warp 0 requests it (a warp's first tile request takes most of a microsecond; the
+    // producer warp spends that time on the first R chunk instead).
+    if (warp == 0 && sh.grp >= 0) {
+        if (lane == 0) mbar_arrive_expect_tx(x_bar, (uint32_t)(sh.nb * 4 * x_sub));
+        if (lane < sh.nb * 4) tma_tile(xs + lane * x_sub, &tmX, sh.blk_begin * 256 + 64 * lane, 0, x_bar);
+    }
     if (sh.grp >= 0) ok = mbar_wait(x_bar, 0) && ok;       // the activation slice is in shared memory
     STAMP(1);
 
