@@ -538,47 +538,22 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
             }
             if ((threadIdx.x & 127) == 0) PSTAMP(2, it);
         }
-        // ---- epilogue.  TMEM gives a thread one output row and 32 tokens at a time; global memory
-        // wants rows contiguous.  Each half of the converter warps (128 threads, half of the token
-        // columns) turns 32-token chunks through shared memory (the stage ring is idle by now) and
-        // stores eight rows of one token per thread: 16-byte stores instead of 2-byte ones.
+        // ---- epilogue: thread = output row, TMEM columns = tokens; the two halves split the columns
         ok = mbar_wait(acc_full, 0, abort_flag) && ok;
         fence_after_sync();
         if (threadIdx.x == 0) PSTAMP(5, 46);
-        float* turn = reinterpret_cast<float*>(stages) + half * (2 * 32 * kPM);     // two 16 KB buffers per half
-        const int tl = threadIdx.x & 127;
-        const int rc = (tl & 15) * 8;                 // first of the eight rows this thread stores
-        int chunk = 0;
+        const int orow = m0 + row;
 #pragma unroll 1
-        for (int c0 = half * (N / 2); c0 < (half + 1) * (N / 2); c0 += 32, ++chunk) {
+        for (int c0 = half * (N / 2); c0 < (half + 1) * (N / 2); c0 += 32) {
             uint32_t r[32];
             tmem_ld32(tmem_base + lane_base + c0, r);
-            float* buf = turn + (chunk & 1) * (32 * kPM);
+            if (orow < p.m_total) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) buf[c * kPM + row] = __uint_as_float(r[c]);
-            // the 128 threads of this half (the other half runs its own chunks)
-            if (half) asm volatile("bar.sync 2, 128;" ::: "memory");
-            else      asm volatile("bar.sync 1, 128;" ::: "memory");
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int t_local = (tl >> 4) + 8 * k;
-                const int token = n0 + c0 + t_local;
-                const float4 lo = *reinterpret_cast<const float4*>(buf + t_local * kPM + rc);
-                const float4 hi = *reinterpret_cast<const float4*>(buf + t_local * kPM + rc + 4);
-                if (token < p.b && m0 + rc < p.m_total) {
-                    if (PRE && p.part) {
-                        float* dst = p.part + ((size_t)blockIdx.z * p.b + token) * p.ldo + m0 + rc;
-                        *reinterpret_cast<float4*>(dst) = lo;
-                        *reinterpret_cast<float4*>(dst + 4) = hi;
-                    } else {
-                        __nv_bfloat162 v0 = __floats2bfloat162_rn(p.scale * lo.x, p.scale * lo.y);
-                        __nv_bfloat162 v1 = __floats2bfloat162_rn(p.scale * lo.z, p.scale * lo.w);
-                        __nv_bfloat162 v2 = __floats2bfloat162_rn(p.scale * hi.x, p.scale * hi.y);
-                        __nv_bfloat162 v3 = __floats2bfloat162_rn(p.scale * hi.z, p.scale * hi.w);
-                        uint4 o;
-                        o.x = *reinterpret_cast<uint32_t*>(&v0); o.y = *reinterpret_cast<uint32_t*>(&v1);
-                        o.z = *reinterpret_cast<uint32_t*>(&v2); o.w = *reinterpret_cast<uint32_t*>(&v3);
-                        *reinterpret_cast<uint4*>(p.out + (size_t)token * p.ldo + m0 + rc) = o;
+                for (int c = 0; c < 32; ++c) {
+                    const int token = n0 + c0 + c;
+                    if (token < p.b) {
+                        if (PRE && p.part) p.part[((size_t)blockIdx.z * p.b + token) * p.ldo + orow] = __uint_as_float(r[c]);
+                        else p.out[(size_t)token * p.ldo + orow] = __float2bfloat16_rn(p.scale * __uint_as_float(r[c]));
                     }
                 }
             }
