@@ -199,7 +199,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2410_09615_b200 import binding as K
-    from paper_2410_09615_b200 import build
+    from paper_2410_09615_b200 import build, replicas
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -314,12 +314,9 @@ def run_ours(args):
     elapsed_ms = e0.elapsed_time(e1)
     if K.read_status(status) != 0:
         raise RuntimeError(f"device status {K.read_status(status):#x}")
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = replicas.max_over_ranks(elapsed_ms, dev)
     ms_per_step = elapsed_ms / args.steps
-    value = 1e3 * ms_per_step / (CALLS_PER_STEP * world)
+    value = replicas.whole_job_us_per_call(ms_per_step, CALLS_PER_STEP, world)
 
     # ---- roofline of the dominant kernel over the timed region
     step_bytes = sum(algorithmic_bytes(ly["d_in"], ly["d_out"], ly["r"], b) for ly, b, _ in step_calls)
@@ -478,7 +475,7 @@ def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, wor
     and Y goes back to pinned host memory inside every call."""
     import ctypes
     import torch
-    import torch.distributed as dist
+    from paper_2410_09615_b200 import replicas
     P = ctypes.c_void_p
     host = {}
     for ly in layers:
@@ -511,11 +508,8 @@ def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, wor
     e1.record(stream)
     barrier()
     ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return {"value": 1e3 * ms / steps / (CALLS_PER_STEP * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    ms = replicas.max_over_ranks(ms, "cuda")
+    return {"value": replicas.whole_job_us_per_call(ms / steps, CALLS_PER_STEP, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "steps": steps, "api": "slim_linear_fwd_host"}
 
 
