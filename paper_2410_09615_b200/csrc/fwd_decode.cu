@@ -16,8 +16,8 @@
 // (cp.async.bulk.tensor.2d, 128-byte rows, 128-byte swizzle, mbarrier
 // completion): the CTA's slice of the activations once, then a ring of 16 KB
 // slots for the streamed matrices.  The lanes of a ninth, producer warp issue
-// the tiles of a chunk in parallel (one thread can start only ~6 TMA loads per
-// microsecond); the eight consumer warps read MMA fragments from shared memory.
+// the tiles of a chunk in parallel (a thread is held about 160 cycles by every
+// tile request it starts); the eight consumer warps read MMA fragments from shared memory.
 //
 // Work split.  d_in is cut into 256-column blocks and into k-slices of <= 8
 // blocks; a CTA belongs to one slice, one block per consumer warp.  Each CTA
