@@ -41,12 +41,12 @@ WORKLOAD = "llama2_7b_decode_layer_set"
 BATCHES = (1, 16)
 SHAPES = inputs.LLAMA2_SHAPES["7b"]            # (name, d_in, d_out, count per block)
 CALLS_PER_STEP = sum(c for *_x, c in SHAPES) * len(BATCHES)
-HBM_FALLBACK_GBS = 6650.0                      # earlier measurement on this machine
+HBM_FALLBACK_GBS = 6650.0                      # an earlier copy-bandwidth measurement on B200
 NOMINAL_HBM_GBS = 8000.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch divided by
 # the call's algorithmic bytes, from an ncu capture of the (4096, 11008, 416, 16)
-# case (profiles/decode_kernel_llama2_7b_decode_layer_set.md): 29.81 MB / 29.96 MB.
+# case (its summary is kept with the other profiler summaries): 29.80 MB / 29.96 MB.
 # Traffic grows in proportion to the bytes streamed, so the bench scales it to its
 # own launches.  Set to None whenever decode_kernel changes after the capture.
 NCU_TRAFFIC_RATIO = 0.995
