@@ -68,3 +68,15 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libslim.so")
     with pytest.raises(binding.SlimError):
         binding.lib()
+
+
+def test_header_enums_match_the_binding():
+    """Every SLIM_ERR_* / SLIM_KERNEL_* value of the header has the same value in the binding."""
+    import re
+    text = open(os.path.join(ROOT, "include", "slim.h")).read()
+    pairs = re.findall(r"\b(SLIM_(?:ERR|KERNEL)_[A-Z_]+|SLIM_OK)\s*=\s*(\d+)", text)
+    assert len(pairs) >= 12
+    for name, value in pairs:
+        py = name if name.startswith("SLIM_ERR") or name == "SLIM_OK" else name.replace("SLIM_", "")
+        assert hasattr(binding, py), f"{name} missing from the binding"
+        assert getattr(binding, py) == int(value), name
