@@ -47,6 +47,8 @@ def _load():
         lib.oracle_pack.restype = ctypes.c_int
         lib.oracle_unpack.argtypes = [P, P, ctypes.c_int, ctypes.c_int, P, P]
         lib.oracle_unpack.restype = ctypes.c_int
+        lib.oracle_repack_tiled.argtypes = [P, P, ctypes.c_int, ctypes.c_int, P]
+        lib.oracle_repack_tiled.restype = ctypes.c_int
         lib.oracle_linear_fwd.argtypes = [P, ctypes.c_int, P, P, ctypes.c_float, P, P, ctypes.c_int,
                                           ctypes.c_int, ctypes.c_int, P, ctypes.c_int, P]
         lib.oracle_linear_fwd.restype = ctypes.c_int
@@ -96,6 +98,17 @@ def unpack(vals: np.ndarray, meta: np.ndarray):
     if rc != OK:
         raise OracleError(rc)
     return codes, mask
+
+
+def repack_tiled(vals: np.ndarray, meta: np.ndarray) -> np.ndarray:
+    """(vals, meta) -> the decode-tiled copy, uint8 [d_out * d_in * 3 / 8]."""
+    vals, meta = _c(vals, np.uint8), _c(meta, np.uint8)
+    d_out, d_in = vals.shape[0], vals.shape[1] * 4
+    out = np.zeros(d_out * d_in * 3 // 8, np.uint8)
+    rc = _load().oracle_repack_tiled(_p(vals), _p(meta), d_out, d_in, _p(out))
+    if rc != OK:
+        raise OracleError(rc)
+    return out
 
 
 def linear_fwd(X, vals, meta, s, L, R, rows=None) -> np.ndarray:

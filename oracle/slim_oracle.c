@@ -152,6 +152,70 @@ int oracle_unpack(const uint8_t *vals, const uint8_t *meta, int d_out, int d_in,
 }
 
 /*
+ * Decode-tiled copy of a packed weight: the same nibbles and position indices as
+ * (vals, meta), re-ordered so that a 32-lane group that multiplies a 16-row x
+ * 32-column piece reads its share as consecutive 32-bit words.  Like the packed
+ * format itself this layout is the project's own (the paper leaves storage to a
+ * third-party kernel, Sec. 4 "Speedup"); nothing is computed, bytes only move.
+ *
+ * d_out % 16 == 0, d_in % 256 == 0.  The matrix is cut into tiles of 16 rows and
+ * blocks of 256 columns; (tile, block) occupies 1536 bytes at
+ * ((tile * d_in/256) + block) * 1536.  Inside a block, a "step" j = 0..7 is 32
+ * columns (8 groups of four), a "lane" is (g, t) = (lane / 4, lane % 4):
+ *   value words, bytes [0, 1024):  word (j, lane) at (j / 4) * 512 + lane * 16 + (j % 4) * 4.
+ *     It holds four value bytes B_i, i = 0..3, taken from row 16 tile + g + 8 (i % 2),
+ *     group 8 j + 4 (i / 2) + t of the block: the low nibble of B_i sits at bits
+ *     [4 i, 4 i + 3], the high nibble at bits [16 + 4 i, 16 + 4 i + 3].
+ *   index words, bytes [1024, 1536):  word (lane, jj), jj = 0..3, at 1024 + lane * 16 + jj * 4,
+ *     belongs to step j = 4 (t / 2) + jj.  Bits 0-15 are the index bytes of row
+ *     16 tile + g for 16 of the step's 32 columns (the first 16 when t is even, the
+ *     last 16 when t is odd), as a little-endian 16-bit number; bits 16-31 the same
+ *     for row 16 tile + g + 8.
+ * Words are stored little-endian.  out: d_out * d_in * 3 / 8 bytes.
+ */
+int oracle_repack_tiled(const uint8_t *vals, const uint8_t *meta, int d_out, int d_in, uint8_t *out)
+{
+    if (!vals || !meta || !out || d_out < 16 || d_in < 256 || d_out % 16 != 0 || d_in % 256 != 0)
+        return ORACLE_BAD_ARG;
+    const int nblk = d_in / 256, tiles = d_out / 16;
+    const size_t vrow = (size_t)d_in / 4, mrow = (size_t)d_in / 8;
+    for (int tile = 0; tile < tiles; ++tile) {
+        for (int blk = 0; blk < nblk; ++blk) {
+            uint8_t *base = out + ((size_t)tile * nblk + blk) * 1536;
+            for (int j = 0; j < 8; ++j) {
+                for (int lane = 0; lane < 32; ++lane) {
+                    const int g = lane / 4, t = lane % 4;
+                    uint32_t w = 0;
+                    for (int i = 0; i < 4; ++i) {
+                        const int row = 16 * tile + g + 8 * (i % 2);
+                        const int group = 64 * blk + 8 * j + 4 * (i / 2) + t;
+                        const uint32_t B = vals[(size_t)row * vrow + group];
+                        w |= (B & 0xFu) << (4 * i);
+                        w |= (B >> 4) << (16 + 4 * i);
+                    }
+                    uint8_t *dst = base + (j / 4) * 512 + lane * 16 + (j % 4) * 4;
+                    dst[0] = (uint8_t)w; dst[1] = (uint8_t)(w >> 8); dst[2] = (uint8_t)(w >> 16); dst[3] = (uint8_t)(w >> 24);
+                }
+            }
+            for (int lane = 0; lane < 32; ++lane) {
+                const int g = lane / 4, t = lane % 4;
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = 4 * (t / 2) + jj;
+                    uint8_t *dst = base + 1024 + lane * 16 + jj * 4;
+                    for (int up = 0; up < 2; ++up) {
+                        const int row = 16 * tile + g + 8 * up;
+                        const uint8_t *mb = meta + (size_t)row * mrow + 32 * blk + 4 * j + 2 * (t % 2);
+                        dst[2 * up] = mb[0];
+                        dst[2 * up + 1] = mb[1];
+                    }
+                }
+            }
+        }
+    }
+    return ORACLE_OK;
+}
+
+/*
  * Factored forward  Y = X (s Q)^T + (X R^T) L^T  in fp64, dense loops over the
  * whole contraction axis (the zeros of the 2:4 pattern are multiplied, not
  * skipped), no intermediate rounding  [Sec. 2 Eq. 1; Sec. 3.2; App. Rank

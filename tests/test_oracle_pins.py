@@ -218,3 +218,86 @@ def test_flop_reduction_matches_printed_table():
         d, n, dff, V, rr, printed = int(d), int(n), int(dff), int(V), float(rr), float(printed)
         got = oracle.flop_reduction(d, n, dff / d, V, rr)
         assert abs(got - printed) <= 0.005 + 1e-9, (got, printed)
+
+
+# ---------------------------------------------------------------- decode-tiled copy
+def test_repack_tiled_bytes_by_hand():
+    """One value byte and one index byte placed by hand arithmetic.
+    Row 9 = lane row g = 1, upper half of the tile; group 5 of the row = step 0,
+    second half of the step (4 + t with t = 1): value word of lane 4*1 + 1 = 5, step 0,
+    slot i = 3 (upper row, second half): low nibble at bits 12-15, high nibble at bits 28-31.
+    Index byte 2 of row 9 = columns 16-23 of step 0: second half of the step, so the
+    word of lane (g = 1, t = 1) for step 0, upper row in bits 16-31."""
+    vals = np.zeros((16, 64), np.uint8)
+    meta = np.zeros((16, 32), np.uint8)
+    vals[9, 5] = 0xA3
+    meta[9, 2] = 0xE4
+    out = oracle.repack_tiled(vals, meta)
+    assert out.size == 1536
+    expect = np.zeros(1536, np.uint8)
+    expect[5 * 16 + 0: 5 * 16 + 4] = [0x00, 0x30, 0x00, 0xA0]           # 0xA0003000 little-endian
+    expect[1024 + 5 * 16 + 0: 1024 + 5 * 16 + 4] = [0x00, 0x00, 0xE4, 0x00]
+    assert np.array_equal(out, expect)
+    # a byte of the second half of the block (step 6 -> second 512 bytes, word 2 of the lane),
+    # lower row, first half of the step (t = 2): slot i = 0
+    vals[:] = 0
+    meta[:] = 0
+    vals[3, 8 * 6 + 2] = 0x7C
+    meta[3, 4 * 6 + 1] = 0x9D        # columns 8-15 of step 6: first half -> lane t even of steps 4-7: t = 2
+    out = oracle.repack_tiled(vals, meta)
+    expect = np.zeros(1536, np.uint8)
+    lane = 3 * 4 + 2
+    expect[512 + lane * 16 + 2 * 4: 512 + lane * 16 + 2 * 4 + 4] = [0x0C, 0x00, 0x07, 0x00]
+    expect[1024 + lane * 16 + 2 * 4: 1024 + lane * 16 + 2 * 4 + 4] = [0x00, 0x9D, 0x00, 0x00]
+    assert np.array_equal(out, expect)
+
+
+def dense_from_tiled(buf, d_out, d_in):
+    """Read a decode-tiled buffer the way its consumer does (per lane and step: four
+    value slots, index half-words from the lane that holds them) and rebuild the dense
+    code matrix.  Written from the layout's description, not from the oracle's loops."""
+    nblk = d_in // 256
+    words = buf.view("<u4").reshape(d_out // 16, nblk, 384)
+    dense = np.zeros((d_out, d_in), np.int64)
+    sext = lambda n: n - 16 if n >= 8 else n
+    for tile in range(d_out // 16):
+        for blk in range(nblk):
+            wv = words[tile, blk, :256].reshape(2, 32, 4)       # [half of the steps][lane][word]
+            wm = words[tile, blk, 256:].reshape(32, 4)          # [lane][word]
+            for j in range(8):
+                for lane in range(32):
+                    g, t = divmod(lane, 4)
+                    w = int(wv[j // 4, lane, j % 4])
+                    for i in range(4):
+                        up, second = i % 2, i // 2
+                        lo, hi = (w >> (4 * i)) & 15, (w >> (16 + 4 * i)) & 15
+                        # the index half-word of this half of the step lives in lane (g, 2 * (j // 4) + second)
+                        e = int(wm[g * 4 + 2 * (j // 4) + second, j % 4])
+                        half = (e >> (16 * up)) & 0xFFFF
+                        nib = (half >> (4 * t)) & 15
+                        p0, p1 = nib & 3, nib >> 2
+                        col = 256 * blk + 32 * j + 16 * second + 4 * t
+                        row = 16 * tile + g + 8 * up
+                        dense[row, col + p0] += sext(lo)
+                        dense[row, col + p1] += sext(hi)
+    return dense
+
+
+def test_repack_tiled_keeps_every_code_and_position():
+    rng = np.random.default_rng(5)
+    d_out, d_in = 48, 768
+    codes = rng.integers(-8, 8, size=(d_out, d_in)).astype(np.int8)
+    mask = inputs.top2_mask(rng.standard_normal((d_out, d_in)).astype(np.float32))
+    vals, meta = oracle.pack(codes, mask)
+    tiled = oracle.repack_tiled(vals, meta)
+    assert tiled.size == d_out * d_in * 3 // 8
+    assert np.array_equal(dense_from_tiled(tiled, d_out, d_in), codes.astype(np.int64) * mask)
+    # a permutation of the input bits: same population of set bits
+    assert int(np.unpackbits(tiled).sum()) == int(np.unpackbits(vals).sum() + np.unpackbits(meta).sum())
+
+
+def test_repack_tiled_rejects_shapes_it_cannot_tile():
+    with pytest.raises(oracle.OracleError):
+        oracle.repack_tiled(np.zeros((8, 64), np.uint8), np.zeros((8, 32), np.uint8))
+    with pytest.raises(oracle.OracleError):
+        oracle.repack_tiled(np.zeros((16, 32), np.uint8), np.zeros((16, 16), np.uint8))
