@@ -53,7 +53,7 @@ extern "C" {
 
 typedef enum {
     SLIM_OK = 0,
-    SLIM_ERR_INVALID_ARG = 1,        /* null / misaligned pointer, b < 1, negative size */
+    SLIM_ERR_INVALID_ARG = 1,        /* null / misaligned pointer, b < 1, negative size, scale not finite */
     SLIM_ERR_UNSUPPORTED_SHAPE = 2,  /* d_in % 64, d_out % 16 or r % 16 not zero */
     SLIM_ERR_BAD_MASK = 3,           /* device: more than two kept values in a group */
     SLIM_ERR_CODE_RANGE = 4,         /* device: kept code outside [-8, 7] */
@@ -88,8 +88,9 @@ slim_status_t slim_pack(const int8_t* codes, const uint8_t* mask, int d_out, int
                         uint8_t* vals, uint8_t* meta, uint32_t* status_dev, void* cuda_stream);
 
 /*
- * Inverse of slim_pack: dense int8 codes (0 where nothing is stored) and a mask
- * holding 1 at the two stored positions of every group.  `mask` may be NULL.
+ * Inverse of slim_pack (reads the packed format described at the top of this file; 2:4
+ * pattern: Sec. 1; 4-bit codes: Sec. 3.1 Eq. 2): dense int8 codes (0 where nothing is
+ * stored) and a mask holding 1 at the two stored positions of every group.  `mask` may be NULL.
  */
 slim_status_t slim_unpack(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in,
                           int8_t* codes, uint8_t* mask, void* cuda_stream);
@@ -99,7 +100,8 @@ slim_status_t slim_unpack(const uint8_t* vals, const uint8_t* meta, int d_out, i
  * partial sums, the adapter intermediate T = X R^T, and a call counter).
  * Returns 0 for illegal arguments.  A workspace must be initialised once with
  * slim_workspace_reset before its first use (counter zero, every hand-over slot
- * marked empty); each call leaves it ready for the next one unless it reported
+ * marked empty); each call, whichever kernel it runs, leaves it ready for the next
+ * one, of any shape the workspace is large enough for, unless it reported
  * SLIM_ERR_TIMEOUT, after which it must be reset again.  Calls that share a
  * workspace must not overlap on the GPU.
  */
@@ -117,9 +119,13 @@ slim_status_t slim_workspace_reset(void* workspace, size_t workspace_bytes, void
  * be rounded once to bf16; Y is rounded to bf16 (nearest even).
  *   X [b, d_in] bf16, vals/meta as produced by slim_pack, s fp32 scale,
  *   L [d_out, r] bf16, R [r, d_in] bf16 (both NULL iff r == 0), Y [b, d_out] bf16 (out).
- * Shape rules: b >= 1, d_in % 64 == 0, d_out % 16 == 0, r % 16 == 0.
- * The kernel is chosen from b: the streaming decode kernel for b <= 16, the
- * tcgen05 prefill kernel above.
+ * Shape rules: b >= 1, d_in % 64 == 0, d_out % 16 == 0, r % 16 == 0; s must be finite
+ * (NaN or infinity: SLIM_ERR_INVALID_ARG).
+ * The kernel is chosen from b and the shape: for b <= 16 the streaming decode kernel, which
+ * needs d_in % 256 == 0; above, the tcgen05 prefill kernel, which needs d_in % 128 == 0 and
+ * d_out % 128 == 0.  Every other legal shape runs on a plain CUDA-core kernel (one warp per
+ * output element) that is orders of magnitude slower: it exists for correctness, not speed.
+ * For b <= 16 the fast path is slim_linear_fwd_tiled on the decode-tiled copy of the weight.
  */
 slim_status_t slim_linear_fwd(const void* X, int b, const uint8_t* vals, const uint8_t* meta,
                               float s, const void* L, const void* R, int r, int d_out, int d_in,
@@ -131,6 +137,58 @@ slim_status_t slim_linear_fwd_ex(const void* X, int b, const uint8_t* vals, cons
                                  float s, const void* L, const void* R, int r, int d_out, int d_in,
                                  void* Y, void* workspace, size_t workspace_bytes,
                                  uint32_t* status_dev, void* cuda_stream, slim_kernel_t kernel);
+
+/*
+ * Decode-tiled copy of a packed weight, and the small-batch forward that reads it.
+ *
+ * At batch sizes 1-16 the layer is bound by the bytes of the weight it streams (Sec. 4
+ * "Speedup": small decode batches; Fig. 3: quantization contributes most of the speed-up),
+ * and the kernel then has about one instruction slot per three weight bytes.  The packed
+ * format above keeps a row's bytes together, which costs the streaming kernel a byte-pick per
+ * register and four-fold redundant shared-memory reads; the tiled copy holds the same nibbles
+ * and position indices (0.375 byte per weight, nothing is computed) in the order the sparse
+ * tensor-core instruction consumes them.  Like the packed format it is this library's own
+ * layout (the paper leaves storage to a third-party kernel).  Layout SLIM_LAYOUT_DECODE_TILED,
+ * for d_out % 16 == 0 and d_in % 256 == 0:
+ *   the matrix is cut into tiles of 16 rows and blocks of 256 columns; (tile, block) occupies
+ *   1536 bytes at ((tile * d_in / 256) + block) * 1536.  Inside a block a "step" j = 0..7 is 32
+ *   columns (8 groups of four) and a "lane" is (g, t) = (lane / 4, lane % 4), lane = 0..31.
+ *   Value words, bytes [0, 1024): the 32-bit word of (j, lane) sits at
+ *   (j / 4) * 512 + lane * 16 + (j % 4) * 4 and holds four value bytes B_i, i = 0..3, of row
+ *   16 tile + g + 8 (i % 2), group 8 j + 4 (i / 2) + t of the block: low nibble of B_i at bits
+ *   [4 i, 4 i + 3], high nibble at bits [16 + 4 i, 16 + 4 i + 3].
+ *   Index words, bytes [1024, 1536): the word of (lane, jj), jj = 0..3, sits at
+ *   1024 + lane * 16 + jj * 4 and belongs to step j = 4 (t / 2) + jj: bits 0-15 are the two
+ *   index bytes of row 16 tile + g for the step's first (t even) or last (t odd) 16 columns,
+ *   bits 16-31 the same for row 16 tile + g + 8.  Words are little-endian.
+ */
+#define SLIM_LAYOUT_DECODE_TILED 1
+
+/* Bytes of the tiled copy (d_out * d_in * 3 / 8), or 0 when the layout cannot hold the shape. */
+size_t slim_tiled_bytes(int d_out, int d_in, int layout_id);
+
+/*
+ * vals / meta as produced by slim_pack -> tiled_out (slim_tiled_bytes bytes, device, 16-byte
+ * aligned).  Integer-only and bit-exact; done once per layer.
+ */
+slim_status_t slim_repack_tiled(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in, int layout_id,
+                                void* tiled_out, void* cuda_stream);
+
+/*
+ * The layer forward of slim_linear_fwd (same equation, same rounding, same workspace rules) for
+ * 1 <= b <= 16 on a decode-tiled weight.  One kernel launch streams the weight, R and L exactly
+ * once.  Needs d_in % 256 == 0, d_out % 16 == 0, r % 16 == 0, r <= 3072; other problems return
+ * SLIM_ERR_UNSUPPORTED_SHAPE (use slim_linear_fwd on the packed weight).
+ */
+slim_status_t slim_linear_fwd_tiled(const void* X, int b, const void* tiled, int layout_id, float s, const void* L,
+                                    const void* R, int r, int d_out, int d_in, void* Y, void* workspace,
+                                    size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream);
+
+/* Host-buffer form of slim_linear_fwd_tiled (see slim_linear_fwd_host). */
+slim_status_t slim_linear_fwd_tiled_host(const void* X_host, int b, const void* tiled, int layout_id, float s,
+                                         const void* L, const void* R, int r, int d_out, int d_in, void* Y_host,
+                                         void* x_dev, void* y_dev, void* workspace, size_t workspace_bytes,
+                                         uint32_t* status_dev, void* cuda_stream);
 
 /*
  * Host-buffer form of the same operation, for callers whose activations live
@@ -179,6 +237,13 @@ slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* val
 slim_status_t slim_linear_fwd_noalloc(const void* X, int b, const uint8_t* vals, const uint8_t* meta,
                                       float s, const void* L, const void* R, int r, int d_out,
                                       int d_in, void* Y, uint32_t* status_dev, void* cuda_stream);
+
+/*
+ * Bytes of the built-in array slim_linear_fwd_noalloc would use for this problem (host-side
+ * arithmetic, no device needed); 0 when the entry point does not take the problem at all.  A
+ * value above SLIM_NOALLOC_SCRATCH_BYTES means the call would return SLIM_ERR_WORKSPACE.
+ */
+size_t slim_noalloc_scratch_needed(int b, int d_out, int d_in, int r);
 
 /* The kernel family slim_linear_fwd would pick for this problem. */
 slim_kernel_t slim_select_kernel(int b, int d_out, int d_in, int r);

@@ -22,6 +22,7 @@ KERNEL_AUTO, KERNEL_SIMPLE, KERNEL_DECODE, KERNEL_PREFILL, KERNEL_PREFILL_PAIR =
 KERNEL_NAMES = {KERNEL_AUTO: "auto", KERNEL_SIMPLE: "simple", KERNEL_DECODE: "decode", KERNEL_PREFILL: "prefill", KERNEL_PREFILL_PAIR: "prefill_pair"}
 WORKSPACE_SYNC_BYTES = 256
 NOALLOC_SCRATCH_BYTES = 16 << 20
+LAYOUT_DECODE_TILED = 1
 
 # every symbol include/slim.h declares, with (restype, argtypes)
 _P, _I, _F, _SZ = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
@@ -34,6 +35,11 @@ SIGNATURES = {
     "slim_linear_fwd_ex": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P, _I]),
     "slim_linear_fwd_host": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _P, _P, _SZ, _P, _P]),
     "slim_linear_fwd_noalloc": (_I, [_P, _I, _P, _P, _F, _P, _P, _I, _I, _I, _P, _P, _P]),
+    "slim_tiled_bytes": (_SZ, [_I, _I, _I]),
+    "slim_repack_tiled": (_I, [_P, _P, _I, _I, _I, _P, _P]),
+    "slim_linear_fwd_tiled": (_I, [_P, _I, _P, _I, _F, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P]),
+    "slim_linear_fwd_tiled_host": (_I, [_P, _I, _P, _I, _F, _P, _P, _I, _I, _I, _P, _P, _P, _P, _SZ, _P, _P]),
+    "slim_noalloc_scratch_needed": (_SZ, [_I, _I, _I, _I]),
     "slim_select_kernel": (_I, [_I, _I, _I, _I]),
     "slim_last_launch_count": (_I, []),
     "slim_strerror": (ctypes.c_char_p, [_I]),
@@ -137,6 +143,10 @@ def slim_workspace_bytes(b: int, d_out: int, d_in: int, r: int) -> int:
     return int(lib().slim_workspace_bytes(b, d_out, d_in, r))
 
 
+def slim_noalloc_scratch_needed(b: int, d_out: int, d_in: int, r: int) -> int:
+    return int(lib().slim_noalloc_scratch_needed(b, d_out, d_in, r))
+
+
 def slim_select_kernel(b: int, d_out: int, d_in: int, r: int) -> int:
     return int(lib().slim_select_kernel(b, d_out, d_in, r))
 
@@ -182,6 +192,58 @@ def slim_linear_fwd(X, vals, meta, s: float, L, R, Y=None, workspace=None, statu
               r, d_out, d_in, _ptr(Y), _ptr(workspace), workspace.numel(), _ptr(status), _stream(), int(kernel)),
            "slim_linear_fwd")
     return Y
+
+
+def slim_tiled_bytes(d_out: int, d_in: int, layout: int = LAYOUT_DECODE_TILED) -> int:
+    return int(lib().slim_tiled_bytes(d_out, d_in, layout))
+
+
+def slim_repack_tiled(vals: torch.Tensor, meta: torch.Tensor, layout: int = LAYOUT_DECODE_TILED, out=None) -> torch.Tensor:
+    """(vals, meta) of slim_pack -> the decode-tiled copy (uint8, one flat buffer)."""
+    _dev(vals, torch.uint8, "vals"), _dev(meta, torch.uint8, "meta")
+    d_out, d_in = vals.shape[0], vals.shape[1] * 4
+    n = slim_tiled_bytes(d_out, d_in, layout)
+    if n == 0 or tuple(meta.shape) != (d_out, d_in // 8):
+        raise SlimError(SLIM_ERR_UNSUPPORTED_SHAPE, "slim_repack_tiled", "shape cannot be tiled")
+    if out is None:
+        out = torch.empty(n, dtype=torch.uint8, device=vals.device)
+    _check(lib().slim_repack_tiled(_ptr(vals), _ptr(meta), d_out, d_in, layout, _ptr(out), _stream()), "slim_repack_tiled")
+    return out
+
+
+def slim_linear_fwd_tiled(X, tiled, d_out: int, s: float, L, R, Y=None, workspace=None, status=None,
+                          layout: int = LAYOUT_DECODE_TILED):
+    """Small-batch forward on a decode-tiled weight.  Returns Y (bf16 [b, d_out])."""
+    _dev(X, torch.bfloat16, "X"), _dev(tiled, torch.uint8, "tiled")
+    b, d_in = X.shape
+    r = 0 if L is None else L.shape[1]
+    if r:
+        _dev(L, torch.bfloat16, "L"), _dev(R, torch.bfloat16, "R")
+        if tuple(L.shape) != (d_out, r) or tuple(R.shape) != (r, d_in):
+            raise ValueError("adapter shapes do not match the weight")
+    if tiled.numel() != slim_tiled_bytes(d_out, d_in, layout):
+        raise ValueError("tiled weight does not match the shape")
+    if Y is None:
+        Y = torch.empty((b, d_out), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = new_workspace(b, d_out, d_in, r, X.device)
+    _check(lib().slim_linear_fwd_tiled(_ptr(X), b, _ptr(tiled), layout, float(s), _ptr(L) if r else None,
+                                       _ptr(R) if r else None, r, d_out, d_in, _ptr(Y), _ptr(workspace),
+                                       workspace.numel(), _ptr(status), _stream()), "slim_linear_fwd_tiled")
+    return Y
+
+
+def slim_linear_fwd_tiled_host(X_host: torch.Tensor, tiled, d_out: int, s: float, L, R, Y_host: torch.Tensor,
+                               x_dev, y_dev, workspace, status=None, layout: int = LAYOUT_DECODE_TILED):
+    """Host-buffer form of :func:`slim_linear_fwd_tiled` (copies inside the call, stream synchronised)."""
+    b, d_in = X_host.shape
+    r = 0 if L is None else L.shape[1]
+    _check(lib().slim_linear_fwd_tiled_host(ctypes.c_void_p(X_host.data_ptr()), b, _ptr(tiled), layout, float(s),
+                                            _ptr(L) if r else None, _ptr(R) if r else None, r, d_out, d_in,
+                                            ctypes.c_void_p(Y_host.data_ptr()), _ptr(x_dev), _ptr(y_dev),
+                                            _ptr(workspace), workspace.numel(), _ptr(status), _stream()),
+           "slim_linear_fwd_tiled_host")
+    return Y_host
 
 
 def slim_linear_fwd_host(X_host: torch.Tensor, vals, meta, s: float, L, R, Y_host: torch.Tensor,

@@ -8,7 +8,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libslim.so")
-SOURCES = ["api.cu", "pack.cu", "fwd_simple.cu", "fwd_decode.cu", "fwd_prefill.cu", "fwd_noalloc.cu"]
+SOURCES = ["api.cu", "pack.cu", "repack.cu", "fwd_simple.cu", "fwd_decode.cu", "fwd_decode_tiled.cu", "fwd_prefill.cu",
+           "fwd_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math"]
 
@@ -21,33 +22,41 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every CUDA source into ``libslim.so`` next to this file."""
-    if not force and not _stale():
+def build(force: bool = False, verbose: bool = False, defines=(), out: str | None = None) -> str:
+    """Compile every CUDA source into ``libslim.so`` next to this file.
+
+    ``defines``: extra ``-D`` macros (the kernels' optional hooks: ``SLIM_DECODE_TUNE`` lets the
+    environment override the decode plan, ``SLIM_DECODE_TRACE`` records a per-CTA timeline); such a
+    build goes to ``out`` (required then), never to the library the package loads by default."""
+    if defines and not out:
+        raise ValueError("a build with extra defines needs its own output path")
+    if not defines and not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     objs = []
-    bdir = os.path.join(HERE, "_build")
+    bdir = os.path.join(HERE, "_build" + ("_" + "_".join(sorted(defines)) if defines else ""))
     os.makedirs(bdir, exist_ok=True)
     procs = []
     for src in SOURCES:
         obj = os.path.join(bdir, src.replace(".cu", ".o"))
-        cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *[f"-D{d}" for d in defines], "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, src),
+               "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     for src, pr in procs:
-        out, _ = pr.communicate()
+        log, _ = pr.communicate()
         if pr.returncode != 0:
-            raise RuntimeError(f"nvcc failed on {src}:\n{out}")
-        if verbose and out:
-            print(out)
-    tmp = LIB + f".tmp{os.getpid()}"
+            raise RuntimeError(f"nvcc failed on {src}:\n{log}")
+        if verbose and log:
+            print(log)
+    target = out or LIB
+    tmp = target + f".tmp{os.getpid()}"
     subprocess.check_call([nvcc, "-shared", "-o", tmp, *objs, "-cudart", "static"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, target)
+    return target
 
 
 if __name__ == "__main__":

@@ -1,24 +1,29 @@
 // C-ABI entry points of libslim: argument checks, dispatch by batch size,
 // per-device attribute cache.  All arithmetic lives in the kernel files.
+#include <atomic>
+#include <cmath>
 #include <mutex>
 #include "common.cuh"
 
 namespace slim {
 
 static DeviceInfo g_info[64];
+static std::atomic<bool> g_info_ready[64];
 static std::mutex g_info_mutex;
 static thread_local int t_launches = 0;
 
 void count_launch(int n) { t_launches += n; }
 void reset_launch_count() { t_launches = 0; }
 
+// The record of a device is filled once under the mutex and published with a release store;
+// readers take it with an acquire load, so they never see a half-written record.
 const DeviceInfo* device_info(slim_status_t* err) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = SLIM_ERR_CUDA; return nullptr; }
     DeviceInfo& di = g_info[dev];
-    if (!di.ready) {
+    if (!g_info_ready[dev].load(std::memory_order_acquire)) {
         std::lock_guard<std::mutex> lock(g_info_mutex);
-        if (!di.ready) {
+        if (!g_info_ready[dev].load(std::memory_order_relaxed)) {
             cudaDeviceProp prop;
             if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { *err = SLIM_ERR_CUDA; return nullptr; }
             di.cc_major = prop.major;
@@ -26,12 +31,28 @@ const DeviceInfo* device_info(slim_status_t* err) {
             if (prop.major == 10) {
                 di.decode_ctas_per_sm[0] = decode_query_residency(1);
                 di.decode_ctas_per_sm[1] = decode_query_residency(2);
+                di.decode_tiled_ok = decode_tiled_query_residency();
             }
-            di.ready = true;
+            g_info_ready[dev].store(true, std::memory_order_release);
         }
     }
     if (di.cc_major != 10) { *err = SLIM_ERR_ARCH; return nullptr; }
     return &di;
+}
+
+void* tensor_map_encoder() {
+    static std::atomic<void*> cached{nullptr};
+    void* fn = cached.load(std::memory_order_acquire);
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess && ptr) {
+            cached.store(ptr, std::memory_order_release);      // every thread finds the same address
+            fn = ptr;
+        }
+    }
+    return fn;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -54,6 +75,8 @@ static size_t workspace_bytes(int b, int d_out, int d_in, int r) {
     if (d > need) need = d;
     const size_t pf = prefill_workspace_bytes(b, d_out, d_in, r);
     if (pf > need) need = pf;
+    const size_t dt = b <= 16 ? decode_tiled_workspace_bytes(b, d_out, d_in, r) : 0;
+    if (dt > need) need = dt;
     need = (need + 255) / 256 * 256;
     return SLIM_WORKSPACE_SYNC_BYTES + need;
 }
@@ -114,7 +137,7 @@ slim_status_t slim_linear_fwd_ex(const void* X, int b, const uint8_t* vals, cons
                                  uint32_t* status_dev, void* cuda_stream, slim_kernel_t kernel)
 {
     reset_launch_count();
-    if (!X || !vals || !meta || !Y || b < 1 || r < 0) return SLIM_ERR_INVALID_ARG;
+    if (!X || !vals || !meta || !Y || b < 1 || r < 0 || !std::isfinite(s)) return SLIM_ERR_INVALID_ARG;
     if ((r > 0) != (L != nullptr) || (r > 0) != (R != nullptr)) return SLIM_ERR_INVALID_ARG;
     slim_status_t st = check_weight_shape(d_out, d_in);
     if (st != SLIM_OK) return st;
@@ -158,6 +181,59 @@ slim_status_t slim_linear_fwd(const void* X, int b, const uint8_t* vals, const u
                               status_dev, cuda_stream, SLIM_KERNEL_AUTO);
 }
 
+size_t slim_tiled_bytes(int d_out, int d_in, int layout_id)
+{
+    if (layout_id != SLIM_LAYOUT_DECODE_TILED || d_out < 16 || d_in < 256 || d_out % 16 != 0 || d_in % 256 != 0) return 0;
+    return (size_t)d_out * (size_t)d_in / 8 * 3;
+}
+
+slim_status_t slim_repack_tiled(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in, int layout_id,
+                                void* tiled_out, void* cuda_stream)
+{
+    reset_launch_count();
+    if (!vals || !meta || !tiled_out || d_out < 1 || d_in < 1) return SLIM_ERR_INVALID_ARG;
+    if (slim_tiled_bytes(d_out, d_in, layout_id) == 0) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(vals) || !aligned16(meta) || !aligned16(tiled_out)) return SLIM_ERR_INVALID_ARG;
+    return launch_repack_tiled(vals, meta, d_out, d_in, static_cast<uint8_t*>(tiled_out), (cudaStream_t)cuda_stream);
+}
+
+slim_status_t slim_linear_fwd_tiled(const void* X, int b, const void* tiled, int layout_id, float s, const void* L,
+                                    const void* R, int r, int d_out, int d_in, void* Y, void* workspace,
+                                    size_t workspace_bytes_, uint32_t* status_dev, void* cuda_stream)
+{
+    reset_launch_count();
+    if (!X || !tiled || !Y || b < 1 || r < 0 || d_out < 1 || d_in < 1 || !std::isfinite(s)) return SLIM_ERR_INVALID_ARG;
+    if ((r > 0) != (L != nullptr) || (r > 0) != (R != nullptr)) return SLIM_ERR_INVALID_ARG;
+    if (slim_tiled_bytes(d_out, d_in, layout_id) == 0 || r % 16 != 0 || b > 16) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(X) || !aligned16(tiled) || !aligned16(Y) || !aligned16(L) || !aligned16(R) || !aligned16(workspace))
+        return SLIM_ERR_INVALID_ARG;
+    if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return SLIM_ERR_INVALID_ARG;
+    slim_status_t derr;
+    if (!device_info(&derr)) return derr;
+    if (!decode_tiled_supports(b, d_out, d_in, r)) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    if (!workspace || workspace_bytes_ < workspace_bytes(b, d_out, d_in, r)) return SLIM_ERR_WORKSPACE;
+    return launch_decode_tiled(static_cast<const __nv_bfloat16*>(X), b, static_cast<const uint8_t*>(tiled), s,
+                               static_cast<const __nv_bfloat16*>(L), static_cast<const __nv_bfloat16*>(R), r, d_out, d_in,
+                               static_cast<__nv_bfloat16*>(Y), workspace, status_dev, (cudaStream_t)cuda_stream);
+}
+
+slim_status_t slim_linear_fwd_tiled_host(const void* X_host, int b, const void* tiled, int layout_id, float s,
+                                         const void* L, const void* R, int r, int d_out, int d_in, void* Y_host,
+                                         void* x_dev, void* y_dev, void* workspace, size_t workspace_bytes_,
+                                         uint32_t* status_dev, void* cuda_stream)
+{
+    if (!X_host || !Y_host || !x_dev || !y_dev || b < 1 || d_in < 1 || d_out < 1) return SLIM_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(x_dev, X_host, (size_t)b * d_in * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return SLIM_ERR_CUDA;
+    slim_status_t st = slim_linear_fwd_tiled(x_dev, b, tiled, layout_id, s, L, R, r, d_out, d_in, y_dev, workspace,
+                                             workspace_bytes_, status_dev, cuda_stream);
+    if (st != SLIM_OK) return st;
+    if (cudaMemcpyAsync(Y_host, y_dev, (size_t)b * d_out * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return SLIM_ERR_CUDA;
+    return cudaStreamSynchronize(stream) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+}
+
 slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* vals,
                                    const uint8_t* meta, float s, const void* L, const void* R,
                                    int r, int d_out, int d_in, void* Y_host, void* x_dev,
@@ -194,6 +270,6 @@ const char* slim_strerror(slim_status_t status)
     return "unknown status";
 }
 
-const char* slim_version(void) { return "libslim 0.1 (sm_100a)"; }
+const char* slim_version(void) { return "libslim 0.2 (sm_100a)"; }
 
 }  // extern "C"

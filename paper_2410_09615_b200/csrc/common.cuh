@@ -16,12 +16,20 @@ __host__ __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b -
 
 // Per-device facts the launchers need (filled once per device, read-only after).
 struct DeviceInfo {
-    bool ready;
     int cc_major;
     int sm_count;
     int decode_ctas_per_sm[2];   // cooperative residency of the decode kernel, NT = 1, 2
+    int decode_tiled_ok;         // every variant of the tiled decode kernel can be resident once per SM
 };
 const DeviceInfo* device_info(slim_status_t* err);
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda);
+// nullptr when the driver does not have it.  Thread-safe.
+void* tensor_map_encoder();
+
+// The decode kernels keep the published T = X R^T at the start of the workspace, in a region of
+// this fixed size, so that calls of different shapes and kernels never read one kind of slot as another.
+constexpr size_t kDecodeTfinalBytes = 198656;
 
 // Launch bookkeeping for slim_last_launch_count().
 void count_launch(int n);
@@ -45,6 +53,15 @@ slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, 
                             int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
                             cudaStream_t st);
 int decode_query_residency(int nt);
+
+bool decode_tiled_supports(int b, int d_out, int d_in, int r);
+size_t decode_tiled_workspace_bytes(int b, int d_out, int d_in, int r);
+slim_status_t launch_decode_tiled(const __nv_bfloat16* X, int b, const uint8_t* W, float s, const __nv_bfloat16* L,
+                                  const __nv_bfloat16* R, int r, int d_out, int d_in, __nv_bfloat16* Y, void* ws,
+                                  uint32_t* status_dev, cudaStream_t st);
+int decode_tiled_query_residency();
+
+slim_status_t launch_repack_tiled(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in, uint8_t* out, cudaStream_t st);
 
 bool prefill_supports(int b, int d_out, int d_in, int r);
 size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r);

@@ -61,7 +61,8 @@ constexpr int kSlotBytes = 8 * kSubTile;
 constexpr size_t kSmemBudget = 227 * 1024;
 // The published T sits at a fixed place in the workspace (right after the call counter) so
 // that calls of different shapes sharing a workspace never read one kind of slot as the other.
-constexpr size_t kTfinalBytes = 16 * (size_t)(((kMaxDecodeRank + 63) / 64 * 64 + 32) / 2) * 8;
+constexpr size_t kTfinalBytes = kDecodeTfinalBytes;
+static_assert(16 * (size_t)(((kMaxDecodeRank + 63) / 64 * 64 + 32) / 2) * 8 <= kTfinalBytes, "published T does not fit its region");
 constexpr uint32_t kEmpty = 0xFFFFFFFFu;                   // "no value yet" in a partial-sum slot
 constexpr uint32_t kNanBits = 0x7FFFFFFFu;                 // what a computed all-ones NaN is stored as
 
@@ -149,16 +150,19 @@ __device__ __forceinline__ uint32_t ld_gpu(const uint32_t* p) {
 #endif
     return v;
 }
+// A published entry of T is read and written as ONE 64-bit access: only a scalar access is
+// guaranteed to be seen whole (value and call number together).
 __device__ __forceinline__ uint2 ld_gpu2(const uint2* p) {
-    uint2 v;
-    asm volatile("ld.relaxed.gpu.global.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
-    return v;
+    unsigned long long u;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(u) : "l"(p) : "memory");
+    return make_uint2((uint32_t)u, (uint32_t)(u >> 32));
 }
 __device__ __forceinline__ void st_gpu(uint32_t* p, uint32_t v) {
     asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void st_gpu2(uint2* p, uint2 v) {
-    asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1,%2};" :: "l"(p), "r"(v.x), "r"(v.y) : "memory");
+    const unsigned long long u = ((unsigned long long)v.y << 32) | v.x;
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" :: "l"(p), "l"(u) : "memory");
 }
 __device__ __forceinline__ unsigned long long ld_gpu64(const unsigned long long* p) {
     unsigned long long v;
@@ -787,27 +791,14 @@ size_t decode_workspace_bytes(int b, int d_out, int d_in, int r) {
     return pl.p_bytes + pl.tpart_bytes + pl.tfinal_bytes;
 }
 
-// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-static EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
-}
-
 // Row-major 2-D tensor [rows][row_elems] of `esize`-byte elements, tiles of box_rows x 128 bytes.
 static bool make_tile_map(CUtensorMap* map, const void* base, CUtensorMapDataType type, int esize,
                           uint64_t row_elems, uint64_t rows, int box_rows) {
-    EncodeTiledFn fn = encode_tiled_fn();
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(tensor_map_encoder());
     if (!fn) return false;
     cuuint64_t dims[2] = {row_elems, rows};
     cuuint64_t strides[1] = {row_elems * (uint64_t)esize};

@@ -1,0 +1,802 @@
+// Decode-phase forward (b <= 16) on the decode-tiled weight: one persistent cooperative kernel
+// that streams the weight and the adapters from HBM exactly once.
+//
+// Every consumer warp is a stream of its own.  The three operands are cut into slots of at
+// most 6 KB: a weight slot is MT row tiles of 16 rows x NB blocks of 256 columns of the
+// decode-tiled buffer (MT * NB = 4; contiguous pieces, fetched with cp.async.bulk), an
+// adapter slot is 16 rows x 128 columns of R or L (two TMA tiles).  A list of slots (R, then
+// the weight, then L) is divided evenly, in list order, among all consumer warps of the grid;
+// a warp fetches its slots through a private ring (it requests slot i + depth after it has
+// consumed slot i: no producer warp, no empty barriers, no barrier shared between warps) and
+// keeps the accumulators of the row tile it is walking in registers.  Whenever its range
+// leaves a row tile it writes the partial tile (fp32, MMA fragment order) to a slot of the
+// workspace.  Nothing is summed across warps in shared memory.
+//
+// Tensor-core mapping: the batch is the N dimension (one or two n-tiles of 8 tokens) of
+// mma.sp::ordered_metadata.m16n8k32 for the weight (the tiled buffer holds the A registers
+// and the metadata words as the instruction takes them) and of mma.m16n8k16 for the adapters.
+// Activations (and later T) sit in shared memory in B-fragment order, b tokens only.
+//
+// Large d_in: the activation slice a CTA can hold is bounded, so d_in is cut into KS slices and
+// a CTA belongs to one slice for the R and weight phases (the L phase has no such limit).
+//
+// Hand-over between CTAs, without fences or grid barriers (the launch is cooperative, all
+// CTAs are resident): a partial-sum slot holds a reserved NaN pattern while empty; its one
+// reader polls it, takes the value and marks it empty again.
+//   T = X R^T:   service warps (four per CTA) sum the partials of a 16-column piece in list
+//                order, round to bf16 and publish {two columns, call number} as one 64-bit
+//                word; the call number comes from a counter every CTA increments when it
+//                leaves.  The same warps then bring all of T into shared memory while the
+//                weight phase runs, and arrive on a barrier the consumers wait on before L.
+//   Y:           after its L range a warp finishes whole 16-row output tiles:
+//                Y = s * sum(weight partials) + sum(adapter partials), in list order.
+// All polls are bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on.
+// Reductions have a fixed order: results are bit-identical from run to run.
+#include <cuda.h>
+#include <cstdlib>
+#include <cstring>
+#include "decode_tile.cuh"
+
+namespace slim {
+
+namespace {
+
+using namespace dt;
+
+constexpr int kCW = 8;                                  // consumer warps
+constexpr int kSW = 4;                                  // service warps
+constexpr int kThreads = (kCW + kSW) * 32;
+constexpr int kMaxSlotBytes = 6144;
+constexpr int kBlockBytes = 1536;                       // one 16-row x 256-column block of the tiled weight
+constexpr int kMaxRing = 8;                             // slots per warp
+constexpr int kDCols = 128;                             // adapter columns per slot
+constexpr int kMaxRank = 3072;
+constexpr size_t kSmemBudget = 227 * 1024;
+constexpr uint32_t kPollLimit = 1u << 22;
+constexpr uint32_t kMbarSpinLimit = 1u << 26;
+constexpr uint32_t kEmpty = 0xFFFFFFFFu;                // "no value yet" in a partial-sum slot
+constexpr uint32_t kNanBits = 0x7FFFFFFFu;              // what a computed all-ones NaN is stored as
+constexpr size_t kTfinalBytes = kDecodeTfinalBytes;
+static_assert(16 * (size_t)(kMaxRank / 2) * 8 <= kTfinalBytes, "published T does not fit its region");
+
+struct Params {
+    const __nv_bfloat16* X; const uint8_t* W; __nv_bfloat16* Y;
+    uint32_t* Ppart; uint32_t* Apart; uint32_t* Tpart;
+    unsigned long long* Tfinal;          // [b][r / 2]  {bf16 pair, call number}
+    unsigned long long* departures;      // CTAs that ever left a call on this workspace
+    uint32_t* status;
+    float s;
+    int b, r, d_out, d_in;
+    int KS, G;                           // k-slices; CTAs per slice
+    int nblk;                            // 256-column blocks of a row
+    int NB;                              // blocks per weight slot (MT * NB = 4)
+    int unitsW, tilesW, tilesR, nqL;     // ceil(tilesW / MT); d_out / 16; r / 16; ceil(r / 128)
+    int wnR;                             // workers per slice in the R phase (<= G * kCW)
+    int muW, muR, muL;                   // partial slots a worker owns in each phase
+    int ring, slot_bytes;                // ring slots per warp; bytes between slots (a multiple of 1024)
+    int x_bytes;                         // activation slice region
+};
+
+// Optional timeline: built with -DSLIM_TILED_TRACE, lane 0 of consumer warp 0 (entries 0-7) and of service
+// warp 0 (entries 8-9) of every CTA record the global timer (read back with slim_debug_read_tiled_trace).
+#ifdef SLIM_TILED_TRACE
+__device__ unsigned long long g_tiled_dbg[16];
+__device__ unsigned long long g_tiled_trace[256 * 16];
+#define TSTAMP(w, i) do { if (warp == (w) && lane == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_tiled_trace[blockIdx.x * 16 + (i)] = t_; } } while (0)
+#else
+#define TSTAMP(w, i) do { } while (0)
+#endif
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t it = 0; it < kMbarSpinLimit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_tile(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 :: "r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+// Contiguous bytes global -> shared (both 16-byte aligned, size a multiple of 16).
+__device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// Device-scope accesses that bypass L1: the hand-over slots.
+__device__ __forceinline__ uint32_t ld_gpu(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_gpu(uint32_t* p, uint32_t v) {
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_gpu64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_gpu64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" :: "l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t slot_bits(float v) {    // fp32 bits that never equal kEmpty
+    const uint32_t u = __float_as_uint(v);
+    return u == kEmpty ? kNanBits : u;
+}
+
+// ---------------------------------------------------------------- even division of a list
+// S list positions among Wn workers, in order: the first S % Wn workers get one more.
+struct Split { int len, rem; };
+__host__ __device__ __forceinline__ Split make_split(int S, int Wn) { Split sp; sp.len = S / Wn; sp.rem = S % Wn; return sp; }
+__host__ __device__ __forceinline__ int split_start(const Split& sp, int w) { return w * sp.len + (w < sp.rem ? w : sp.rem); }
+__host__ __device__ __forceinline__ int split_count(const Split& sp, int w) { return sp.len + (w < sp.rem ? 1 : 0); }
+__host__ __device__ __forceinline__ int split_owner(const Split& sp, int pos) {
+    const int edge = sp.rem * (sp.len + 1);
+    return pos < edge ? pos / (sp.len + 1) : sp.rem + (pos - edge) / sp.len;   // pos >= edge implies len > 0
+}
+
+// Blocks [b0, b1) of k-slice ks.
+__host__ __device__ __forceinline__ void slice_blocks(int ks, int KS, int nblk, int* b0, int* b1) {
+    *b0 = (int)((long long)ks * nblk / KS);
+    *b1 = (int)((long long)(ks + 1) * nblk / KS);
+}
+
+// Walks, in list order, the partial-sum slots that the workers of one phase left for one list
+// unit: every worker whose range meets the unit's positions owns `mu` slots of `stride` words,
+// the unit's being number (unit - first unit of the worker's range).
+struct PartWalk {
+    const Split sp; const int nq, mu, unit; const size_t stride; uint32_t* const base;
+    int w, w_last;
+    __device__ PartWalk(uint32_t* base_, const Split& sp_, int nq_, int mu_, int unit_, size_t stride_, int worker0)
+        : sp(sp_), nq(nq_), mu(mu_), unit(unit_), stride(stride_), base(base_ + (size_t)worker0 * mu_ * stride_) {
+        w = nq > 0 ? split_owner(sp, unit * nq) : 0;
+        w_last = nq > 0 ? split_owner(sp, unit * nq + nq - 1) : -1;
+    }
+    __device__ uint32_t* next() {
+        if (w > w_last) return nullptr;
+        const int u0 = split_start(sp, w) / nq;
+        uint32_t* p = base + ((size_t)w * mu + (unit - u0)) * stride;
+        ++w;
+        return p;
+    }
+};
+
+constexpr int kBatch = 8;        // partial slots requested together
+
+// Adds to sum[e] (e < E: elements lane + 32 e of a fragment-ordered tile at `off` words inside a
+// slot) the next up-to-kBatch slots of the walk; empties them.  Returns false when the walk is over.
+template <int E>
+__device__ __forceinline__ bool take_batch(PartWalk& pw, int off, int lane, float (&sum)[E], bool* ok) {
+    uint32_t* ptr[kBatch];
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k) ptr[k] = pw.next();
+    if (!ptr[0]) return false;
+    uint32_t v[kBatch][E];
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k)
+#pragma unroll
+        for (int e = 0; e < E; ++e) v[k][e] = ptr[k] ? ld_gpu(ptr[k] + off + e * 32 + lane) : 0u;
+    for (uint32_t spins = 0;; ++spins) {
+        bool all = true;
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k)
+#pragma unroll
+            for (int e = 0; e < E; ++e)
+                if (v[k][e] == kEmpty) { v[k][e] = ld_gpu(ptr[k] + off + e * 32 + lane); all = false; }
+        if (all) break;
+        if (spins > kPollLimit) { *ok = false; break; }
+    }
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k)
+        if (ptr[k]) {
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                sum[e] += __uint_as_float(v[k][e]);
+                st_gpu(ptr[k] + off + e * 32 + lane, kEmpty);
+            }
+        }
+    return ptr[kBatch - 1] != nullptr;
+}
+
+template <int NT, int MT>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmL)
+{
+    constexpr int frag = NT * 128;                   // words of one 16-row partial tile
+    constexpr int E = NT * 4;                        // fragment elements per lane
+    extern __shared__ unsigned char smem_raw[];
+    // layout (1024-byte aligned for the swizzle): rings | X slice | T | barriers
+    unsigned char* rings = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char* xs = rings + (size_t)kCW * p.ring * p.slot_bytes;
+    unsigned char* ts = xs + p.x_bytes;
+    const int t_bytes = p.nqL * 4 * p.b * 64;
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(ts + t_bytes);      // [kCW][kMaxRing]
+    uint64_t* t_bar = full_bar + kCW * kMaxRing;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_ctas = gridDim.x, cta = blockIdx.x;
+    const LaneCtx lc = make_lane_ctx(lane);
+    const int NB = p.NB;
+
+    // this CTA's k-slice
+    const bool in_slice = cta < p.KS * p.G;
+    const int ks = in_slice ? cta % p.KS : 0, grp = in_slice ? cta / p.KS : 0;
+    int blk0, blk1;
+    slice_blocks(ks, p.KS, p.nblk, &blk0, &blk1);
+    const int nqW = ceil_div(blk1 - blk0, NB);               // weight slots per unit in this slice
+    const int nqR = (blk1 - blk0) * 2;                       // adapter slots per R tile in this slice
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kCW * kMaxRing; ++i) mbar_init(&full_bar[i], 1);
+        mbar_init(t_bar, kSW);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    // which kind of wait expired, if any: reported in bits 16-23 of the status word beside SLIM_ERR_TIMEOUT
+    // (1 R slot, 2 weight slot, 4 T in shared memory, 8 L slot, 16 partials of an output tile,
+    //  64 partials of T, 128 published T)
+    uint32_t expired = 0;
+    bool ok = true;
+    TSTAMP(0, 0);
+#ifdef SLIM_TILED_TRACE
+    if (threadIdx.x == 0) { g_tiled_trace[blockIdx.x * 16 + 11] = 0; g_tiled_trace[blockIdx.x * 16 + 12] = 0; g_tiled_trace[blockIdx.x * 16 + 13] = clock64(); }
+#endif
+    if (warp < kCW) {
+        // ================================ consumer warps ================================
+        const Split spR = make_split(p.tilesR * nqR, p.wnR);
+        const Split spW = make_split(p.unitsW * nqW, p.G * kCW);
+        const Split spL = make_split(p.tilesW * p.nqL, n_ctas * kCW);
+        const int wi = grp * kCW + warp;                      // worker number inside the slice
+        const int wl = cta * kCW + warp;                      // worker number in the grid
+        const int nR = in_slice && wi < p.wnR ? split_count(spR, wi) : 0, sR = split_start(spR, wi);
+        const int nW = in_slice ? split_count(spW, wi) : 0, sW = split_start(spW, wi);
+        const int nL = split_count(spL, wl), sL = split_start(spL, wl);
+        const int total = nR + nW + nL;
+        uint64_t* my_bar = full_bar + warp * kMaxRing;
+        const uint32_t my_ring = smem_u32(rings + (size_t)warp * p.ring * p.slot_bytes);
+
+        // Request the slot of job j into ring slot j % ring (the whole warp calls this).
+        auto issue = [&](int j) {
+            const int slot = j % p.ring;
+            uint64_t* bar = &my_bar[slot];
+            const uint32_t dst = my_ring + slot * p.slot_bytes;
+            if (j < nR) {
+                const int pos = sR + j, tile = pos / nqR, q = pos % nqR;
+                if (lane == 0) mbar_arrive_expect_tx(bar, 4096);
+                if (lane < 2) tma_tile(dst + lane * 2048, &tmR, blk0 * 256 + q * kDCols + 64 * lane, tile * 16, bar);
+            } else if (j < nR + nW) {
+                const int pos = sW + (j - nR), u = pos / nqW, q = pos % nqW;
+                const int nb = min(NB, blk1 - blk0 - q * NB), mt = min(MT, p.tilesW - u * MT);
+                if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(mt * nb * kBlockBytes));
+                if (lane < mt)
+                    bulk_copy(dst + lane * NB * kBlockBytes,
+                              p.W + ((size_t)(u * MT + lane) * p.nblk + blk0 + q * NB) * kBlockBytes, (uint32_t)(nb * kBlockBytes), bar);
+            } else {
+                const int pos = sL + (j - nR - nW), tile = pos / p.nqL, q = pos % p.nqL;
+                if (lane == 0) mbar_arrive_expect_tx(bar, 4096);
+                if (lane < 2) tma_tile(dst + lane * 2048, &tmL, q * kDCols + 64 * lane, tile * 16, bar);
+            }
+        };
+        const int pre = min(total, p.ring);
+        for (int j = 0; j < pre; ++j) issue(j);
+        TSTAMP(0, 10);
+
+        // ---- the CTA's slice of the activations into shared memory, fragment order.  A thread
+        // requests several 16-byte pieces before it stores the first (one global round trip per batch).
+        if (in_slice) {
+            const int cols = (blk1 - blk0) * 256, chunks = cols / 8;      // 16-byte chunks per token
+            const __nv_bfloat16* xsrc = p.X + (size_t)blk0 * 256;
+            const int n_chunks = p.b * chunks;
+            constexpr int kXBatch = 8;
+            for (int i0 = threadIdx.x; i0 < n_chunks; i0 += kCW * 32 * kXBatch) {
+                uint4 v[kXBatch];
+#pragma unroll
+                for (int k = 0; k < kXBatch; ++k) {
+                    const int idx = i0 + k * kCW * 32;
+                    if (idx < n_chunks) {
+                        const int tok = idx / chunks, c = idx - tok * chunks;
+                        v[k] = __ldg(reinterpret_cast<const uint4*>(xsrc + (size_t)tok * p.d_in + 8 * c));
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < kXBatch; ++k) {
+                    const int idx = i0 + k * kCW * 32;
+                    if (idx < n_chunks) {
+                        const int tok = idx / chunks, c = idx - tok * chunks;
+                        // columns 8c .. 8c+7 = step c/4, register i = c%4, pairs t = 0..3
+                        uint32_t* dst = reinterpret_cast<uint32_t*>(xs) + (((c >> 2) * p.b + tok) * 16 + (c & 3));
+                        dst[0] = v[k].x; dst[4] = v[k].y; dst[8] = v[k].z; dst[12] = v[k].w;
+                    }
+                }
+            }
+        }
+        asm volatile("bar.sync 1, %0;" :: "n"(kCW * 32) : "memory");          // the consumer warps only
+        TSTAMP(0, 1);
+
+        const uint32_t xs_addr = smem_u32(xs), ts_addr = smem_u32(ts);
+        uint32_t* const Pmine = p.Ppart + ((size_t)(ks * p.G * kCW + wi) * p.muW) * (MT * frag);
+        uint32_t* const Tmine = p.Tpart + ((size_t)(ks * p.wnR + wi) * p.muR) * frag;
+        uint32_t* const Amine = p.Apart + ((size_t)wl * p.muL) * frag;
+
+        float acc[MT][NT][4];
+        auto zero_acc = [&]() {
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+#pragma unroll
+                for (int h = 0; h < NT; ++h)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[m][h][e] = 0.f;
+        };
+        auto store_tile = [&](uint32_t* dst, const float (&a)[NT][4]) {
+#pragma unroll
+            for (int h = 0; h < NT; ++h)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) st_gpu(dst + (h * 4 + e) * 32 + lane, slot_bits(a[h][e]));
+        };
+        zero_acc();
+        int cur = -1;                 // list unit whose accumulators are live
+        bool t_ready = p.r == 0;
+
+        for (int j = 0; j < total; ++j) {
+            const int slot = j % p.ring;
+            const uint32_t src = my_ring + slot * p.slot_bytes;
+            if (j < nR) {
+                // ---------------------------------------------------------------- R slot
+                const int pos = sR + j, tile = pos / nqR, q = pos % nqR;
+                if (tile != cur) {
+                    if (cur >= 0) store_tile(Tmine + (size_t)(cur - sR / nqR) * frag, acc[0]);
+                    zero_acc();
+                    cur = tile;
+                }
+                if (!mbar_wait(&my_bar[slot], (j / p.ring) & 1)) expired |= 1u;
+                if (j == 0) TSTAMP(0, 2);
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    uint4 xb[NT];
+                    load_x_step<NT>(xb, xs_addr, q * 4 + jj, p.b, lc);
+                    dense_step<NT>(acc[0], src + (jj >> 1) * 2048, jj & 1, xb, lc);
+                }
+                if (j + 1 == nR) { store_tile(Tmine + (size_t)(cur - sR / nqR) * frag, acc[0]); zero_acc(); cur = -1; }
+            } else if (j < nR + nW) {
+                // ---------------------------------------------------------------- weight slot
+                const int pos = sW + (j - nR), u = pos / nqW, q = pos % nqW;
+                if (u != cur) {
+                    if (cur >= 0) {
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) store_tile(Pmine + ((size_t)(cur - sW / nqW) * MT + m) * frag, acc[m]);
+                    }
+                    zero_acc();
+                    cur = u;
+                }
+                const int nb = min(NB, blk1 - blk0 - q * NB), mt = min(MT, p.tilesW - u * MT);
+#ifdef SLIM_TILED_TRACE
+                const long long w0_ = clock64();
+#endif
+                if (!mbar_wait(&my_bar[slot], (j / p.ring) & 1)) expired |= 2u;
+#ifdef SLIM_TILED_TRACE
+                if (warp == 0 && lane == 0) { g_tiled_trace[blockIdx.x * 16 + 11] += clock64() - w0_; g_tiled_trace[blockIdx.x * 16 + 12] += 1; }
+#endif
+                if (j == nR) TSTAMP(0, 3);
+                for (int bi = 0; bi < nb; ++bi) {
+                    uint4 xf[8][NT];
+                    load_x_block<NT>(xf, xs_addr, (q * NB + bi) * 8, p.b, lc);
+#pragma unroll
+                    for (int m = 0; m < MT; ++m)
+                        if (m < mt) sparse_block<NT>(acc[m], src + (m * NB + bi) * kBlockBytes, xf, lc);
+                }
+                if (j + 1 == nR + nW) {
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) store_tile(Pmine + ((size_t)(cur - sW / nqW) * MT + m) * frag, acc[m]);
+                    zero_acc(); cur = -1;
+                }
+            } else {
+                // ---------------------------------------------------------------- L slot
+                const int pos = sL + (j - nR - nW), tile = pos / p.nqL, q = pos % p.nqL;
+                if (tile != cur) {
+                    if (cur >= 0) store_tile(Amine + (size_t)(cur - sL / p.nqL) * frag, acc[0]);
+                    zero_acc();
+                    cur = tile;
+                }
+                if (j == nR + nW) TSTAMP(0, 4);
+                if (!t_ready) { if (!mbar_wait(t_bar, 0)) expired |= 4u; t_ready = true; TSTAMP(0, 5); }
+                if (!mbar_wait(&my_bar[slot], (j / p.ring) & 1)) expired |= 8u;
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    uint4 tb[NT];
+                    load_x_step<NT>(tb, ts_addr, q * 4 + jj, p.b, lc);
+                    dense_step<NT>(acc[0], src + (jj >> 1) * 2048, jj & 1, tb, lc);
+                }
+                if (j + 1 == total) { store_tile(Amine + (size_t)(cur - sL / p.nqL) * frag, acc[0]); cur = -1; }
+            }
+            __syncwarp();                                   // every lane is done reading the slot
+            if (j + p.ring < total) issue(j + p.ring);
+        }
+
+        TSTAMP(0, 6);
+        // ---------------------------------------------------------------- output tiles
+        const Split spF = make_split(p.tilesW, n_ctas * kCW);
+        const int f0 = split_start(spF, wl), f1 = f0 + split_count(spF, wl);
+        for (int tile = f0; tile < f1; ++tile) {
+            float psum[E], asum[E];
+#pragma unroll
+            for (int e = 0; e < E; ++e) { psum[e] = 0.f; asum[e] = 0.f; }
+            const int u = tile / MT, m = tile % MT;
+            // walk state: slice of the weight partials being walked (p.KS = the adapter partials, then the end)
+            int k2 = -1, w = 0, w_last = -1, nq2 = 1;
+            Split sp2 = spL;
+            auto next_part = [&](bool* is_adapter) -> uint32_t* {
+                while (w > w_last) {
+                    ++k2;
+                    if (k2 > p.KS || (k2 == p.KS && p.r == 0)) return nullptr;
+                    if (k2 < p.KS) {
+                        int c0, c1;
+                        slice_blocks(k2, p.KS, p.nblk, &c0, &c1);
+                        nq2 = ceil_div(c1 - c0, NB);
+                        sp2 = make_split(p.unitsW * nq2, p.G * kCW);
+                        w = split_owner(sp2, u * nq2); w_last = split_owner(sp2, u * nq2 + nq2 - 1);
+                    } else {
+                        nq2 = p.nqL; sp2 = spL;
+                        w = split_owner(sp2, tile * nq2); w_last = split_owner(sp2, tile * nq2 + nq2 - 1);
+                    }
+                }
+                const int u0 = split_start(sp2, w) / nq2;
+                uint32_t* ptr;
+                if (k2 < p.KS) ptr = p.Ppart + (((size_t)(k2 * p.G * kCW + w) * p.muW + (u - u0)) * MT + m) * frag;
+                else           ptr = p.Apart + ((size_t)w * p.muL + (tile - u0)) * frag;
+                *is_adapter = k2 == p.KS;
+                ++w;
+                return ptr;
+            };
+            for (bool more = true; more;) {
+                uint32_t* ptr[kBatch];
+                bool adapter[kBatch];
+#pragma unroll
+                for (int k = 0; k < kBatch; ++k) { adapter[k] = false; ptr[k] = more ? next_part(&adapter[k]) : nullptr; if (!ptr[k]) more = false; }
+                uint32_t v[kBatch][E];
+#pragma unroll
+                for (int k = 0; k < kBatch; ++k)
+#pragma unroll
+                    for (int e = 0; e < E; ++e) v[k][e] = ptr[k] ? ld_gpu(ptr[k] + e * 32 + lane) : 0u;
+                for (uint32_t spins = 0;; ++spins) {
+                    bool all = true;
+#pragma unroll
+                    for (int k = 0; k < kBatch; ++k)
+#pragma unroll
+                        for (int e = 0; e < E; ++e)
+                            if (v[k][e] == kEmpty) { v[k][e] = ld_gpu(ptr[k] + e * 32 + lane); all = false; }
+                    if (all) break;
+                    if (spins > kPollLimit) {
+                        expired |= 16u;
+#ifdef SLIM_TILED_TRACE
+                        for (int k = 0; k < kBatch; ++k)
+                            for (int e = 0; e < E; ++e)
+                                if (v[k][e] == kEmpty && atomicAdd(&g_tiled_dbg[0], 1ull) == 0) {
+                                    g_tiled_dbg[1] = tile; g_tiled_dbg[2] = adapter[k]; g_tiled_dbg[3] = (unsigned long long)(ptr[k] - (adapter[k] ? p.Apart : p.Ppart));
+                                    g_tiled_dbg[4] = blockIdx.x * 100 + warp; g_tiled_dbg[5] = e * 32 + lane; g_tiled_dbg[6] = k;
+                                }
+#endif
+                        break;
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < kBatch; ++k)
+                    if (ptr[k]) {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            if (adapter[k]) asum[e] += __uint_as_float(v[k][e]); else psum[e] += __uint_as_float(v[k][e]);
+                            st_gpu(ptr[k] + e * 32 + lane, kEmpty);
+                        }
+                    }
+            }
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const int h = e >> 2, q = e & 3;
+                const int n = tile * 16 + lc.g + 8 * (q >> 1);
+                const int tok = 8 * h + 2 * lc.t + (q & 1);
+                if (tok < p.b) p.Y[(size_t)tok * p.d_out + n] = __float2bfloat16_rn(fmaf(psum[e], p.s, asum[e]));
+            }
+        }
+        TSTAMP(0, 7);
+#ifdef SLIM_TILED_TRACE
+        if (warp == 0 && lane == 0) g_tiled_trace[blockIdx.x * 16 + 13] = clock64() - g_tiled_trace[blockIdx.x * 16 + 13];
+#endif
+    } else if (p.r > 0) {
+        // ================================ service warps ================================
+        const int sw = warp - kCW;
+        const uint32_t call = (uint32_t)(ld_gpu64(p.departures) / (unsigned)n_ctas) + 1u;
+        const int pairs = p.r / 2;
+        // ---- sum the partials of T, 32 fragment elements per item, and publish them
+        const int items = p.tilesR * E;
+        for (int it = cta * kSW + sw; it < items; it += n_ctas * kSW) {
+            const int jt = it / E, e = it % E;
+            float sum[1] = {0.f};
+            for (int k2 = 0; k2 < p.KS; ++k2) {
+                int c0, c1;
+                slice_blocks(k2, p.KS, p.nblk, &c0, &c1);
+                const int nq2 = (c1 - c0) * 2;
+                PartWalk pw(p.Tpart, make_split(p.tilesR * nq2, p.wnR), nq2, p.muR, jt, (size_t)frag, k2 * p.wnR);
+                while (take_batch<1>(pw, e * 32, lane, sum, &ok)) { }
+                if (!ok) expired |= 64u;
+            }
+            // element (h, q, lane) of the fragment is T[token 8h + 2(lane%4) + (q&1)][16 jt + lane/4 + 8(q>>1)]:
+            // lanes 8i + t and 8i + 4 + t hold neighbouring columns
+            const float other = __shfl_xor_sync(0xffffffffu, sum[0], 4);
+            const int h = e >> 2, q = e & 3;
+            const int tok = 8 * h + 2 * lc.t + (q & 1);
+            if (!(lc.g & 1) && tok < p.b) {
+                const int col = jt * 16 + lc.g + 8 * (q >> 1);
+                const __nv_bfloat162 pr = __floats2bfloat162_rn(sum[0], other);
+                st_gpu64(p.Tfinal + (size_t)tok * pairs + (col >> 1),
+                         ((unsigned long long)call << 32) | *reinterpret_cast<const uint32_t*>(&pr));
+            }
+        }
+        TSTAMP(kCW, 8);
+        // ---- all of T into shared memory (fragment order; columns past r are zero)
+        const int st = threadIdx.x - kCW * 32;
+        uint32_t* tsw = reinterpret_cast<uint32_t*>(ts);
+        for (int i = st; i < t_bytes / 4; i += kSW * 32) tsw[i] = 0u;
+        asm volatile("bar.sync 2, %0;" :: "n"(kSW * 32) : "memory");            // the service warps only
+        const int entries = p.b * pairs;
+        constexpr int kFetch = 8;
+        for (int e0 = st; e0 < entries; e0 += kSW * 32 * kFetch) {
+            unsigned long long v[kFetch];
+#pragma unroll
+            for (int k = 0; k < kFetch; ++k) {
+                const int e = e0 + k * kSW * 32;
+                v[k] = e < entries ? ld_gpu64(p.Tfinal + e) : ((unsigned long long)call << 32);
+            }
+            for (uint32_t spins = 0;; ++spins) {
+                bool all = true;
+#pragma unroll
+                for (int k = 0; k < kFetch; ++k)
+                    if ((uint32_t)(v[k] >> 32) != call) { v[k] = ld_gpu64(p.Tfinal + e0 + k * kSW * 32); all = false; }
+                if (all) break;
+                if (spins > kPollLimit) { expired |= 128u; break; }
+            }
+#pragma unroll
+            for (int k = 0; k < kFetch; ++k) {
+                const int e = e0 + k * kSW * 32;
+                if (e < entries) {
+                    const int tok = e / pairs, col = 2 * (e % pairs);
+                    // column col = 32 step + 2 t + 8 i
+                    const int step = col >> 5, i = (col >> 3) & 3, t = (col >> 1) & 3;
+                    tsw[((step * p.b + tok) * 4 + t) * 4 + i] = (uint32_t)v[k];
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(t_bar);
+        TSTAMP(kCW, 9);
+    }
+
+    if (expired && p.status) atomicOr(p.status, (1u << SLIM_ERR_TIMEOUT) | (expired << 16));
+    __syncthreads();                                       // every poll of this CTA is over
+    if (threadIdx.x == 0) atomicAdd(p.departures, 1ull);
+}
+
+// ------------------------------------------------------------------ host side
+struct Plan {
+    int nt, mt, nb, KS, G, nblk, ring, slot_bytes;
+    int unitsW, tilesW, tilesR, nqL, wnR, muW, muR, muL;
+    int x_bytes;
+    size_t smem, p_bytes, a_bytes, t_bytes;
+};
+
+// Slots a worker needs: one per list unit its range can meet.
+int slots_per_worker(int S, int Wn, int nq) {
+    if (S == 0 || nq == 0) return 1;
+    const int longest = S / Wn + (S % Wn ? 1 : 0);
+    return (longest + nq - 2) / nq + 1;
+}
+
+bool shape_ok(int b, int d_out, int d_in, int r) {
+    return b >= 1 && b <= 16 && d_in % 256 == 0 && d_in >= 256 && d_out % 16 == 0 && d_out >= 16 && r % 16 == 0 && r >= 0 &&
+           r <= kMaxRank;
+}
+
+bool make_plan(int b, int d_out, int d_in, int r, int ctas, Plan* pl) {
+    if (!shape_ok(b, d_out, d_in, r) || ctas < 1) return false;
+    pl->nt = b <= 8 ? 1 : 2;
+    pl->nblk = d_in / 256;
+    pl->tilesW = d_out / 16;
+    pl->tilesR = r / 16;
+    pl->nqL = ceil_div(r, kDCols);
+    const int workers = ctas * kCW;
+    // Row tiles per weight slot: wide slots share the activation fragments of a block among more
+    // rows (the activation reads are what loads shared memory), but leave fewer, larger list
+    // units; take the widest one that still gives every warp a few slots.
+    const long long tile_blocks = (long long)pl->tilesW * pl->nblk;
+    pl->mt = 1;
+    if (tile_blocks >= 6LL * workers && pl->tilesW >= 2) pl->mt = 2;
+    if (tile_blocks >= 8LL * workers && pl->tilesW >= 4 && pl->nt == 2) pl->mt = 4;
+    pl->nb = 4 / pl->mt;
+    if (tile_blocks < 4LL * workers) pl->nb = pl->nb > 2 ? 2 : pl->nb;      // small problems: finer slots
+    if (tile_blocks < 2LL * workers) pl->nb = 1;
+#ifdef SLIM_DECODE_TUNE
+    // experiments only: the environment overrides the slot shape
+    if (const char* e = getenv("SLIM_MT")) { const int v = atoi(e); if ((v == 1 || v == 2 || (v == 4 && pl->nt == 2)) && pl->tilesW >= v) { pl->mt = v; pl->nb = 4 / v; } }
+    if (const char* e = getenv("SLIM_NB")) { const int v = atoi(e); if (v >= 1 && v * pl->mt <= 4) pl->nb = v; }
+#endif
+    pl->unitsW = ceil_div(pl->tilesW, pl->mt);
+    // shared memory: T, the rings, and the activation slice (b tokens x 2 bytes per column).  The rings want
+    // to hold what HBM delivers during one round trip (about 18 KB per warp); the slice wants to be wide,
+    // because every k-slice adds a set of partial sums.  Take the deepest ring (up to kMaxRing slots)
+    // that still leaves the whole row to one slice, else three slots, else two.
+    const size_t t_smem = (size_t)pl->nqL * 4 * b * 64;
+    const size_t fixed = 1024 + t_smem + (kCW * kMaxRing + 1) * 8 + 64;
+    int slot = pl->mt * pl->nb * kBlockBytes;
+    if (r > 0 && slot < 4096) slot = 4096;
+    slot = (slot + 1023) / 1024 * 1024;
+    pl->slot_bytes = slot;
+    const size_t row_bytes = (size_t)pl->nblk * 512 * b;
+    auto left_with = [&](int ring) -> size_t {
+        const size_t used = fixed + (size_t)kCW * ring * slot;
+        return kSmemBudget > used ? kSmemBudget - used : 0;
+    };
+    pl->ring = 2;
+    for (int ring = kMaxRing; ring >= 3; --ring)
+        if (left_with(ring) >= row_bytes || (ring == 3 && left_with(3) >= (size_t)b * 512 * 4)) { pl->ring = ring; break; }
+#ifdef SLIM_DECODE_TUNE
+    if (const char* e = getenv("SLIM_RING")) { const int v = atoi(e); if (v >= 2 && v <= kMaxRing && left_with(v) >= (size_t)b * 512) pl->ring = v; }
+#endif
+    const size_t left = left_with(pl->ring);
+    const int max_blocks = (int)(left / ((size_t)b * 512));
+    if (max_blocks < 1) return false;
+    pl->KS = ceil_div(pl->nblk, max_blocks);
+    if (pl->KS > ctas) return false;
+    pl->G = ctas / pl->KS;
+    int widest = 0, nq_min = 1 << 30, nqr_min = 1 << 30, muW = 1, muR = 1;
+    const int slice_workers = pl->G * kCW;
+    // R phase: at least two slots per worker, so that a piece of T has fewer partials to collect
+    {
+        int b0, b1;
+        slice_blocks(0, pl->KS, pl->nblk, &b0, &b1);
+        const int S = pl->tilesR * (b1 - b0) * 2;
+        int wn = S / 2;
+        pl->wnR = wn < 1 ? 1 : (wn > slice_workers ? slice_workers : wn);
+    }
+    for (int ks = 0; ks < pl->KS; ++ks) {
+        int b0, b1;
+        slice_blocks(ks, pl->KS, pl->nblk, &b0, &b1);
+        if (b1 - b0 > widest) widest = b1 - b0;
+        const int nq = ceil_div(b1 - b0, pl->nb), nqr = (b1 - b0) * 2;
+        if (nq < nq_min) nq_min = nq;
+        if (nqr < nqr_min) nqr_min = nqr;
+        const int mw = slots_per_worker(pl->unitsW * nq, slice_workers, nq), mr = slots_per_worker(pl->tilesR * nqr, pl->wnR, nqr);
+        if (mw > muW) muW = mw;
+        if (mr > muR) muR = mr;
+    }
+    pl->muW = muW; pl->muR = muR;
+    pl->muL = slots_per_worker(pl->tilesW * pl->nqL, workers, pl->nqL);
+    pl->x_bytes = widest * 512 * b;
+    pl->smem = fixed + (size_t)kCW * pl->ring * pl->slot_bytes + pl->x_bytes;
+    const size_t frag_bytes = (size_t)pl->nt * 128 * sizeof(float);
+    pl->p_bytes = (size_t)pl->KS * slice_workers * pl->muW * pl->mt * frag_bytes;
+    pl->a_bytes = r > 0 ? (size_t)workers * pl->muL * frag_bytes : 0;
+    pl->t_bytes = r > 0 ? (size_t)pl->KS * pl->wnR * pl->muR * frag_bytes : 0;
+    return pl->smem <= kSmemBudget;
+}
+
+template <int NT, int MT>
+int query_residency() {
+    int n = 0;
+    if (cudaFuncSetAttribute(decode_tiled_kernel<NT, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+        return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_tiled_kernel<NT, MT>, kThreads, kSmemBudget) != cudaSuccess) return 0;
+    return n > 0 ? 1 : 0;
+}
+
+int grid_ctas() {
+    slim_status_t err;
+    const DeviceInfo* di = device_info(&err);
+    if (!di) return 148;       // sizing queries without a device assume a full B200
+    return di->decode_tiled_ok ? di->sm_count : 0;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Row-major bf16 matrix [rows][cols], tiles of 16 rows x 64 columns (128 bytes), 128-byte swizzle.
+bool make_tile_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows) {
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(tensor_map_encoder());
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {64, 16};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int decode_tiled_query_residency() {
+    return query_residency<1, 1>() && query_residency<1, 2>() && query_residency<2, 1>() && query_residency<2, 2>() &&
+           query_residency<2, 4>();
+}
+
+bool decode_tiled_supports(int b, int d_out, int d_in, int r) {
+    Plan pl;
+    const int ctas = grid_ctas();
+    return ctas > 0 && make_plan(b, d_out, d_in, r, ctas, &pl);
+}
+
+size_t decode_tiled_workspace_bytes(int b, int d_out, int d_in, int r) {
+    Plan pl;
+    const int ctas = grid_ctas();
+    if (ctas < 1 || !make_plan(b, d_out, d_in, r, ctas, &pl)) return 0;
+    return kTfinalBytes + pl.p_bytes + pl.a_bytes + pl.t_bytes;
+}
+
+slim_status_t launch_decode_tiled(const __nv_bfloat16* X, int b, const uint8_t* W, float s, const __nv_bfloat16* L,
+                                  const __nv_bfloat16* R, int r, int d_out, int d_in, __nv_bfloat16* Y, void* ws,
+                                  uint32_t* status_dev, cudaStream_t st)
+{
+    slim_status_t err;
+    const DeviceInfo* di = device_info(&err);
+    if (!di) return err;
+    Plan pl;
+    const int ctas = grid_ctas();
+    if (ctas < 1 || !make_plan(b, d_out, d_in, r, ctas, &pl)) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    Params p;
+    p.X = X; p.W = W; p.Y = Y;
+    char* base = reinterpret_cast<char*>(ws);
+    p.departures = reinterpret_cast<unsigned long long*>(base);
+    p.Tfinal = reinterpret_cast<unsigned long long*>(base + SLIM_WORKSPACE_SYNC_BYTES);
+    p.Ppart = reinterpret_cast<uint32_t*>(base + SLIM_WORKSPACE_SYNC_BYTES + kTfinalBytes);
+    p.Apart = reinterpret_cast<uint32_t*>(base + SLIM_WORKSPACE_SYNC_BYTES + kTfinalBytes + pl.p_bytes);
+    p.Tpart = reinterpret_cast<uint32_t*>(base + SLIM_WORKSPACE_SYNC_BYTES + kTfinalBytes + pl.p_bytes + pl.a_bytes);
+    p.status = status_dev;
+    p.s = s; p.b = b; p.r = r; p.d_out = d_out; p.d_in = d_in;
+    p.KS = pl.KS; p.G = pl.G; p.nblk = pl.nblk; p.NB = pl.nb;
+    p.unitsW = pl.unitsW; p.tilesW = pl.tilesW; p.tilesR = pl.tilesR; p.nqL = pl.nqL;
+    p.wnR = pl.wnR; p.muW = pl.muW; p.muR = pl.muR; p.muL = pl.muL;
+    p.ring = pl.ring; p.slot_bytes = pl.slot_bytes; p.x_bytes = pl.x_bytes;
+    CUtensorMap tmR, tmL;
+    if (r > 0) {
+        if (!make_tile_map(&tmR, R, (uint64_t)d_in, (uint64_t)r) || !make_tile_map(&tmL, L, (uint64_t)r, (uint64_t)d_out))
+            return SLIM_ERR_CUDA;
+    } else {
+        memset(&tmR, 0, sizeof tmR); memset(&tmL, 0, sizeof tmL);      // never used when r == 0
+    }
+    void* args[] = {&p, &tmR, &tmL};
+    const dim3 grid(ctas), block(kThreads);
+    const void* fn = nullptr;
+    if (pl.nt == 1) fn = pl.mt == 1 ? (const void*)decode_tiled_kernel<1, 1> : (const void*)decode_tiled_kernel<1, 2>;
+    else fn = pl.mt == 1 ? (const void*)decode_tiled_kernel<2, 1> : pl.mt == 2 ? (const void*)decode_tiled_kernel<2, 2>
+                                                                                : (const void*)decode_tiled_kernel<2, 4>;
+    const cudaError_t e = cudaLaunchCooperativeKernel(fn, grid, block, args, pl.smem, st);
+    count_launch(1);
+    return e == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+}
+
+}  // namespace slim
+
+#ifdef SLIM_TILED_TRACE
+extern "C" int slim_debug_read_tiled_dbg(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, slim::g_tiled_dbg, sizeof(slim::g_tiled_dbg));
+}
+extern "C" int slim_debug_read_tiled_trace(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, slim::g_tiled_trace, sizeof(slim::g_tiled_trace));
+}
+#endif

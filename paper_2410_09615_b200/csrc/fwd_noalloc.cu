@@ -34,6 +34,13 @@ static bool is_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p)
 
 using namespace slim;
 
+extern "C" size_t slim_noalloc_scratch_needed(int b, int d_out, int d_in, int r)
+{
+    if (b < 1 || b > 16 || r < 0 || d_out < 1 || d_in < 1 || d_in % 64 != 0 || d_out % 16 != 0 || r % 16 != 0) return 0;
+    const size_t need = decode_workspace_bytes(b, d_out, d_in, r);
+    return need ? SLIM_WORKSPACE_SYNC_BYTES + need : 0;
+}
+
 extern "C" slim_status_t slim_linear_fwd_noalloc(const void* X, int b, const uint8_t* vals,
                                                  const uint8_t* meta, float s, const void* L,
                                                  const void* R, int r, int d_out, int d_in, void* Y,

@@ -44,6 +44,7 @@
 // is requested ~600 ns after the MMAs that free the slot were issued and lands ~900 ns later, over
 // the 5 stages that fit in shared memory.
 // Every wait is bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on.
+#include <atomic>
 #include <cuda.h>
 #include "common.cuh"
 
@@ -613,22 +614,10 @@ typedef CUresult (*PfEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-static PfEncodeTiledFn pf_encode_fn() {
-    static PfEncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<PfEncodeTiledFn>(ptr);
-    }
-    return fn;
-}
-
 // Row-major 2-D tensor [rows][row_elems]; box of box_rows x box_elems elements.
 static bool pf_map(CUtensorMap* map, const void* base, CUtensorMapDataType type, int esize, uint64_t row_elems,
                    uint64_t rows, int box_elems, int box_rows, int swizzle_bytes) {
-    PfEncodeTiledFn fn = pf_encode_fn();
+    PfEncodeTiledFn fn = reinterpret_cast<PfEncodeTiledFn>(tensor_map_encoder());
     if (!fn) return false;
     cuuint64_t dims[2] = {row_elems, rows};
     cuuint64_t strides[1] = {row_elems * (uint64_t)esize};
@@ -652,7 +641,7 @@ size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r) {
     return tq + (pl.slices > 1 ? (size_t)pl.slices * b * r * sizeof(float) : 0);
 }
 
-static bool g_prefill_attr_set[64];
+static std::atomic<bool> g_prefill_attr_set[64];   // attributes set once per device (setting them twice is harmless)
 
 template <int N, bool TWO, bool PRE = false>
 static slim_status_t launch_tile_kernel(const PrefillParams& q, int m_rows, const CUtensorMap& tmV, const CUtensorMap& tmM,
@@ -683,14 +672,14 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     if (!prefill_supports(b, d_out, d_in, r)) return SLIM_ERR_UNSUPPORTED_SHAPE;
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !g_prefill_attr_set[dev]) {
+    if (dev >= 0 && dev < 64 && !g_prefill_attr_set[dev].load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(prefill_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256, true>::kSmem) != cudaSuccess ||
             cudaFuncSetAttribute(prefill_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256, false>::kSmem) != cudaSuccess ||
             cudaFuncSetAttribute(prefill_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<64, false>::kSmem) != cudaSuccess ||
             cudaFuncSetAttribute(prefill_kernel<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<64, false, true>::kSmem) != cudaSuccess ||
             cudaFuncSetAttribute(prefill_kernel<256, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PfCfg<256, false, true>::kSmem) != cudaSuccess)
             return SLIM_ERR_CUDA;
-        g_prefill_attr_set[dev] = true;
+        g_prefill_attr_set[dev].store(true, std::memory_order_release);
     }
     __nv_bfloat16* Tq = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + SLIM_WORKSPACE_SYNC_BYTES);
     const float s_eff = s != 0.f ? s : 1.f;       // with s == 0 only the adapter term remains
@@ -742,9 +731,15 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     p.scale = s_eff; p.status = status_dev; p.part = nullptr; p.k_per = 0;
     if (p.n1 + p.n2 == 0)             // s == 0 and no adapters: the result is zero
         return cudaMemsetAsync(Y, 0, (size_t)b * d_out * 2, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
-    if (!wide) return launch_tile_kernel<64, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
-    return pair ? launch_tile_kernel<256, true>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st)
-                                  : launch_tile_kernel<256, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
+    slim_status_t rc;
+    if (!wide) rc = launch_tile_kernel<64, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
+    else rc = pair ? launch_tile_kernel<256, true>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st)
+                   : launch_tile_kernel<256, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
+    if (rc != SLIM_OK) return rc;
+    // T' and the partial tiles were written where the decode kernels keep their hand-over slots
+    // (all ones = empty): leave the region as they expect it.
+    if (r > 0 && cudaMemsetAsync(Tq, 0xFF, prefill_workspace_bytes(b, d_out, d_in, r), st) != cudaSuccess) return SLIM_ERR_CUDA;
+    return SLIM_OK;
 }
 
 }  // namespace slim

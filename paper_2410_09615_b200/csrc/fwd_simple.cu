@@ -90,7 +90,10 @@ slim_status_t launch_simple(const __nv_bfloat16* X, int b, const uint8_t* vals, 
     simple_y_kernel<<<(int)(blocks < cap ? blocks : cap), 256, 0, st>>>(X, vals, meta, s, L, T, b, r,
                                                                       d_out, d_in, Y);
     count_launch(1);
-    return cudaGetLastError() == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return SLIM_ERR_CUDA;
+    // The decode kernels read this region as hand-over slots (all ones = empty): leave it as they expect it.
+    if (r > 0 && cudaMemsetAsync(T, 0xFF, (size_t)b * r * sizeof(float), st) != cudaSuccess) return SLIM_ERR_CUDA;
+    return SLIM_OK;
 }
 
 }  // namespace slim

@@ -63,6 +63,23 @@ def test_host_side_argument_checks_need_no_device(lib):
     assert lib.slim_pack(one + 4, one, 16, 64, one, one, None, None) == binding.SLIM_ERR_INVALID_ARG
 
 
+def test_tiled_entry_points_host_logic(lib):
+    assert binding.slim_tiled_bytes(4096, 4096) == 4096 * 4096 * 3 // 8
+    assert binding.slim_tiled_bytes(4096, 4096, 2) == 0           # unknown layout
+    assert binding.slim_tiled_bytes(4100, 4096) == 0 and binding.slim_tiled_bytes(4096, 4160) == 0
+    one = 16
+    assert lib.slim_repack_tiled(None, None, 16, 256, 1, None, None) == binding.SLIM_ERR_INVALID_ARG
+    assert lib.slim_repack_tiled(one, one, 16, 320, 1, one, None) == binding.SLIM_ERR_UNSUPPORTED_SHAPE
+    assert lib.slim_linear_fwd_tiled(None, 1, None, 1, 1.0, None, None, 0, 16, 256, None, None, 0, None,
+                                     None) == binding.SLIM_ERR_INVALID_ARG
+    # a scale that is not finite is an argument error, before any device work
+    for bad in (float("nan"), float("inf"), -float("inf")):
+        assert lib.slim_linear_fwd(one, 1, one, one, bad, None, None, 0, 16, 64, one, one, 1 << 20, None,
+                                   None) == binding.SLIM_ERR_INVALID_ARG
+        assert lib.slim_linear_fwd_tiled(one, 1, one, 1, bad, None, None, 0, 16, 256, one, one, 1 << 20, None,
+                                         None) == binding.SLIM_ERR_INVALID_ARG
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libslim.so")

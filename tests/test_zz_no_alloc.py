@@ -27,11 +27,13 @@ def test_noalloc_rejects_problems_beyond_its_scratch_on_the_host():
                                        None) == K.SLIM_ERR_UNSUPPORTED_SHAPE
     assert lib.slim_linear_fwd_noalloc(None, 4, fake, fake, 1.0, None, None, 0, 512, 512, fake, None,
                                        None) == K.SLIM_ERR_INVALID_ARG
+    assert K.slim_noalloc_scratch_needed(16, 65536, 28672, 64) > K.NOALLOC_SCRATCH_BYTES      # the case refused above
+    assert K.slim_noalloc_scratch_needed(17, 512, 512, 0) == 0 and K.slim_noalloc_scratch_needed(4, 512, 320, 0) == 0
     # every LLaMA-2 layer shape of the workload table fits the array
     for model in inputs.LLAMA2_SHAPES.values():
         for _name, d_in, d_out, _n in model:
             r = inputs.rank_for_ratio(0.2, d_in, d_out)
-            assert 0 < K.slim_workspace_bytes(16, d_out, d_in, r) <= K.NOALLOC_SCRATCH_BYTES
+            assert 0 < K.slim_noalloc_scratch_needed(16, d_out, d_in, r) <= K.NOALLOC_SCRATCH_BYTES
 
 
 @pytest.mark.gpu
