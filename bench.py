@@ -3,27 +3,30 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-Workload: the LLaMA-2-7B decode layer set.  One step = the seven linears of one
-transformer block (4 x 4096->4096, 2 x 4096->11008, 1 x 11008->4096; int4 2:4
-weights, per-layer fp32 scale, rank-416 bf16 adapters) run once at batch 1 and
-once at batch 16: 14 calls of slim_linear_fwd.  Two full sets of packed weights
-and adapters (141 MB each) alternate, so 282 MB stream through the 126 MB L2
-between two uses of the same bytes and every call reads its weights from HBM.
-The step is captured in a CUDA graph and replayed; time is taken with CUDA
-events on the launching stream, max over ranks.  Prints one JSON line.
+Workload: the LLaMA-2-70B decode layer set, the largest configuration that fits one GPU.  One
+step = the seven linears of one transformer block (2 x 8192->8192, 2 x 8192->1024 grouped-query
+k/v, 2 x 8192->28672, 1 x 28672->8192; int4 2:4 weights, per-layer fp32 scale, bf16 adapters of
+rank 0.1 x the smaller dimension) run once at batch 1 and once at batch 16: 14 calls of
+slim_linear_fwd_tiled on the decode-tiled weights (repacked once, outside the timed region).
+Every linear has its own copy of weight and adapters; the set is 563 MB, so each call reads its
+operands from HBM (the L2 holds 126 MB).  The step is captured in a CUDA graph and replayed; time
+is taken with CUDA events on the launching stream, max over ranks.  Prints one JSON line, which
+also carries per-case tables for the 7B / 13B / 70B shapes, prefill tables (2048 and 4096 tokens,
+rank sweep on the 70B shapes), an end-to-end figure through the host-buffer entry point and the CPU
+oracle timed on this machine.
 
-With N > 1 every rank runs the same step on its own GPU (independent replicas,
-no collective on the data path).
+With N > 1 every rank runs the same step on its own GPU (independent replicas, no collective on
+the data path).
 
---impl reference times the CPU oracle (oracle/) on this machine's host cores on the
-same workload: each step runs each distinct (shape, batch) call once and
-weights it by how often the block uses it.
+--impl reference times the CPU oracle (oracle/) on this machine's host cores on the same workload:
+each step runs each distinct (shape, batch) call once and weights it by how often the block uses it.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import subprocess
 import sys
 import threading
 import time
@@ -37,19 +40,19 @@ from paper_2410_09615_b200 import inputs  # noqa: E402
 
 METRIC = "slim_linear_us_per_call"
 UNIT = "us/call"
-WORKLOAD = "llama2_7b_decode_layer_set"
+MODEL = "70b"
+WORKLOAD = "llama2_70b_decode_layer_set"
 BATCHES = (1, 16)
-SHAPES = inputs.LLAMA2_SHAPES["7b"]            # (name, d_in, d_out, count per block)
+SHAPES = inputs.LLAMA2_SHAPES[MODEL]           # (name, d_in, d_out, count per block)
 CALLS_PER_STEP = sum(c for *_x, c in SHAPES) * len(BATCHES)
 HBM_FALLBACK_GBS = 6650.0                      # an earlier copy-bandwidth measurement on B200
 NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126e6
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel launch divided by
-# the call's algorithmic bytes, from an ncu capture of the (4096, 11008, 416, 16)
-# case (its summary is kept with the other profiler summaries): 29.80 MB / 29.96 MB.
-# Traffic grows in proportion to the bytes streamed, so the bench scales it to its
-# own launches.  Set to None whenever decode_kernel changes after the capture.
-NCU_TRAFFIC_RATIO = 0.995
+# DRAM traffic of one launch of the dominant kernel relative to the call's algorithmic bytes, from an
+# ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) whose summary is kept with the other
+# profiler summaries.  None = no capture of the current kernel: the bench then reports traffic null.
+NCU_TRAFFIC = None     # e.g. {"ratio": 1.0, "source": "profiles/<file>", "case": "d_in,d_out,r,b"}
 
 
 def algorithmic_bytes(d_in, d_out, r, b):
@@ -62,6 +65,10 @@ def executed_flops(d_in, d_out, r, b):
     return 2.0 * b * d_out * d_in / 2.0 + 2.0 * b * r * (d_in + d_out)
 
 
+def dense_equiv_flops(d_in, d_out, r, b):
+    return 2.0 * b * d_out * d_in + 2.0 * b * r * (d_in + d_out)
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -69,6 +76,15 @@ def measured_peaks():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return HBM_FALLBACK_GBS, "fallback"
+
+
+def dense_tflops_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
 
 
 # ------------------------------------------------------------------ clocks
@@ -143,20 +159,50 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ host data
-def host_layers():
-    """The three distinct layers of the block, generated once on the host."""
+def host_layers(model=MODEL, ratio=0.1, cfg=4, batches=BATCHES):
+    """The distinct layers of one block of `model`, generated once on the host with the recipe of
+    paper_2410_09615_b200/inputs.py."""
     out = []
-    for li, (name, d_in, d_out, count) in enumerate(SHAPES):
-        r = inputs.default_rank(d_in, d_out)
-        wseed = 1000 + 10 * li
+    for li, (name, d_in, d_out, count) in enumerate(inputs.LLAMA2_SHAPES[model]):
+        r = inputs.rank_for_ratio(ratio, d_in, d_out)
+        wseed = 1000 * cfg + 10 * li
         s, codes, mask = inputs.make_weights(d_out, d_in, wseed)
         L, R = inputs.make_adapters(d_out, d_in, r, wseed)
         out.append(dict(name=name, d_in=d_in, d_out=d_out, r=r, count=count, s=s, codes=codes, mask=mask,
-                        L=L, R=R, X={b: inputs.make_activations(b, d_in, wseed + bi) for bi, b in enumerate(BATCHES)}))
+                        L=L, R=R, X={b: inputs.make_activations(b, d_in, wseed + bi) for bi, b in enumerate(batches)}))
     return out
 
 
+def cpu_model():
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except Exception:
+        pass
+    return "unknown"
+
+
 # ------------------------------------------------------------------ reference arm
+def oracle_step(layers, oracle):
+    """One pass of the oracle over each distinct (layer shape, batch) pair; returns the time of the whole
+    block (each pair weighted by the number of such linears) and the raw wall time."""
+    t_weighted, t_raw = 0.0, 0.0
+    for ly in layers:
+        for b in BATCHES:
+            t0 = time.perf_counter()
+            oracle.linear_fwd(ly["X"][b], ly["ovals"], ly["ometa"], ly["s"], ly["L"], ly["R"])
+            dt = time.perf_counter() - t0
+            t_raw += dt
+            t_weighted += dt * ly["count"]
+    return t_weighted, t_raw
+
+
+SAMPLE_TEXT = ("each step runs the oracle once per distinct (layer shape, batch) pair of the block, all token rows and all "
+               "output columns, and weights the time by the number of such linears in the block (2/2/2/1)")
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -164,30 +210,19 @@ def run_reference(args):
     import oracle
     layers = host_layers()
     for ly in layers:
-        ly["vals"], ly["meta"] = oracle.pack(ly["codes"], ly["mask"])
-
-    def step():
-        t_weighted = 0.0
-        for ly in layers:
-            for b in BATCHES:
-                t0 = time.perf_counter()
-                oracle.linear_fwd(ly["X"][b], ly["vals"], ly["meta"], ly["s"], ly["L"], ly["R"])
-                t_weighted += (time.perf_counter() - t0) * ly["count"]
-        return t_weighted
-
+        ly["ovals"], ly["ometa"] = oracle.pack(ly["codes"], ly["mask"])
+        del ly["codes"], ly["mask"]
     for _ in range(args.warmup):
-        step()
-    total = sum(step() for _ in range(args.steps))
+        oracle_step(layers, oracle)
+    total = sum(oracle_step(layers, oracle)[0] for _ in range(args.steps))
     ms_per_step = 1e3 * total / args.steps
     value = 1e3 * ms_per_step / CALLS_PER_STEP
-    sample = ("each step runs the oracle once per distinct (layer shape, batch) pair, all token rows, "
-              "and weights the time by the number of such linears in the block (4/2/1)")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": WORKLOAD, "batches": list(BATCHES), "calls_per_step": CALLS_PER_STEP},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                             "sample": sample},
+                             "sample": SAMPLE_TEXT, "cpu": cpu_model()},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
     return 0
@@ -212,50 +247,43 @@ def run_ours(args):
     build.build()
     lib = K.lib()
     dev = torch.device("cuda", local)
+    P = ctypes.c_void_p
 
-    # ---- weights: packed on the GPU by slim_pack, two full sets of the block
+    # ---- weights: packed by slim_pack and repacked by slim_repack_tiled on the GPU; one copy per linear
     layers = host_layers()
-    n_sets = 2
-    slots = []            # one entry per linear of the block and per set
     for ly in layers:
         codes_d, mask_d = torch.from_numpy(ly["codes"]).to(dev), torch.from_numpy(ly["mask"]).to(dev)
-        vals, meta = K.slim_pack(codes_d, mask_d)
-        del codes_d, mask_d
-        ly["vals"], ly["meta"] = vals, meta
+        ly["vals"], ly["meta"] = K.slim_pack(codes_d, mask_d)
+        del codes_d, mask_d, ly["codes"], ly["mask"]
+        ly["tiled"] = K.slim_repack_tiled(ly["vals"], ly["meta"])
         ly["Ld"], ly["Rd"] = K.bf16_from_bits(ly["L"], dev), K.bf16_from_bits(ly["R"], dev)
         ly["Xd"] = {b: K.bf16_from_bits(ly["X"][b], dev) for b in BATCHES}
         ly["Yd"] = {b: torch.empty((b, ly["d_out"]), dtype=torch.bfloat16, device=dev) for b in BATCHES}
-        ly["copies"] = [[(vals.clone(), meta.clone(), ly["Ld"].clone(), ly["Rd"].clone())
-                         for _ in range(ly["count"])] for _ in range(n_sets)]
+        ly["copies"] = [(ly["tiled"].clone(), ly["Ld"].clone(), ly["Rd"].clone()) for _ in range(ly["count"])]
     ws_bytes = max(K.slim_workspace_bytes(b, ly["d_out"], ly["d_in"], ly["r"]) for ly in layers for b in BATCHES)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     K.slim_workspace_reset(ws)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    set_bytes = sum(c[0].numel() + c[1].numel() + 2 * c[2].numel() + 2 * c[3].numel()
-                    for ly in layers for c in ly["copies"][0])
+    set_bytes = sum(c[0].numel() + 2 * c[1].numel() + 2 * c[2].numel() for ly in layers for c in ly["copies"])
+    torch.cuda.synchronize()
 
-    fwd = lib.slim_linear_fwd
-    P = ctypes.c_void_p
+    fwd = lib.slim_linear_fwd_tiled
 
     def call_args(ly, b, copy):
-        vals, meta, L, R = copy
-        return (P(ly["Xd"][b].data_ptr()), b, P(vals.data_ptr()), P(meta.data_ptr()), ctypes.c_float(ly["s"]),
+        tiled, L, R = copy
+        return (P(ly["Xd"][b].data_ptr()), b, P(tiled.data_ptr()), K.LAYOUT_DECODE_TILED, ctypes.c_float(ly["s"]),
                 P(L.data_ptr()), P(R.data_ptr()), ly["r"], ly["d_out"], ly["d_in"], P(ly["Yd"][b].data_ptr()),
                 P(ws.data_ptr()), ws_bytes, P(status.data_ptr()))
 
-    # the 14 calls of one step: batch 1 on weight set 0, batch 16 on weight set 1
-    step_calls = []
-    for si, b in enumerate(BATCHES):
-        for ly in layers:
-            for copy in ly["copies"][si % n_sets]:
-                step_calls.append((ly, b, call_args(ly, b, copy)))
+    # the 14 calls of one step: the block at batch 1, then the block at batch 16
+    step_calls = [(ly, b, call_args(ly, b, copy)) for b in BATCHES for ly in layers for copy in ly["copies"]]
     assert len(step_calls) == CALLS_PER_STEP
 
     def issue_step(stream_ptr):
         for _ly, _b, a in step_calls:
             rc = fwd(*a, stream_ptr)
             if rc != 0:
-                raise RuntimeError(f"slim_linear_fwd failed: {K.strerror(rc)}")
+                raise RuntimeError(f"slim_linear_fwd_tiled failed: {K.strerror(rc)}")
 
     stream = torch.cuda.Stream(device=dev)
     sp = P(stream.cuda_stream)
@@ -322,28 +350,50 @@ def run_ours(args):
     step_bytes = sum(algorithmic_bytes(ly["d_in"], ly["d_out"], ly["r"], b) for ly, b, _ in step_calls)
     peak, peak_kind = measured_peaks()
     achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
-    traffic = None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * step_bytes / len(step_calls)
-    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    traffic = None if NCU_TRAFFIC is None else NCU_TRAFFIC["ratio"] * step_bytes / len(step_calls)
+    roofline = {"bound": "hbm", "kernel": "decode_tiled_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "traffic": traffic, "bytes_per_launch": step_bytes / len(step_calls),
-                "avg_launch_us": 1e3 * ms_per_step / len(step_calls)}
+                "traffic": traffic,
+                "traffic_kind": None if NCU_TRAFFIC is None else
+                f"scaled by bytes from {NCU_TRAFFIC['source']}, case {NCU_TRAFFIC['case']}",
+                "bytes_per_launch": step_bytes / len(step_calls), "avg_launch_us": 1e3 * ms_per_step / len(step_calls)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "batches": list(BATCHES), "calls_per_step": CALLS_PER_STEP,
                        "layers": [[ly["name"], ly["d_in"], ly["d_out"], ly["r"], ly["count"]] for ly in layers],
-                       "l2": f"inputs larger than L2: {n_sets} weight sets of {set_bytes / 1e6:.0f} MB alternate",
+                       "weight_format": "decode-tiled (slim_repack_tiled, once, outside the timed region)",
+                       "l2": f"inputs larger than L2: every linear has its own copy, {set_bytes / 1e6:.0f} MB per step pass",
                        "launch": launch_mode, "parallelism": f"replicas x{world}"},
             "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
             "clocks": sampler.summary()}
 
-    if rank == 0 and not args.skip_extras:
-        line["per_case"] = per_case_table(K, lib, layers, ws, ws_bytes, status, stream, peak)
-        line["prefill"] = prefill_table(K, layers, stream)
-        line["pack"] = time_pack(K, layers[1], stream)
     # ---- end to end through the host-buffer entry point
     line["e2e"] = time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, world, barrier)
+    if rank == 0 and not args.skip_extras:
+        tables, prefill_rows = [], []
+        tables += per_case_table(K, lib, layers, "70b", ws, ws_bytes, status, stream, peak)
+        prefill_rows += prefill_table(K, layers, "70b", stream, 4096, sweep=True)
+        host70 = layers
+        for model, cfg in (("7b", 1), ("13b", 3)):
+            small = host_layers(model, 0.1, cfg)
+            for ly in small:
+                ly["vals"], ly["meta"] = K.slim_pack(torch.from_numpy(ly["codes"]).to(dev), torch.from_numpy(ly["mask"]).to(dev))
+                del ly["codes"], ly["mask"]
+                ly["tiled"] = K.slim_repack_tiled(ly["vals"], ly["meta"])
+                ly["Ld"], ly["Rd"] = K.bf16_from_bits(ly["L"], dev), K.bf16_from_bits(ly["R"], dev)
+                ly["Xd"] = {b: K.bf16_from_bits(ly["X"][b], dev) for b in BATCHES}
+                ly["Yd"] = {b: torch.empty((b, ly["d_out"]), dtype=torch.bfloat16, device=dev) for b in BATCHES}
+            wsb = max(K.slim_workspace_bytes(b, ly["d_out"], ly["d_in"], ly["r"]) for ly in small for b in BATCHES)
+            ws2 = ws if wsb <= ws_bytes else K.new_workspace(16, max(l["d_out"] for l in small), max(l["d_in"] for l in small), small[0]["r"])
+            tables += per_case_table(K, lib, small, model, ws2, ws2.numel(), status, stream, peak)
+            prefill_rows += prefill_table(K, small, model, stream, 2048)
+            del small
+        line["per_case"] = tables
+        line["prefill"] = prefill_rows
+        line["roofline_prefill"] = prefill_roofline(prefill_rows)
+        line["pack"] = time_pack(K, host70[0], stream)
     if rank == 0 and world == 1 and not args.skip_cpu:
         line["cpu_baseline"] = time_cpu_baseline(layers)
     if rank == 0:
@@ -353,8 +403,8 @@ def run_ours(args):
     return 0
 
 
-def time_graph_of_calls(lib, calls, stream, replays=20):
-    """Median per-call time (us) of a CUDA graph holding `calls`, replayed."""
+def time_graph_of_calls(fn, calls, stream, replays=10):
+    """Median per-call time (us) of a CUDA graph holding `calls` of the C function `fn`, replayed."""
     import ctypes
     import torch
     P = ctypes.c_void_p
@@ -362,7 +412,7 @@ def time_graph_of_calls(lib, calls, stream, replays=20):
     with torch.cuda.graph(g, stream=stream):
         cur = P(torch.cuda.current_stream().cuda_stream)
         for a in calls:
-            lib.slim_linear_fwd(*a, cur)
+            fn(*a, cur)
     times = []
     with torch.cuda.stream(stream):
         for _ in range(3):
@@ -377,101 +427,124 @@ def time_graph_of_calls(lib, calls, stream, replays=20):
     return float(np.median(times)), float(np.min(times))
 
 
-def per_case_table(K, lib, layers, ws, ws_bytes, status, stream, peak):
-    """Per (layer, batch): us/call over rotating weight copies (> 2x L2 between
+def per_case_table(K, lib, layers, model, ws, ws_bytes, status, stream, peak):
+    """Per (layer, batch): us/call of slim_linear_fwd_tiled over rotating copies (> 2x L2 between
     reuses), algorithmic GB/s and fraction of the HBM roofline."""
     import ctypes
+    import torch
     P = ctypes.c_void_p
     rows = []
     for ly in layers:
-        per_copy = ly["vals"].numel() + ly["meta"].numel() + 2 * ly["Ld"].numel() + 2 * ly["Rd"].numel()
-        n_copies = int(np.ceil(2 * 126e6 / per_copy)) + 1
-        copies = [(ly["vals"].clone(), ly["meta"].clone(), ly["Ld"].clone(), ly["Rd"].clone()) for _ in range(n_copies)]
+        per_copy = ly["tiled"].numel() + 2 * ly["Ld"].numel() + 2 * ly["Rd"].numel()
+        n_copies = int(np.ceil(2 * L2_BYTES / per_copy)) + 1
+        copies = [(ly["tiled"].clone(), ly["Ld"].clone(), ly["Rd"].clone()) for _ in range(n_copies)]
+        torch.cuda.synchronize()
         for b in BATCHES:
-            calls = [(P(ly["Xd"][b].data_ptr()), b, P(c[0].data_ptr()), P(c[1].data_ptr()), ctypes.c_float(ly["s"]),
-                      P(c[2].data_ptr()), P(c[3].data_ptr()), ly["r"], ly["d_out"], ly["d_in"],
+            calls = [(P(ly["Xd"][b].data_ptr()), b, P(c[0].data_ptr()), K.LAYOUT_DECODE_TILED, ctypes.c_float(ly["s"]),
+                      P(c[1].data_ptr()), P(c[2].data_ptr()), ly["r"], ly["d_out"], ly["d_in"],
                       P(ly["Yd"][b].data_ptr()), P(ws.data_ptr()), ws_bytes, P(status.data_ptr()))
                      for c in copies] * 3
             try:
-                med, best = time_graph_of_calls(lib, calls, stream)
+                med, best = time_graph_of_calls(lib.slim_linear_fwd_tiled, calls, stream)
             except Exception as e:
-                rows.append({"layer": ly["name"], "b": b, "error": str(e)[:80]})
+                rows.append({"model": model, "layer": ly["name"], "b": b, "error": str(e)[:80]})
                 continue
             nbytes = algorithmic_bytes(ly["d_in"], ly["d_out"], ly["r"], b)
             gbs = nbytes / (med * 1e-6) / 1e9
-            rows.append({"layer": ly["name"], "d_in": ly["d_in"], "d_out": ly["d_out"], "r": ly["r"], "b": b,
+            rows.append({"model": model, "layer": ly["name"], "d_in": ly["d_in"], "d_out": ly["d_out"], "r": ly["r"], "b": b,
                          "us": round(med, 3), "us_min": round(best, 3), "GBs": round(gbs, 1),
                          "frac_measured": round(gbs / peak, 4), "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
-                         "executed_TFLOPs": round(executed_flops(ly["d_in"], ly["d_out"], ly["r"], b) / (med * 1e-6) / 1e12, 2)})
+                         "roofline_us": round(nbytes / peak / 1e3, 3)})
         del copies
     return rows
 
 
-def dense_tflops_peak():
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    try:
-        with open(path) as f:
-            return float(json.load(f)["bf16_tflops"]), "measured"
-    except Exception:
-        return 1590.0, "fallback"
-
-
-def prefill_table(K, layers, stream, tokens=2048):
-    """The same three layers at 2048 tokens (tcgen05 prefill kernel): us/call,
-    dense-equivalent TFLOP/s (the 2:4 product counted as if dense, adapters at
-    face value) and its fraction of the sparse bf16 peak, taken as twice the
-    measured dense bf16 peak."""
+def prefill_table(K, layers, model, stream, tokens, sweep=False):
+    """The layers of one model at `tokens` tokens (tcgen05 prefill kernel on the packed weight): us/call,
+    dense-equivalent TFLOP/s (the 2:4 product counted as if dense, adapters at face value) and its
+    fraction of the sparse bf16 peak, taken as twice the measured dense bf16 peak.  `sweep`: ranks of
+    0, 0.05, 0.1 and 0.2 x the smaller dimension instead of 0.1 only."""
     import torch
     dense_peak, kind = dense_tflops_peak()
     rows = []
     for ly in layers:
         X = K.bf16_from_bits(inputs.make_activations(tokens, ly["d_in"], 7))
         Y = torch.empty((tokens, ly["d_out"]), dtype=torch.bfloat16, device=X.device)
-        ws = K.new_workspace(tokens, ly["d_out"], ly["d_in"], ly["r"])
-        with torch.cuda.stream(stream):
-            for _ in range(3):
-                K.slim_linear_fwd(X, ly["vals"], ly["meta"], ly["s"], ly["Ld"], ly["Rd"], Y=Y, workspace=ws)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n = 20
-            e0.record(stream)
-            for _ in range(n):
-                K.slim_linear_fwd(X, ly["vals"], ly["meta"], ly["s"], ly["Ld"], ly["Rd"], Y=Y, workspace=ws)
-            e1.record(stream)
-            e1.synchronize()
-        us = 1e3 * e0.elapsed_time(e1) / n
-        dense_eq = 2.0 * tokens * ly["d_out"] * ly["d_in"] + 2.0 * tokens * ly["r"] * (ly["d_in"] + ly["d_out"])
-        tf = dense_eq / (us * 1e-6) / 1e12
-        rows.append({"layer": ly["name"], "d_in": ly["d_in"], "d_out": ly["d_out"], "r": ly["r"], "tokens": tokens,
-                     "kernel": K.KERNEL_NAMES[K.slim_select_kernel(tokens, ly["d_out"], ly["d_in"], ly["r"])],
-                     "us": round(us, 2), "dense_equiv_TFLOPs": round(tf, 1),
-                     "executed_TFLOPs": round(executed_flops(ly["d_in"], ly["d_out"], ly["r"], tokens) / (us * 1e-6) / 1e12, 1),
-                     "frac_of_sparse_peak": round(tf / (2 * dense_peak), 4), "sparse_peak_TFLOPs": 2 * dense_peak,
-                     "peak_kind": f"2 x dense bf16 of {kind}", "frac_of_nominal_4500": round(tf / 4500.0, 4)})
-        del X, Y, ws
+        for ratio in ((0.0, 0.05, 0.1, 0.2) if sweep else (0.1,)):
+            r = inputs.rank_for_ratio(ratio, ly["d_in"], ly["d_out"])
+            if r == ly["r"]:
+                Ld, Rd = ly["Ld"], ly["Rd"]
+            elif r == 0:
+                Ld = Rd = None
+            else:
+                Lh, Rh = inputs.make_adapters(ly["d_out"], ly["d_in"], r, 77)
+                Ld, Rd = K.bf16_from_bits(Lh), K.bf16_from_bits(Rh)
+            ws = K.new_workspace(tokens, ly["d_out"], ly["d_in"], r)
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    K.slim_linear_fwd(X, ly["vals"], ly["meta"], ly["s"], Ld, Rd, Y=Y, workspace=ws)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                n = 10
+                e0.record(stream)
+                for _ in range(n):
+                    K.slim_linear_fwd(X, ly["vals"], ly["meta"], ly["s"], Ld, Rd, Y=Y, workspace=ws)
+                e1.record(stream)
+                e1.synchronize()
+            us = 1e3 * e0.elapsed_time(e1) / n
+            tf = dense_equiv_flops(ly["d_in"], ly["d_out"], r, tokens) / (us * 1e-6) / 1e12
+            rows.append({"model": model, "layer": ly["name"], "d_in": ly["d_in"], "d_out": ly["d_out"], "r": r, "tokens": tokens,
+                         "kernel": K.KERNEL_NAMES[K.slim_select_kernel(tokens, ly["d_out"], ly["d_in"], r)],
+                         "us": round(us, 2), "dense_equiv_TFLOPs": round(tf, 1),
+                         "executed_TFLOPs": round(executed_flops(ly["d_in"], ly["d_out"], r, tokens) / (us * 1e-6) / 1e12, 1),
+                         "frac_of_sparse_peak": round(tf / (2 * dense_peak), 4), "sparse_peak_TFLOPs": 2 * dense_peak,
+                         "peak_kind": f"2 x dense bf16 of {kind}", "frac_of_nominal_4500": round(tf / 4500.0, 4)})
+            del ws
+        del X, Y
     return rows
 
 
+def prefill_roofline(rows):
+    """One structured entry for the prefill kernel: the 2048-token 7B rows at rank 0.1 taken together
+    (dense-equivalent flops of the three shapes / their summed time)."""
+    sel = [r for r in rows if r.get("model") == "7b" and "us" in r]
+    if not sel:
+        return None
+    flops = sum(dense_equiv_flops(r["d_in"], r["d_out"], r["r"], r["tokens"]) for r in sel)
+    us = sum(r["us"] for r in sel)
+    peak = sel[0]["sparse_peak_TFLOPs"]
+    ach = flops / (us * 1e-6) / 1e12
+    return {"bound": "tensor", "kernel": "prefill_kernel", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+            "peak_kind": sel[0]["peak_kind"], "workload": "llama2_7b layer shapes, 2048 tokens, rank 416 (one call per distinct shape)",
+            "traffic": None, "flops": "dense-equivalent: 2 b d_in d_out + 2 b r (d_in + d_out)"}
+
+
 def time_pack(K, ly, stream):
+    """slim_pack and slim_repack_tiled of one layer (offline steps, outside the per-call metric)."""
     import torch
-    codes, mask = torch.from_numpy(ly["codes"]).cuda(), torch.from_numpy(ly["mask"]).cuda()
+    s, codes_h, mask_h = inputs.make_weights(ly["d_out"], ly["d_in"], 5)
+    codes, mask = torch.from_numpy(codes_h).cuda(), torch.from_numpy(mask_h).cuda()
     vals, meta = K.slim_pack(codes, mask)
+    tiled = K.slim_repack_tiled(vals, meta)
+    out = {"layer": [ly["d_in"], ly["d_out"]]}
     with torch.cuda.stream(stream):
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        for _ in range(3):
-            K.slim_pack(codes, mask, vals, meta, check=False)
-        a0.record(stream)
-        for _ in range(10):
-            K.slim_pack(codes, mask, vals, meta, check=False)
-        a1.record(stream)
-        a1.synchronize()
-    us = 1e3 * a0.elapsed_time(a1) / 10
-    nbytes = 2.375 * ly["d_out"] * ly["d_in"]
-    return {"layer": [ly["d_in"], ly["d_out"]], "us": round(us, 2), "GBs": round(nbytes / us / 1e3, 1),
-            "bytes": "2 B read + 0.375 B written per dense weight"}
+        for name, fn, nbytes in (("pack", lambda: K.slim_pack(codes, mask, vals, meta, check=False), 2.375),
+                                 ("repack_tiled", lambda: K.slim_repack_tiled(vals, meta, out=tiled), 0.75)):
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(3):
+                fn()
+            a0.record(stream)
+            for _ in range(10):
+                fn()
+            a1.record(stream)
+            a1.synchronize()
+            us = 1e3 * a0.elapsed_time(a1) / 10
+            out[name] = {"us": round(us, 2), "GBs": round(nbytes * ly["d_out"] * ly["d_in"] / us / 1e3, 1)}
+    out["bytes"] = "pack: 2 B read + 0.375 B written per dense weight; repack: 0.375 B read + 0.375 B written"
+    return out
 
 
 def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, world, barrier):
-    """Same step through slim_linear_fwd_host: X comes from pinned host memory
+    """Same step through slim_linear_fwd_tiled_host: X comes from pinned host memory
     and Y goes back to pinned host memory inside every call."""
     import ctypes
     import torch
@@ -486,21 +559,22 @@ def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, wor
     calls, h2d, d2h = [], 0, 0
     for ly, b, a in step_calls:
         xh, yh = host[(ly["name"], b)]
+        # (X_host, b, tiled, layout, s, L, R, r, d_out, d_in, Y_host, x_dev, y_dev, ws, ws_bytes, status)
         calls.append((P(xh.data_ptr()), b, a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], P(yh.data_ptr()),
                       P(ly["Xd"][b].data_ptr()), P(ly["Yd"][b].data_ptr()), a[11], a[12], a[13]))
         h2d += xh.numel() * 2
         d2h += yh.numel() * 2
     sp = P(stream.cuda_stream)
-    steps = max(1, min(args.steps, 200))
+    steps = max(1, min(args.steps, 100))
 
     def run(n):
         for _ in range(n):
             for c in calls:
-                rc = lib.slim_linear_fwd_host(*c, sp)
+                rc = lib.slim_linear_fwd_tiled_host(*c, sp)
                 if rc != 0:
-                    raise RuntimeError(f"slim_linear_fwd_host failed: {K.strerror(rc)}")
+                    raise RuntimeError(f"slim_linear_fwd_tiled_host failed: {K.strerror(rc)}")
 
-    run(min(args.warmup, 20))
+    run(min(args.warmup, 10))
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -510,30 +584,49 @@ def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, wor
     ms = e0.elapsed_time(e1)
     ms = replicas.max_over_ranks(ms, "cuda")
     return {"value": replicas.whole_job_us_per_call(ms / steps, CALLS_PER_STEP, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h, "steps": steps, "api": "slim_linear_fwd_host"}
+            "d2h_bytes_per_step": d2h, "steps": steps, "api": "slim_linear_fwd_tiled_host"}
 
 
-def time_cpu_baseline(layers, repeats=8):
+def time_cpu_baseline(layers, repeats=2):
+    """The oracle, as it stands, on this machine's host cores: the whole step (a bounded sample: one pass over
+    each distinct (shape, batch) pair per repeat), plus a single-thread timing of the smallest layer."""
     import oracle
+    host = []
+    for ly in layers:
+        h = dict(ly)
+        h["ovals"], h["ometa"] = ly["vals"].cpu().numpy(), ly["meta"].cpu().numpy()
+        host.append(h)
     t_weighted, t_raw = 0.0, 0.0
-    host = [(ly, ly["vals"].cpu().numpy(), ly["meta"].cpu().numpy()) for ly in layers]
     for _ in range(repeats):
-        for ly, vals, meta in host:
-            for b in BATCHES:
-                t0 = time.perf_counter()
-                oracle.linear_fwd(ly["X"][b], vals, meta, ly["s"], ly["L"], ly["R"])
-                dt = time.perf_counter() - t0
-                t_raw += dt
-                t_weighted += dt * ly["count"]
-    return {"value": 1e6 * t_weighted / repeats / CALLS_PER_STEP, "unit": UNIT, "cores": oracle.num_threads(),
-            "kind": "oracle",
-            "sample": f"one oracle call per distinct (layer shape, batch) pair of the step, all token rows, "
-                      f"repeated {repeats} times ({t_raw:.1f} s of wall time on all cores), weighted by the "
-                      f"block's 4/2/1 layer counts"}
+        tw, tr = oracle_step(host, oracle)
+        t_weighted += tw
+        t_raw += tr
+    out = {"value": 1e6 * t_weighted / repeats / CALLS_PER_STEP, "unit": UNIT, "cores": oracle.num_threads(),
+           "kind": "oracle", "cpu": cpu_model(),
+           "sample": f"{SAMPLE_TEXT}; repeated {repeats} times ({t_raw:.1f} s of wall time on all cores)"}
+    # single thread: one call of the smallest layer at batch 16 in a child process pinned to one OpenMP thread
+    small = min(host, key=lambda h: h["d_in"] * h["d_out"])
+    try:
+        code = ("import sys, time; sys.path.insert(0, %r); import numpy as np, oracle; "
+                "from paper_2410_09615_b200 import inputs; "
+                "s, c, m = inputs.make_weights(%d, %d, 9); v, mt = oracle.pack(c, m); L, R = inputs.make_adapters(%d, %d, %d, 9); "
+                "X = inputs.make_activations(16, %d, 9); oracle.linear_fwd(X, v, mt, s, L, R); t = time.perf_counter(); "
+                "oracle.linear_fwd(X, v, mt, s, L, R); print(time.perf_counter() - t, oracle.num_threads())"
+                % (ROOT, small["d_out"], small["d_in"], small["d_out"], small["d_in"], small["r"], small["d_in"]))
+        res = {}
+        for label, env in (("one_thread", {"OMP_NUM_THREADS": "1"}), ("all_threads", {})):
+            o = subprocess.run([sys.executable, "-c", code], env={**os.environ, **env}, capture_output=True, text=True, timeout=600)
+            sec, thr = o.stdout.split()[-2:]
+            res[label] = {"us": round(1e6 * float(sec), 1), "threads": int(thr)}
+        out["single_thread"] = {"case": [small["d_in"], small["d_out"], small["r"], 16], **res}
+    except Exception as e:
+        out["single_thread"] = {"error": str(e)[:100]}
+    return out
 
 
 def run_single_case(args):
-    """Plain stream launches of one (d_in, d_out, r, b) case: the command ncu captures."""
+    """Plain stream launches of one (d_in, d_out, r, b) case, L2 flushed between them: the command a
+    profiler captures.  b <= 16: slim_linear_fwd_tiled; above: slim_linear_fwd on the packed weight."""
     import torch
     from paper_2410_09615_b200 import binding as K, build
     build.build()
@@ -541,6 +634,7 @@ def run_single_case(args):
     s, codes, mask = inputs.make_weights(d_out, d_in, 1)
     L, R = inputs.make_adapters(d_out, d_in, r, 1)
     vals, meta = K.slim_pack(torch.from_numpy(codes).cuda(), torch.from_numpy(mask).cuda())
+    tiled = K.slim_repack_tiled(vals, meta) if b <= 16 else None
     Ld = K.bf16_from_bits(L) if r else None
     Rd = K.bf16_from_bits(R) if r else None
     X = K.bf16_from_bits(inputs.make_activations(b, d_in, 1))
@@ -552,12 +646,16 @@ def run_single_case(args):
     for _ in range(args.calls):
         flush.zero_()                       # evict the weights from L2 between calls
         e0.record()
-        K.slim_linear_fwd(X, vals, meta, s, Ld, Rd, Y=Y, workspace=ws)
+        if tiled is not None:
+            K.slim_linear_fwd_tiled(X, tiled, d_out, s, Ld, Rd, Y=Y, workspace=ws)
+        else:
+            K.slim_linear_fwd(X, vals, meta, s, Ld, Rd, Y=Y, workspace=ws)
         e1.record()
         e1.synchronize()
         times.append(1e3 * e0.elapsed_time(e1))
     print(json.dumps({"case": [d_in, d_out, r, b], "calls": args.calls, "us_median": float(np.median(times)),
-                      "us_min": float(np.min(times)), "kernel": K.KERNEL_NAMES[K.slim_select_kernel(b, d_out, d_in, r)],
+                      "us_min": float(np.min(times)), "path": "tiled decode" if tiled is not None else
+                      K.KERNEL_NAMES[K.slim_select_kernel(b, d_out, d_in, r)],
                       "algorithmic_bytes": algorithmic_bytes(d_in, d_out, r, b)}))
     return 0
 
@@ -567,11 +665,11 @@ def main():
     ap.add_argument("--case", default=None, help="d_in,d_out,r,b: run plain launches of one case (for profilers)")
     ap.add_argument("--calls", type=int, default=5)
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA graph")
-    ap.add_argument("--skip-extras", action="store_true", help="skip the per-case table and the pack timing")
+    ap.add_argument("--skip-extras", action="store_true", help="skip the per-case and prefill tables and the pack timing")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU-oracle baseline")
     args = ap.parse_args()
     if args.case:
@@ -579,8 +677,8 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
-        args.steps = min(args.steps, 20)      # the oracle takes seconds per step
-        args.warmup = min(args.warmup, 3)
+        args.steps = min(args.steps, 3)       # the oracle takes seconds per step
+        args.warmup = min(args.warmup, 1)
         return run_reference(args)
     return run_ours(args)
 

@@ -251,6 +251,14 @@ slim_kernel_t slim_select_kernel(int b, int d_out, int d_in, int r);
 /* Number of kernels the last slim_linear_fwd* call on this host thread launched. */
 int slim_last_launch_count(void);
 
+/*
+ * Token-tile width (64 or 256 tokens) of the prefill kernel the last slim_linear_fwd* call on this host
+ * thread launched, 0 if that call ran another kernel.  The prefill kernel has a wide variant for problems
+ * that give every SM a 128-row x 256-token tile and a narrow one for the rest; tests use this query to
+ * make sure they exercise the variant they mean to.
+ */
+int slim_last_token_tile(void);
+
 const char* slim_strerror(slim_status_t status);
 const char* slim_version(void);
 

@@ -42,6 +42,7 @@ SIGNATURES = {
     "slim_noalloc_scratch_needed": (_SZ, [_I, _I, _I, _I]),
     "slim_select_kernel": (_I, [_I, _I, _I, _I]),
     "slim_last_launch_count": (_I, []),
+    "slim_last_token_tile": (_I, []),
     "slim_strerror": (ctypes.c_char_p, [_I]),
     "slim_version": (ctypes.c_char_p, []),
 }
@@ -153,6 +154,10 @@ def slim_select_kernel(b: int, d_out: int, d_in: int, r: int) -> int:
 
 def slim_last_launch_count() -> int:
     return int(lib().slim_last_launch_count())
+
+
+def slim_last_token_tile() -> int:
+    return int(lib().slim_last_token_tile())
 
 
 def new_workspace(b: int, d_out: int, d_in: int, r: int, device="cuda") -> torch.Tensor:

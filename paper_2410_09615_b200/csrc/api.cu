@@ -11,9 +11,11 @@ static DeviceInfo g_info[64];
 static std::atomic<bool> g_info_ready[64];
 static std::mutex g_info_mutex;
 static thread_local int t_launches = 0;
+static thread_local int t_token_tile = 0;
 
 void count_launch(int n) { t_launches += n; }
-void reset_launch_count() { t_launches = 0; }
+void reset_launch_count() { t_launches = 0; t_token_tile = 0; }
+void note_token_tile(int n) { t_token_tile = n; }
 
 // The record of a device is filled once under the mutex and published with a release store;
 // readers take it with an acquire load, so they never see a half-written record.
@@ -253,6 +255,8 @@ slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* val
 }
 
 int slim_last_launch_count(void) { return t_launches; }
+
+int slim_last_token_tile(void) { return t_token_tile; }
 
 const char* slim_strerror(slim_status_t status)
 {

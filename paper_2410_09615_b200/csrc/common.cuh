@@ -34,6 +34,7 @@ constexpr size_t kDecodeTfinalBytes = 198656;
 // Launch bookkeeping for slim_last_launch_count().
 void count_launch(int n);
 void reset_launch_count();
+void note_token_tile(int n);      // token-tile width of the prefill main launch, for slim_last_token_tile()
 
 // ---- launchers (defined in the kernel files) --------------------------------
 slim_status_t launch_pack(const int8_t* codes, const uint8_t* mask, int d_out, int d_in,

@@ -10,15 +10,14 @@ namespace dt {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// Shared-memory reads by 32-bit shared address.  Plain loads, so that the compiler may move them
+// ahead of the arithmetic of the previous block; the barrier waits and arrivals around a slot carry
+// memory clobbers, which keeps the reads inside the slot's lifetime.
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
+    return *reinterpret_cast<const uint4*>(__cvta_shared_to_generic(addr));
 }
 __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
+    return *reinterpret_cast<const uint32_t*>(__cvta_shared_to_generic(addr));
 }
 
 // Byte offset inside a TMA tile of 128-byte rows stored with the 128-byte swizzle (tile
@@ -31,7 +30,7 @@ __device__ __forceinline__ uint32_t swz128(int row, int byte_off) {
 // SEL picks which thread pair of every quad supplies the metadata word.
 template <int SEL>
 __device__ __forceinline__ void mma_sp_16832(float* c, const uint32_t* a, const uint4& b, uint32_t e) {
-    asm volatile(
+    asm(
         "mma.sp::ordered_metadata.sync.aligned.m16n8k32.row.col.f32.bf16.bf16.f32 "
         "{%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9,%10,%11}, {%0,%1,%2,%3}, %12, %13;"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -40,7 +39,7 @@ __device__ __forceinline__ void mma_sp_16832(float* c, const uint32_t* a, const 
 // D(16x8, fp32) += A(16x16 bf16) * B(16x8 bf16)
 __device__ __forceinline__ void mma_16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                           uint32_t b0, uint32_t b1) {
-    asm volatile(
+    asm(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 "
         "{%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])

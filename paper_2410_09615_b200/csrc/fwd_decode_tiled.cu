@@ -44,9 +44,9 @@ namespace {
 using namespace dt;
 
 constexpr int kCW = 8;                                  // consumer warps
-constexpr int kSW = 4;                                  // service warps
-constexpr int kThreads = (kCW + kSW) * 32;
-constexpr int kMaxSlotBytes = 6144;
+constexpr int kProducerWarp = kCW;                      // one warp requests every slot of the CTA
+constexpr int kSW = 3;                                  // service warps
+constexpr int kThreads = (kCW + 1 + kSW) * 32;
 constexpr int kBlockBytes = 1536;                       // one 16-row x 256-column block of the tiled weight
 constexpr int kMaxRing = 8;                             // slots per warp
 constexpr int kDCols = 128;                             // adapter columns per slot
@@ -178,7 +178,7 @@ struct PartWalk {
     }
 };
 
-constexpr int kBatch = 8;        // partial slots requested together
+constexpr int kBatch = 8;        // partial slots requested together (T partials)
 
 // Adds to sum[e] (e < E: elements lane + 32 e of a fragment-ordered tile at `off` words inside a
 // slot) the next up-to-kBatch slots of the walk; empties them.  Returns false when the walk is over.
@@ -215,6 +215,34 @@ __device__ __forceinline__ bool take_batch(PartWalk& pw, int off, int lane, floa
     return ptr[kBatch - 1] != nullptr;
 }
 
+// The jobs of one consumer warp: nR slots of the R list from sR, nW of the weight list, nL of the L list.
+struct Jobs { int nR, sR, nW, sW, nL, sL, total; };
+struct SliceGeo { bool in_slice; int ks, grp, blk0, blk1, nqW, nqR; };
+
+__device__ __forceinline__ SliceGeo make_geo(const Params& p, int cta) {
+    SliceGeo g;
+    g.in_slice = cta < p.KS * p.G;
+    g.ks = g.in_slice ? cta % p.KS : 0;
+    g.grp = g.in_slice ? cta / p.KS : 0;
+    slice_blocks(g.ks, p.KS, p.nblk, &g.blk0, &g.blk1);
+    g.nqW = ceil_div(g.blk1 - g.blk0, p.NB);              // weight slots per unit in this slice
+    g.nqR = (g.blk1 - g.blk0) * 2;                        // adapter slots per R tile in this slice
+    return g;
+}
+__device__ __forceinline__ Jobs make_jobs(const Params& p, const SliceGeo& g, int cta, int n_ctas, int cwarp) {
+    const Split spR = make_split(p.tilesR * g.nqR, p.wnR);
+    const Split spW = make_split(p.unitsW * g.nqW, p.G * kCW);
+    const Split spL = make_split(p.tilesW * p.nqL, n_ctas * kCW);
+    const int wi = g.grp * kCW + cwarp;                   // worker number inside the slice
+    const int wl = cta * kCW + cwarp;                     // worker number in the grid
+    Jobs jb;
+    jb.nR = g.in_slice && wi < p.wnR ? split_count(spR, wi) : 0; jb.sR = split_start(spR, wi);
+    jb.nW = g.in_slice ? split_count(spW, wi) : 0; jb.sW = split_start(spW, wi);
+    jb.nL = split_count(spL, wl); jb.sL = split_start(spL, wl);
+    jb.total = jb.nR + jb.nW + jb.nL;
+    return jb;
+}
+
 template <int NT, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmL)
@@ -228,23 +256,18 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
     unsigned char* ts = xs + p.x_bytes;
     const int t_bytes = p.nqL * 4 * p.b * 64;
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(ts + t_bytes);      // [kCW][kMaxRing]
-    uint64_t* t_bar = full_bar + kCW * kMaxRing;
+    uint64_t* empty_bar = full_bar + kCW * kMaxRing;                     // [kCW][kMaxRing]
+    uint64_t* t_bar = empty_bar + kCW * kMaxRing;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_ctas = gridDim.x, cta = blockIdx.x;
     const LaneCtx lc = make_lane_ctx(lane);
     const int NB = p.NB;
-
-    // this CTA's k-slice
-    const bool in_slice = cta < p.KS * p.G;
-    const int ks = in_slice ? cta % p.KS : 0, grp = in_slice ? cta / p.KS : 0;
-    int blk0, blk1;
-    slice_blocks(ks, p.KS, p.nblk, &blk0, &blk1);
-    const int nqW = ceil_div(blk1 - blk0, NB);               // weight slots per unit in this slice
-    const int nqR = (blk1 - blk0) * 2;                       // adapter slots per R tile in this slice
+    const SliceGeo geo = make_geo(p, cta);
+    const int blk0 = geo.blk0, blk1 = geo.blk1, nqW = geo.nqW, nqR = geo.nqR, ks = geo.ks;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kCW * kMaxRing; ++i) mbar_init(&full_bar[i], 1);
+        for (int i = 0; i < kCW * kMaxRing; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
         mbar_init(t_bar, kSW);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -252,56 +275,91 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
 
     // which kind of wait expired, if any: reported in bits 16-23 of the status word beside SLIM_ERR_TIMEOUT
     // (1 R slot, 2 weight slot, 4 T in shared memory, 8 L slot, 16 partials of an output tile,
-    //  64 partials of T, 128 published T)
+    //  32 ring slot not freed, 64 partials of T, 128 published T)
     uint32_t expired = 0;
-    bool ok = true;
     TSTAMP(0, 0);
 #ifdef SLIM_TILED_TRACE
-    if (threadIdx.x == 0) { g_tiled_trace[blockIdx.x * 16 + 11] = 0; g_tiled_trace[blockIdx.x * 16 + 12] = 0; g_tiled_trace[blockIdx.x * 16 + 13] = clock64(); }
+    if (threadIdx.x == 0) { g_tiled_trace[blockIdx.x * 16 + 11] = 0; g_tiled_trace[blockIdx.x * 16 + 12] = 0; g_tiled_trace[blockIdx.x * 16 + 14] = 0; g_tiled_trace[blockIdx.x * 16 + 13] = clock64(); }
 #endif
-    if (warp < kCW) {
-        // ================================ consumer warps ================================
-        const Split spR = make_split(p.tilesR * nqR, p.wnR);
-        const Split spW = make_split(p.unitsW * nqW, p.G * kCW);
-        const Split spL = make_split(p.tilesW * p.nqL, n_ctas * kCW);
-        const int wi = grp * kCW + warp;                      // worker number inside the slice
-        const int wl = cta * kCW + warp;                      // worker number in the grid
-        const int nR = in_slice && wi < p.wnR ? split_count(spR, wi) : 0, sR = split_start(spR, wi);
-        const int nW = in_slice ? split_count(spW, wi) : 0, sW = split_start(spW, wi);
-        const int nL = split_count(spL, wl), sL = split_start(spL, wl);
-        const int total = nR + nW + nL;
-        uint64_t* my_bar = full_bar + warp * kMaxRing;
-        const uint32_t my_ring = smem_u32(rings + (size_t)warp * p.ring * p.slot_bytes);
-
-        // Request the slot of job j into ring slot j % ring (the whole warp calls this).
-        auto issue = [&](int j) {
-            const int slot = j % p.ring;
-            uint64_t* bar = &my_bar[slot];
-            const uint32_t dst = my_ring + slot * p.slot_bytes;
-            if (j < nR) {
-                const int pos = sR + j, tile = pos / nqR, q = pos % nqR;
-                if (lane == 0) mbar_arrive_expect_tx(bar, 4096);
-                if (lane < 2) tma_tile(dst + lane * 2048, &tmR, blk0 * 256 + q * kDCols + 64 * lane, tile * 16, bar);
-            } else if (j < nR + nW) {
-                const int pos = sW + (j - nR), u = pos / nqW, q = pos % nqW;
-                const int nb = min(NB, blk1 - blk0 - q * NB), mt = min(MT, p.tilesW - u * MT);
-                if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)(mt * nb * kBlockBytes));
-                if (lane < mt)
-                    bulk_copy(dst + lane * NB * kBlockBytes,
-                              p.W + ((size_t)(u * MT + lane) * p.nblk + blk0 + q * NB) * kBlockBytes, (uint32_t)(nb * kBlockBytes), bar);
-            } else {
-                const int pos = sL + (j - nR - nW), tile = pos / p.nqL, q = pos % p.nqL;
-                if (lane == 0) mbar_arrive_expect_tx(bar, 4096);
-                if (lane < 2) tma_tile(dst + lane * 2048, &tmL, q * kDCols + 64 * lane, tile * 16, bar);
+    if (warp == kProducerWarp) {
+        // ================================ producer warp ================================
+        // Lane w < kCW requests the slots of consumer warp w, in that warp's job order, as its ring
+        // slots come free.  A request is held until the copy engine has room for it (with full rings
+        // that is most of the time), so it must not sit in the warps that compute.
+        const bool serves = lane < kCW;
+        const Jobs jb = make_jobs(p, geo, cta, n_ctas, serves ? lane : 0);
+        const int total = serves ? jb.total : 0;
+        int longest = total;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) longest = max(longest, __shfl_xor_sync(0xffffffffu, longest, o));
+        uint64_t* fbar = full_bar + (serves ? lane : 0) * kMaxRing;
+        uint64_t* ebar = empty_bar + (serves ? lane : 0) * kMaxRing;
+        const uint32_t ring0 = smem_u32(rings + (size_t)(serves ? lane : 0) * p.ring * p.slot_bytes);
+        // running (unit, slot in unit) of this lane's position in each list
+        int r_tile = nqR > 0 ? jb.sR / nqR : 0, r_q = nqR > 0 ? jb.sR % nqR : 0;
+        int w_u = jb.sW / nqW, w_q = jb.sW % nqW;
+        int l_tile = p.nqL > 0 ? jb.sL / p.nqL : 0, l_q = p.nqL > 0 ? jb.sL % p.nqL : 0;
+        // Every lane walks its own job list at its own pace: in each round a lane whose next ring slot is
+        // free (a test that does not wait) requests its next job, the others sit the round out, so one slow
+        // consumer does not hold up the requests of the other seven.
+        int j = 0, slot = 0;
+        uint32_t parity = 0;                                // phase of the "slot left" barrier awaited in the second lap; flips per lap
+        (void)longest;
+        for (uint32_t idle = 0;;) {
+            const bool has = j < total;
+            if (!__any_sync(0xffffffffu, has)) break;
+            bool can = has;
+            if (has && j >= p.ring) {
+                uint32_t ok_;
+                asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                             : "=r"(ok_) : "r"(smem_u32(&ebar[slot])), "r"(parity) : "memory");
+                can = ok_ != 0;
             }
-        };
-        const int pre = min(total, p.ring);
-        for (int j = 0; j < pre; ++j) issue(j);
-        TSTAMP(0, 10);
+            if (can) {
+                uint64_t* bar = &fbar[slot];
+                const uint32_t dst = ring0 + slot * p.slot_bytes;
+                if (j < jb.nR) {
+                    mbar_arrive_expect_tx(bar, 4096);
+                    tma_tile(dst, &tmR, blk0 * 256 + r_q * kDCols, r_tile * 16, bar);
+                    tma_tile(dst + 2048, &tmR, blk0 * 256 + r_q * kDCols + 64, r_tile * 16, bar);
+                    if (++r_q == nqR) { r_q = 0; ++r_tile; }
+                } else if (j < jb.nR + jb.nW) {
+                    const int nb = min(NB, blk1 - blk0 - w_q * NB), mt = min(MT, p.tilesW - w_u * MT);
+                    mbar_arrive_expect_tx(bar, (uint32_t)(mt * nb * kBlockBytes));
+#pragma unroll
+                    for (int m = 0; m < MT; ++m)
+                        if (m < mt)
+                            bulk_copy(dst + m * NB * kBlockBytes,
+                                      p.W + ((size_t)(w_u * MT + m) * p.nblk + blk0 + w_q * NB) * kBlockBytes, (uint32_t)(nb * kBlockBytes), bar);
+                    if (++w_q == nqW) { w_q = 0; ++w_u; }
+                } else {
+                    mbar_arrive_expect_tx(bar, 4096);
+                    tma_tile(dst, &tmL, l_q * kDCols, l_tile * 16, bar);
+                    tma_tile(dst + 2048, &tmL, l_q * kDCols + 64, l_tile * 16, bar);
+                    if (++l_q == p.nqL) { l_q = 0; ++l_tile; }
+                }
+                if (++slot == p.ring) { slot = 0; if (j >= p.ring) parity ^= 1u; }
+                ++j;
+            }
+            if (__any_sync(0xffffffffu, can)) idle = 0;
+            else {
+                if (++idle > kMbarSpinLimit) { expired |= 32u; break; }
+                __nanosleep(64);
+            }
+        }
+    } else if (warp < kCW) {
+        // ================================ consumer warps ================================
+        const Jobs jb = make_jobs(p, geo, cta, n_ctas, warp);
+        const int nR = jb.nR, sR = jb.sR, nW = jb.nW, sW = jb.sW, nL = jb.nL, sL = jb.sL;
+        const Split spL = make_split(p.tilesW * p.nqL, n_ctas * kCW);
+        const int wi = geo.grp * kCW + warp, wl = cta * kCW + warp;
+        uint64_t* my_full = full_bar + warp * kMaxRing;
+        uint64_t* my_empty = empty_bar + warp * kMaxRing;
+        const uint32_t my_ring = smem_u32(rings + (size_t)warp * p.ring * p.slot_bytes);
 
         // ---- the CTA's slice of the activations into shared memory, fragment order.  A thread
         // requests several 16-byte pieces before it stores the first (one global round trip per batch).
-        if (in_slice) {
+        if (geo.in_slice) {
             const int cols = (blk1 - blk0) * 256, chunks = cols / 8;      // 16-byte chunks per token
             const __nv_bfloat16* xsrc = p.X + (size_t)blk0 * 256;
             const int n_chunks = p.b * chunks;
@@ -351,95 +409,17 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
 #pragma unroll
                 for (int e = 0; e < 4; ++e) st_gpu(dst + (h * 4 + e) * 32 + lane, slot_bits(a[h][e]));
         };
-        zero_acc();
-        int cur = -1;                 // list unit whose accumulators are live
-        bool t_ready = p.r == 0;
 
-        for (int j = 0; j < total; ++j) {
-            const int slot = j % p.ring;
-            const uint32_t src = my_ring + slot * p.slot_bytes;
-            if (j < nR) {
-                // ---------------------------------------------------------------- R slot
-                const int pos = sR + j, tile = pos / nqR, q = pos % nqR;
-                if (tile != cur) {
-                    if (cur >= 0) store_tile(Tmine + (size_t)(cur - sR / nqR) * frag, acc[0]);
-                    zero_acc();
-                    cur = tile;
-                }
-                if (!mbar_wait(&my_bar[slot], (j / p.ring) & 1)) expired |= 1u;
-                if (j == 0) TSTAMP(0, 2);
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    uint4 xb[NT];
-                    load_x_step<NT>(xb, xs_addr, q * 4 + jj, p.b, lc);
-                    dense_step<NT>(acc[0], src + (jj >> 1) * 2048, jj & 1, xb, lc);
-                }
-                if (j + 1 == nR) { store_tile(Tmine + (size_t)(cur - sR / nqR) * frag, acc[0]); zero_acc(); cur = -1; }
-            } else if (j < nR + nW) {
-                // ---------------------------------------------------------------- weight slot
-                const int pos = sW + (j - nR), u = pos / nqW, q = pos % nqW;
-                if (u != cur) {
-                    if (cur >= 0) {
-#pragma unroll
-                        for (int m = 0; m < MT; ++m) store_tile(Pmine + ((size_t)(cur - sW / nqW) * MT + m) * frag, acc[m]);
-                    }
-                    zero_acc();
-                    cur = u;
-                }
-                const int nb = min(NB, blk1 - blk0 - q * NB), mt = min(MT, p.tilesW - u * MT);
-#ifdef SLIM_TILED_TRACE
-                const long long w0_ = clock64();
-#endif
-                if (!mbar_wait(&my_bar[slot], (j / p.ring) & 1)) expired |= 2u;
-#ifdef SLIM_TILED_TRACE
-                if (warp == 0 && lane == 0) { g_tiled_trace[blockIdx.x * 16 + 11] += clock64() - w0_; g_tiled_trace[blockIdx.x * 16 + 12] += 1; }
-#endif
-                if (j == nR) TSTAMP(0, 3);
-                for (int bi = 0; bi < nb; ++bi) {
-                    uint4 xf[8][NT];
-                    load_x_block<NT>(xf, xs_addr, (q * NB + bi) * 8, p.b, lc);
-#pragma unroll
-                    for (int m = 0; m < MT; ++m)
-                        if (m < mt) sparse_block<NT>(acc[m], src + (m * NB + bi) * kBlockBytes, xf, lc);
-                }
-                if (j + 1 == nR + nW) {
-#pragma unroll
-                    for (int m = 0; m < MT; ++m) store_tile(Pmine + ((size_t)(cur - sW / nqW) * MT + m) * frag, acc[m]);
-                    zero_acc(); cur = -1;
-                }
-            } else {
-                // ---------------------------------------------------------------- L slot
-                const int pos = sL + (j - nR - nW), tile = pos / p.nqL, q = pos % p.nqL;
-                if (tile != cur) {
-                    if (cur >= 0) store_tile(Amine + (size_t)(cur - sL / p.nqL) * frag, acc[0]);
-                    zero_acc();
-                    cur = tile;
-                }
-                if (j == nR + nW) TSTAMP(0, 4);
-                if (!t_ready) { if (!mbar_wait(t_bar, 0)) expired |= 4u; t_ready = true; TSTAMP(0, 5); }
-                if (!mbar_wait(&my_bar[slot], (j / p.ring) & 1)) expired |= 8u;
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    uint4 tb[NT];
-                    load_x_step<NT>(tb, ts_addr, q * 4 + jj, p.b, lc);
-                    dense_step<NT>(acc[0], src + (jj >> 1) * 2048, jj & 1, tb, lc);
-                }
-                if (j + 1 == total) { store_tile(Amine + (size_t)(cur - sL / p.nqL) * frag, acc[0]); cur = -1; }
-            }
-            __syncwarp();                                   // every lane is done reading the slot
-            if (j + p.ring < total) issue(j + p.ring);
-        }
-
-        TSTAMP(0, 6);
-        // ---------------------------------------------------------------- output tiles
-        const Split spF = make_split(p.tilesW, n_ctas * kCW);
-        const int f0 = split_start(spF, wl), f1 = f0 + split_count(spF, wl);
-        for (int tile = f0; tile < f1; ++tile) {
+        // Finishes output tile `tile`: s * (weight partials of every k-slice, in list order) + (own[] +
+        // the adapter partials of the workers from first_w on, in list order), rounded to bf16.
+        auto finish_tile = [&](int tile, const float (&own)[NT][4], int first_w) {
             float psum[E], asum[E];
 #pragma unroll
-            for (int e = 0; e < E; ++e) { psum[e] = 0.f; asum[e] = 0.f; }
+            for (int h = 0; h < NT; ++h)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { psum[h * 4 + e] = 0.f; asum[h * 4 + e] = own[h][e]; }
             const int u = tile / MT, m = tile % MT;
-            // walk state: slice of the weight partials being walked (p.KS = the adapter partials, then the end)
+            // walk state: k-slice of the weight partials being walked (p.KS = the adapter partials, then the end)
             int k2 = -1, w = 0, w_last = -1, nq2 = 1;
             Split sp2 = spL;
             auto next_part = [&](bool* is_adapter) -> uint32_t* {
@@ -454,7 +434,7 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
                         w = split_owner(sp2, u * nq2); w_last = split_owner(sp2, u * nq2 + nq2 - 1);
                     } else {
                         nq2 = p.nqL; sp2 = spL;
-                        w = split_owner(sp2, tile * nq2); w_last = split_owner(sp2, tile * nq2 + nq2 - 1);
+                        w = first_w; w_last = split_owner(sp2, tile * nq2 + nq2 - 1);
                     }
                 }
                 const int u0 = split_start(sp2, w) / nq2;
@@ -465,39 +445,29 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
                 ++w;
                 return ptr;
             };
+            constexpr int kFB = NT == 1 ? 16 : 8;           // partials requested together: one round trip for most tiles
             for (bool more = true; more;) {
-                uint32_t* ptr[kBatch];
-                bool adapter[kBatch];
+                uint32_t* ptr[kFB];
+                bool adapter[kFB];
 #pragma unroll
-                for (int k = 0; k < kBatch; ++k) { adapter[k] = false; ptr[k] = more ? next_part(&adapter[k]) : nullptr; if (!ptr[k]) more = false; }
-                uint32_t v[kBatch][E];
+                for (int k = 0; k < kFB; ++k) { adapter[k] = false; ptr[k] = more ? next_part(&adapter[k]) : nullptr; if (!ptr[k]) more = false; }
+                uint32_t v[kFB][E];
 #pragma unroll
-                for (int k = 0; k < kBatch; ++k)
+                for (int k = 0; k < kFB; ++k)
 #pragma unroll
                     for (int e = 0; e < E; ++e) v[k][e] = ptr[k] ? ld_gpu(ptr[k] + e * 32 + lane) : 0u;
                 for (uint32_t spins = 0;; ++spins) {
                     bool all = true;
 #pragma unroll
-                    for (int k = 0; k < kBatch; ++k)
+                    for (int k = 0; k < kFB; ++k)
 #pragma unroll
                         for (int e = 0; e < E; ++e)
                             if (v[k][e] == kEmpty) { v[k][e] = ld_gpu(ptr[k] + e * 32 + lane); all = false; }
                     if (all) break;
-                    if (spins > kPollLimit) {
-                        expired |= 16u;
-#ifdef SLIM_TILED_TRACE
-                        for (int k = 0; k < kBatch; ++k)
-                            for (int e = 0; e < E; ++e)
-                                if (v[k][e] == kEmpty && atomicAdd(&g_tiled_dbg[0], 1ull) == 0) {
-                                    g_tiled_dbg[1] = tile; g_tiled_dbg[2] = adapter[k]; g_tiled_dbg[3] = (unsigned long long)(ptr[k] - (adapter[k] ? p.Apart : p.Ppart));
-                                    g_tiled_dbg[4] = blockIdx.x * 100 + warp; g_tiled_dbg[5] = e * 32 + lane; g_tiled_dbg[6] = k;
-                                }
-#endif
-                        break;
-                    }
+                    if (spins > kPollLimit) { expired |= 16u; break; }
                 }
 #pragma unroll
-                for (int k = 0; k < kBatch; ++k)
+                for (int k = 0; k < kFB; ++k)
                     if (ptr[k]) {
 #pragma unroll
                         for (int e = 0; e < E; ++e) {
@@ -513,6 +483,115 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
                 const int tok = 8 * h + 2 * lc.t + (q & 1);
                 if (tok < p.b) p.Y[(size_t)tok * p.d_out + n] = __float2bfloat16_rn(fmaf(psum[e], p.s, asum[e]));
             }
+        };
+
+        zero_acc();
+        // Walk of the three lists with running (unit, slot in unit) pairs and a running ring position:
+        // no division inside the loops (a division is a long chain of dependent instructions, and a warp
+        // has only one or two others on its scheduler to hide it behind).
+        int slot = 0; uint32_t parity = 0;
+        auto next_slot = [&]() { if (++slot == p.ring) { slot = 0; parity ^= 1u; } };
+        const int r_first = nqR > 0 ? sR / nqR : 0, w_first = sW / nqW, l_first = p.nqL > 0 ? sL / p.nqL : 0;
+
+        // ---------------------------------------------------------------- R slots
+        {
+            int tile = r_first, q = nqR > 0 ? sR % nqR : 0;
+            for (int j = 0; j < nR; ++j) {
+                const uint32_t src = my_ring + slot * p.slot_bytes;
+                if (!mbar_wait(&my_full[slot], parity)) expired |= 1u;
+                if (j == 0) TSTAMP(0, 2);
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    uint4 xb[NT];
+                    load_x_step<NT>(xb, xs_addr, q * 4 + jj, p.b, lc);
+                    dense_step<NT>(acc[0], src + (jj >> 1) * 2048, jj & 1, xb, lc);
+                }
+                __syncwarp();                               // every lane is done reading the slot
+                if (lane == 0) mbar_arrive(&my_empty[slot]);
+                next_slot();
+                if (++q == nqR || j + 1 == nR) {            // leaving the tile: its partial goes to the workspace
+                    store_tile(Tmine + (size_t)(tile - r_first) * frag, acc[0]);
+                    zero_acc();
+                    q = 0; ++tile;
+                }
+            }
+        }
+        // ---------------------------------------------------------------- weight slots
+        {
+            int u = w_first, q = sW % nqW;
+            for (int j = 0; j < nW; ++j) {
+                const uint32_t src = my_ring + slot * p.slot_bytes;
+                const int nb = min(NB, blk1 - blk0 - q * NB), mt = min(MT, p.tilesW - u * MT);
+#ifdef SLIM_TILED_TRACE
+                const long long w0_ = clock64();
+#endif
+                if (!mbar_wait(&my_full[slot], parity)) expired |= 2u;
+#ifdef SLIM_TILED_TRACE
+                const long long c0_ = clock64();
+                if (warp == 0 && lane == 0) { g_tiled_trace[blockIdx.x * 16 + 11] += c0_ - w0_; g_tiled_trace[blockIdx.x * 16 + 12] += 1; }
+#endif
+                if (j == 0) TSTAMP(0, 3);
+#pragma unroll
+                for (int bi = 0; bi < 4 / MT; ++bi) {
+                    if (bi < nb) {
+                        uint4 xf[8][NT];
+                        load_x_block<NT>(xf, xs_addr, (q * NB + bi) * 8, p.b, lc);
+#pragma unroll
+                        for (int m = 0; m < MT; ++m)
+                            if (m < mt) sparse_block<NT>(acc[m], src + (m * NB + bi) * kBlockBytes, xf, lc);
+                    }
+                }
+#ifdef SLIM_TILED_TRACE
+                if (warp == 0 && lane == 0) g_tiled_trace[blockIdx.x * 16 + 14] += clock64() - c0_;
+#endif
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&my_empty[slot]);
+                next_slot();
+                if (++q == nqW || j + 1 == nW) {
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) store_tile(Pmine + ((size_t)(u - w_first) * MT + m) * frag, acc[m]);
+                    zero_acc();
+                    q = 0; ++u;
+                }
+            }
+        }
+        // ---------------------------------------------------------------- L slots
+        if (nL > 0) {
+            TSTAMP(0, 4);
+            if (!mbar_wait(t_bar, 0)) expired |= 4u;        // all of T is in shared memory
+            TSTAMP(0, 5);
+            int tile = l_first, q = sL % p.nqL;
+            bool head = q == 0;                             // this worker holds the first slot of the tile
+            for (int j = 0; j < nL; ++j) {
+                const uint32_t src = my_ring + slot * p.slot_bytes;
+                if (!mbar_wait(&my_full[slot], parity)) expired |= 8u;
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    uint4 tb[NT];
+                    load_x_step<NT>(tb, ts_addr, q * 4 + jj, p.b, lc);
+                    dense_step<NT>(acc[0], src + (jj >> 1) * 2048, jj & 1, tb, lc);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&my_empty[slot]);
+                next_slot();
+                if (++q == p.nqL || j + 1 == nL) {
+                    // The worker that holds a tile's first slot finishes the tile (the workers after it have long
+                    // written their partials: a range is walked front to back, so the tile a range ends in is the
+                    // first thing the next worker does); any other worker leaves its partial.
+                    if (head) finish_tile(tile, acc[0], wl + 1);
+                    else store_tile(Amine + (size_t)(tile - l_first) * frag, acc[0]);
+                    zero_acc();
+                    q = 0; ++tile; head = true;
+                }
+            }
+        }
+        TSTAMP(0, 6);
+
+        // ---------------------------------------------------------------- output tiles without adapters
+        if (p.r == 0) {
+            const Split spF = make_split(p.tilesW, n_ctas * kCW);
+            const int f0 = split_start(spF, wl), f1 = f0 + split_count(spF, wl);
+            for (int tile = f0; tile < f1; ++tile) finish_tile(tile, acc[0], 0);      // acc is zero here
         }
         TSTAMP(0, 7);
 #ifdef SLIM_TILED_TRACE
@@ -520,9 +599,10 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
 #endif
     } else if (p.r > 0) {
         // ================================ service warps ================================
-        const int sw = warp - kCW;
+        const int sw = warp - kProducerWarp - 1;
         const uint32_t call = (uint32_t)(ld_gpu64(p.departures) / (unsigned)n_ctas) + 1u;
         const int pairs = p.r / 2;
+        bool ok = true;
         // ---- sum the partials of T, 32 fragment elements per item, and publish them
         const int items = p.tilesR * E;
         for (int it = cta * kSW + sw; it < items; it += n_ctas * kSW) {
@@ -548,9 +628,9 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
                          ((unsigned long long)call << 32) | *reinterpret_cast<const uint32_t*>(&pr));
             }
         }
-        TSTAMP(kCW, 8);
+        TSTAMP(kProducerWarp + 1, 8);
         // ---- all of T into shared memory (fragment order; columns past r are zero)
-        const int st = threadIdx.x - kCW * 32;
+        const int st = threadIdx.x - (kProducerWarp + 1) * 32;
         uint32_t* tsw = reinterpret_cast<uint32_t*>(ts);
         for (int i = st; i < t_bytes / 4; i += kSW * 32) tsw[i] = 0u;
         asm volatile("bar.sync 2, %0;" :: "n"(kSW * 32) : "memory");            // the service warps only
@@ -584,7 +664,7 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(t_bar);
-        TSTAMP(kCW, 9);
+        TSTAMP(kProducerWarp + 1, 9);
     }
 
     if (expired && p.status) atomicOr(p.status, (1u << SLIM_ERR_TIMEOUT) | (expired << 16));
@@ -626,13 +706,13 @@ bool make_plan(int b, int d_out, int d_in, int r, int ctas, Plan* pl) {
     const long long tile_blocks = (long long)pl->tilesW * pl->nblk;
     pl->mt = 1;
     if (tile_blocks >= 6LL * workers && pl->tilesW >= 2) pl->mt = 2;
-    if (tile_blocks >= 8LL * workers && pl->tilesW >= 4 && pl->nt == 2) pl->mt = 4;
+    if (tile_blocks >= 8LL * workers && pl->tilesW >= 4) pl->mt = 4;
     pl->nb = 4 / pl->mt;
     if (tile_blocks < 4LL * workers) pl->nb = pl->nb > 2 ? 2 : pl->nb;      // small problems: finer slots
     if (tile_blocks < 2LL * workers) pl->nb = 1;
 #ifdef SLIM_DECODE_TUNE
     // experiments only: the environment overrides the slot shape
-    if (const char* e = getenv("SLIM_MT")) { const int v = atoi(e); if ((v == 1 || v == 2 || (v == 4 && pl->nt == 2)) && pl->tilesW >= v) { pl->mt = v; pl->nb = 4 / v; } }
+    if (const char* e = getenv("SLIM_MT")) { const int v = atoi(e); if ((v == 1 || v == 2 || v == 4) && pl->tilesW >= v) { pl->mt = v; pl->nb = 4 / v; } }
     if (const char* e = getenv("SLIM_NB")) { const int v = atoi(e); if (v >= 1 && v * pl->mt <= 4) pl->nb = v; }
 #endif
     pl->unitsW = ceil_div(pl->tilesW, pl->mt);
@@ -641,7 +721,7 @@ bool make_plan(int b, int d_out, int d_in, int r, int ctas, Plan* pl) {
     // because every k-slice adds a set of partial sums.  Take the deepest ring (up to kMaxRing slots)
     // that still leaves the whole row to one slice, else three slots, else two.
     const size_t t_smem = (size_t)pl->nqL * 4 * b * 64;
-    const size_t fixed = 1024 + t_smem + (kCW * kMaxRing + 1) * 8 + 64;
+    const size_t fixed = 1024 + t_smem + (2 * kCW * kMaxRing + 1) * 8 + 64;
     int slot = pl->mt * pl->nb * kBlockBytes;
     if (r > 0 && slot < 4096) slot = 4096;
     slot = (slot + 1023) / 1024 * 1024;
@@ -731,8 +811,8 @@ bool make_tile_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t r
 }  // namespace
 
 int decode_tiled_query_residency() {
-    return query_residency<1, 1>() && query_residency<1, 2>() && query_residency<2, 1>() && query_residency<2, 2>() &&
-           query_residency<2, 4>();
+    return query_residency<1, 1>() && query_residency<1, 2>() && query_residency<1, 4>() && query_residency<2, 1>() &&
+           query_residency<2, 2>() && query_residency<2, 4>();
 }
 
 bool decode_tiled_supports(int b, int d_out, int d_in, int r) {
@@ -782,7 +862,8 @@ slim_status_t launch_decode_tiled(const __nv_bfloat16* X, int b, const uint8_t* 
     void* args[] = {&p, &tmR, &tmL};
     const dim3 grid(ctas), block(kThreads);
     const void* fn = nullptr;
-    if (pl.nt == 1) fn = pl.mt == 1 ? (const void*)decode_tiled_kernel<1, 1> : (const void*)decode_tiled_kernel<1, 2>;
+    if (pl.nt == 1) fn = pl.mt == 1 ? (const void*)decode_tiled_kernel<1, 1> : pl.mt == 2 ? (const void*)decode_tiled_kernel<1, 2>
+                                                                                : (const void*)decode_tiled_kernel<1, 4>;
     else fn = pl.mt == 1 ? (const void*)decode_tiled_kernel<2, 1> : pl.mt == 2 ? (const void*)decode_tiled_kernel<2, 2>
                                                                                 : (const void*)decode_tiled_kernel<2, 4>;
     const cudaError_t e = cudaLaunchCooperativeKernel(fn, grid, block, args, pl.smem, st);

@@ -731,6 +731,7 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     p.scale = s_eff; p.status = status_dev; p.part = nullptr; p.k_per = 0;
     if (p.n1 + p.n2 == 0)             // s == 0 and no adapters: the result is zero
         return cudaMemsetAsync(Y, 0, (size_t)b * d_out * 2, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
+    note_token_tile(wide ? 256 : 64);
     slim_status_t rc;
     if (!wide) rc = launch_tile_kernel<64, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
     else rc = pair ? launch_tile_kernel<256, true>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st)

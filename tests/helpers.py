@@ -40,6 +40,7 @@ def run_case(d_in, d_out, r, b, seed, wseed=None, kernel=binding.KERNEL_AUTO, ro
     ws = binding.new_workspace(b, d_out, d_in, r)
     Y = binding.slim_linear_fwd(X, vals, meta, s, L, R, workspace=ws, status=status, kernel=kernel)
     launches = binding.slim_last_launch_count()
+    token_tile = binding.slim_last_token_tile()
     torch.cuda.synchronize()
     assert binding.read_status(status) == 0, f"device status {binding.read_status(status):#x}"
     # the workspace is left ready for the next call: same inputs, same bits
@@ -52,4 +53,5 @@ def run_case(d_in, d_out, r, b, seed, wseed=None, kernel=binding.KERNEL_AUTO, ro
     y_ref = oracle.linear_fwd(ly.X, ovals, ometa, s, ly.L, ly.R, rows=rows)
     res = parity.compare(y, y_ref)
     res["launches"] = launches
+    res["token_tile"] = token_tile
     return res

@@ -85,6 +85,52 @@ def test_small_prefill_kernel(d_in, d_out, r, b):
     assert res["launches"] in ((2, 3) if r else (1,))
 
 
+# The wide variant (128 rows x 256 tokens per CTA) is what the dispatcher runs on every full-size
+# prefill configuration; it is chosen when (d_out / 128) * ceil(b / 256) >= the SM count, so these
+# shapes have many row tiles and a short contraction axis (the oracle stays cheap).
+PREFILL_WIDE = [  # d_in, d_out, r, b
+    (384, 4864, 48, 1000),   # ragged last token tile, d_in = 128 mod 256 (no rotated walk), ragged 32-column adapter stage
+    (256, 19072, 0, 130),    # two token tiles, the second almost empty; no adapters
+    (512, 9600, 112, 512),   # whole token tiles, ragged rank
+]
+
+
+@pytest.mark.parametrize("d_in,d_out,r,b", PREFILL_WIDE)
+def test_wide_prefill_kernel_all_elements(d_in, d_out, r, b):
+    res = run_case(d_in, d_out, r, b, seed=16, kernel=K.KERNEL_PREFILL)
+    assert res["token_tile"] == 256, "this shape must run the 256-token variant"
+    assert_ok(res)
+
+
+def test_narrow_prefill_kernel_reports_its_tile():
+    res = run_case(256, 128, 16, 40, seed=13, kernel=K.KERNEL_PREFILL)
+    assert res["token_tile"] == 64 and res["ok"]
+
+
+def test_wide_prefill_integer_inputs_are_exact_and_one_hot_reads_columns():
+    rng = np.random.default_rng(17)
+    d_in, d_out, r, b = 256, 19072, 16, 300
+    codes = rng.integers(-8, 8, size=(d_out, d_in)).astype(np.int8)
+    mask = inputs.top2_mask(rng.standard_normal((d_out, d_in)).astype(np.float32))
+    Xi = rng.integers(-1, 2, size=(b, d_in))
+    Li = rng.integers(-1, 2, size=(d_out, r))
+    Ri = (rng.random((r, d_in)) < 0.05).astype(np.int64) * rng.integers(-1, 2, size=(r, d_in))
+    vals, meta = K.slim_pack(to_dev(codes), to_dev(mask))
+    Y = K.slim_linear_fwd(K.bf16_from_bits(bf(Xi)), vals, meta, 1.0, K.bf16_from_bits(bf(Li)),
+                          K.bf16_from_bits(bf(Ri)), kernel=K.KERNEL_PREFILL)
+    assert K.slim_last_token_tile() == 256
+    exact = Xi @ (codes.astype(np.int64) * mask).T + (Xi @ Ri.T) @ Li.T
+    assert np.abs(exact).max() <= 256
+    assert np.array_equal(inputs.bf16_bits_to_f64(K.bits_from_bf16(Y)), exact.astype(np.float64))
+    # one-hot activations: token m reads back column ks[m] of the weight
+    ks = rng.integers(0, d_in, size=b)
+    X = np.zeros((b, d_in), np.float32)
+    X[np.arange(b), ks] = 1.0
+    Y = K.slim_linear_fwd(K.bf16_from_bits(bf(X)), vals, meta, 0.5, None, None, kernel=K.KERNEL_PREFILL)
+    assert K.slim_last_token_tile() == 256
+    assert np.array_equal(inputs.bf16_bits_to_f64(K.bits_from_bf16(Y)), 0.5 * (codes.astype(np.float64) * mask)[:, ks].T)
+
+
 PREFILL_PAIR = [  # d_in, d_out, r, b: even numbers of 128-row tiles
     (256, 256, 16, 40),
     (1024, 512, 112, 300),   # ragged token tile and rank, more stages than the ring holds
@@ -270,5 +316,10 @@ def test_full_size_prefill_configs(d_in, d_out, r, b, seed, wseed):
     dispatcher picks; compared on sampled token rows (first, middle and last
     rows of the edge tiles plus one seeded row in every other 128-token tile)."""
     assert K.slim_select_kernel(b, d_out, d_in, r) == K.KERNEL_PREFILL
-    rows = inputs.sample_rows(b, tile=128, seed=seed, dense_edges=False)
-    assert_ok(run_case(d_in, d_out, r, b, seed, wseed, rows=rows))
+    # every row of the first and of the last 128-token tile for the square attention layers (the oracle
+    # needs a few seconds per 100 rows of the largest layers, so those keep three rows per edge tile)
+    dense = d_in == d_out
+    rows = inputs.sample_rows(b, tile=128, seed=seed, dense_edges=dense)
+    res = run_case(d_in, d_out, r, b, seed, wseed, rows=rows)
+    assert res["token_tile"] == 256
+    assert_ok(res)

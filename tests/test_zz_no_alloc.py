@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2410_09615_b200 import binding as K, build, inputs, parity
 
 
@@ -40,6 +41,7 @@ def test_noalloc_rejects_problems_beyond_its_scratch_on_the_host():
 @pytest.mark.parametrize("d_in,d_out,r,b", [(2304, 272, 112, 13), (4096, 4096, 416, 16), (1024, 256, 0, 1)])
 def test_noalloc_matches_the_workspace_entry_point_twice(d_in, d_out, r, b):
     ly = inputs.make_layer(d_in, d_out, r, b, seed=4242)
+    ovals, ometa = oracle.pack(ly.codes, ly.mask)
     vals, meta = K.slim_pack(torch.from_numpy(ly.codes).cuda(), torch.from_numpy(ly.mask).cuda())
     L = K.bf16_from_bits(ly.L) if r else None
     R = K.bf16_from_bits(ly.R) if r else None
@@ -47,18 +49,26 @@ def test_noalloc_matches_the_workspace_entry_point_twice(d_in, d_out, r, b):
     y_ref = None
     for call in range(2):
         # fresh activations per call, so a stale partial sum from the previous call would show
-        X = K.bf16_from_bits(inputs.make_activations(b, d_in, 4242 + call))
+        x_bits = inputs.make_activations(b, d_in, 4242 + call)
+        X = K.bf16_from_bits(x_bits)
         want = K.slim_linear_fwd(X, vals, meta, ly.s, L, R, kernel=K.KERNEL_DECODE)
         got = torch.full((b, d_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+        torch.cuda.synchronize()
         before = torch.cuda.memory_allocated()
+        free_before, _total = torch.cuda.mem_get_info()     # the driver's view: sees any cudaMalloc, torch's or not
         K.slim_linear_fwd_noalloc(X, vals, meta, ly.s, L, R, got, status=status)
         assert K.slim_last_launch_count() == 1
-        assert torch.cuda.memory_allocated() <= before     # torch may free earlier temporaries, never grow
         torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() <= before     # torch may free earlier temporaries, never grow
+        if call > 0:                                        # (the first call may load the kernel's code)
+            assert torch.cuda.mem_get_info()[0] >= free_before
         assert K.read_status(status) == 0
         res = parity.compare(inputs.bf16_bits_to_f64(K.bits_from_bf16(got)),
                              inputs.bf16_bits_to_f64(K.bits_from_bf16(want)))
         assert res["ok"], (call, res)
+        # and against the definition itself
+        ref = oracle.linear_fwd(x_bits, ovals, ometa, ly.s, ly.L, ly.R)
+        assert parity.compare(inputs.bf16_bits_to_f64(K.bits_from_bf16(got)), ref)["ok"]
         # same kernel, same reduction order: in fact bit-identical
         assert torch.equal(got.view(torch.int16), want.view(torch.int16))
         if y_ref is not None:
