@@ -159,8 +159,13 @@ int oracle_unpack(const uint8_t *vals, const uint8_t *meta, int d_out, int d_in,
  * third-party kernel, Sec. 4 "Speedup"); nothing is computed, bytes only move.
  *
  * d_out % 16 == 0, d_in % 256 == 0.  The matrix is cut into tiles of 16 rows and
- * blocks of 256 columns; (tile, block) occupies 1536 bytes at
- * ((tile * d_in/256) + block) * 1536.  Inside a block, a "step" j = 0..7 is 32
+ * blocks of 256 columns; (tile, block) occupies 1536 bytes.  Tiles are taken in groups
+ * of four (the last group may have fewer): group g = tile / 4 has T = min(4, d_out/16 - 4 g)
+ * tiles and starts at 4 g * (d_in/256) * 1536; inside a group the blocks follow each
+ * other, and inside a block the group's tiles: (tile, block) sits at
+ *     (4 g * (d_in/256) + block * T + (tile - 4 g)) * 1536,
+ * so the 64 rows x 256 columns a group holds of one block are 6144 contiguous bytes.
+ * Inside a (tile, block) piece, a "step" j = 0..7 is 32
  * columns (8 groups of four), a "lane" is (g, t) = (lane / 4, lane % 4):
  *   value words, bytes [0, 1024):  word (j, lane) at (j / 4) * 512 + lane * 16 + (j % 4) * 4.
  *     It holds four value bytes B_i, i = 0..3, taken from row 16 tile + g + 8 (i % 2),
@@ -180,8 +185,10 @@ int oracle_repack_tiled(const uint8_t *vals, const uint8_t *meta, int d_out, int
     const int nblk = d_in / 256, tiles = d_out / 16;
     const size_t vrow = (size_t)d_in / 4, mrow = (size_t)d_in / 8;
     for (int tile = 0; tile < tiles; ++tile) {
+        const int g4 = 4 * (tile / 4);                          /* first tile of the group */
+        const int T = tiles - g4 < 4 ? tiles - g4 : 4;          /* tiles in the group */
         for (int blk = 0; blk < nblk; ++blk) {
-            uint8_t *base = out + ((size_t)tile * nblk + blk) * 1536;
+            uint8_t *base = out + ((size_t)g4 * nblk + (size_t)blk * T + (tile - g4)) * 1536;
             for (int j = 0; j < 8; ++j) {
                 for (int lane = 0; lane < 32; ++lane) {
                     const int g = lane / 4, t = lane % 4;

@@ -256,14 +256,17 @@ def dense_from_tiled(buf, d_out, d_in):
     """Read a decode-tiled buffer the way its consumer does (per lane and step: four
     value slots, index half-words from the lane that holds them) and rebuild the dense
     code matrix.  Written from the layout's description, not from the oracle's loops."""
-    nblk = d_in // 256
-    words = buf.view("<u4").reshape(d_out // 16, nblk, 384)
+    nblk, tiles = d_in // 256, d_out // 16
+    pieces = buf.view("<u4").reshape(tiles * nblk, 384)         # 1536-byte pieces in storage order
     dense = np.zeros((d_out, d_in), np.int64)
     sext = lambda n: n - 16 if n >= 8 else n
-    for tile in range(d_out // 16):
-        for blk in range(nblk):
-            wv = words[tile, blk, :256].reshape(2, 32, 4)       # [half of the steps][lane][word]
-            wm = words[tile, blk, 256:].reshape(32, 4)          # [lane][word]
+    # storage order: groups of four tiles; in a group block after block; in a block the group's tiles
+    order = [(g4 + t, blk) for g4 in range(0, tiles, 4) for blk in range(nblk) for t in range(min(4, tiles - g4))]
+    assert len(order) == tiles * nblk
+    for piece, (tile, blk) in enumerate(order):
+        if True:
+            wv = pieces[piece, :256].reshape(2, 32, 4)          # [half of the steps][lane][word]
+            wm = pieces[piece, 256:].reshape(32, 4)             # [lane][word]
             for j in range(8):
                 for lane in range(32):
                     g, t = divmod(lane, 4)
@@ -285,7 +288,7 @@ def dense_from_tiled(buf, d_out, d_in):
 
 def test_repack_tiled_keeps_every_code_and_position():
     rng = np.random.default_rng(5)
-    d_out, d_in = 48, 768
+    d_out, d_in = 112, 768      # seven tiles: one full group of four and a group of three
     codes = rng.integers(-8, 8, size=(d_out, d_in)).astype(np.int8)
     mask = inputs.top2_mask(rng.standard_normal((d_out, d_in)).astype(np.float32))
     vals, meta = oracle.pack(codes, mask)
@@ -294,6 +297,25 @@ def test_repack_tiled_keeps_every_code_and_position():
     assert np.array_equal(dense_from_tiled(tiled, d_out, d_in), codes.astype(np.int64) * mask)
     # a permutation of the input bits: same population of set bits
     assert int(np.unpackbits(tiled).sum()) == int(np.unpackbits(vals).sum() + np.unpackbits(meta).sum())
+
+
+def test_repack_tiled_group_order_by_hand():
+    """Where whole pieces go: 6 tiles x 2 blocks.  Group 0 (tiles 0-3) holds block 0 of tiles 0..3, then
+    block 1 of tiles 0..3; group 1 (tiles 4, 5; two tiles) holds block 0 of tiles 4, 5, then block 1."""
+    d_out, d_in = 96, 512
+    vals = np.zeros((d_out, d_in // 4), np.uint8)
+    meta = np.zeros((d_out, d_in // 8), np.uint8)
+    for tile in range(6):
+        for blk in range(2):
+            vals[16 * tile, 64 * blk] = 0x10 * tile + blk + 1      # row g = 0, group 0 of the block: lane 0, step 0, slot 0
+    out = oracle.repack_tiled(vals, meta).reshape(12, 1536)
+    where = {(0, 0): 0, (1, 0): 1, (2, 0): 2, (3, 0): 3, (0, 1): 4, (1, 1): 5, (2, 1): 6, (3, 1): 7,
+             (4, 0): 8, (5, 0): 9, (4, 1): 10, (5, 1): 11}
+    for (tile, blk), piece in where.items():
+        B = 0x10 * tile + blk + 1
+        w = int(out[piece, :4].view("<u4")[0])
+        assert w == (B & 15) | ((B >> 4) << 16), (tile, blk, piece, hex(w))
+        assert not out[piece, 4:].any()
 
 
 def test_repack_tiled_rejects_shapes_it_cannot_tile():
