@@ -124,7 +124,7 @@ __device__ __forceinline__ void sparse_block(float (&acc)[NT][4], uint32_t blk_a
 }
 
 // One step of 32 columns of a dense bf16 tile (16 rows x 64 columns = 128-byte rows,
-// 128-byte swizzle; `half` = which 32 columns) against B fragments in fragment order:
+// 128-byte swizzle, tile base a multiple of 2048 bytes inside a 1024-byte aligned box; `half` = which 32 columns) against B fragments in fragment order:
 // two m16n8k16 MMAs in natural column order.
 template <int NT>
 __device__ __forceinline__ void dense_step(float (&acc)[NT][4], uint32_t tile_addr, int half, const uint4 (&xb)[NT], const LaneCtx& lc) {

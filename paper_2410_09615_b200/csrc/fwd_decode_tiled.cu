@@ -1,35 +1,40 @@
 // Decode-phase forward (b <= 16) on the decode-tiled weight: one persistent cooperative kernel
 // that streams the weight and the adapters from HBM exactly once.
 //
-// Every consumer warp is a stream of its own.  The three operands are cut into slots of at
-// most 6 KB: a weight slot is MT row tiles of 16 rows x NB blocks of 256 columns of the
-// decode-tiled buffer (MT * NB = 4; contiguous pieces, fetched with cp.async.bulk), an
-// adapter slot is 16 rows x 128 columns of R or L (two TMA tiles).  A list of slots (R, then
-// the weight, then L) is divided evenly, in list order, among all consumer warps of the grid;
-// a warp fetches its slots through a private ring (it requests slot i + depth after it has
-// consumed slot i: no producer warp, no empty barriers, no barrier shared between warps) and
-// keeps the accumulators of the row tile it is walking in registers.  Whenever its range
-// leaves a row tile it writes the partial tile (fp32, MMA fragment order) to a slot of the
-// workspace.  Nothing is summed across warps in shared memory.
+// Slots.  The three operands are cut into slots of 6 KB, each fetched by ONE copy request (on B200 a
+// request costs about 300 ns of issue time whatever its size, and one instruction can start eight of
+// them side by side, so a CTA needs requests of several kilobytes to keep up with its share of HBM):
+//   weight slot   one 256-column block of a group of four row tiles of the tiled buffer (64 rows x 256
+//                 columns, contiguous there), fetched with cp.async.bulk;
+//   adapter slot  48 rows x 64 columns of R or of L (three 16-row tiles), one TMA box.
+// Lists.  All slots of R, then of the weight, then of L form lists that are divided evenly, in list
+// order, among all consumer warps of the grid.  A consumer warp owns a ring of slots in shared memory
+// and walks its share of each list front to back, with the accumulators of the rows it is walking in
+// registers; whenever its range leaves a group of rows it writes the partial tiles (fp32, MMA fragment
+// order) to its slots of the workspace.  Nothing is summed across warps in shared memory, and no
+// barrier is shared between consumer warps.  One producer warp requests the slots: lane w serves
+// consumer warp w and requests that warp's next slot as soon as its ring has room (full / empty
+// mbarrier pair per ring slot), so that the held requests do not sit in the warps that compute.
 //
 // Tensor-core mapping: the batch is the N dimension (one or two n-tiles of 8 tokens) of
-// mma.sp::ordered_metadata.m16n8k32 for the weight (the tiled buffer holds the A registers
-// and the metadata words as the instruction takes them) and of mma.m16n8k16 for the adapters.
-// Activations (and later T) sit in shared memory in B-fragment order, b tokens only.
+// mma.sp::ordered_metadata.m16n8k32 for the weight (the tiled buffer holds the A registers and the
+// metadata words as the instruction takes them) and of mma.m16n8k16 for the adapters.  Activations
+// (and later T) sit in shared memory in B-fragment order, b tokens only.
 //
-// Large d_in: the activation slice a CTA can hold is bounded, so d_in is cut into KS slices and
-// a CTA belongs to one slice for the R and weight phases (the L phase has no such limit).
+// Large d_in: the activation slice a CTA can hold is bounded, so d_in is cut into KS slices and a CTA
+// belongs to one slice for the R and weight phases (the L phase has no such limit).
 //
-// Hand-over between CTAs, without fences or grid barriers (the launch is cooperative, all
-// CTAs are resident): a partial-sum slot holds a reserved NaN pattern while empty; its one
-// reader polls it, takes the value and marks it empty again.
-//   T = X R^T:   service warps (four per CTA) sum the partials of a 16-column piece in list
-//                order, round to bf16 and publish {two columns, call number} as one 64-bit
-//                word; the call number comes from a counter every CTA increments when it
-//                leaves.  The same warps then bring all of T into shared memory while the
-//                weight phase runs, and arrive on a barrier the consumers wait on before L.
-//   Y:           after its L range a warp finishes whole 16-row output tiles:
-//                Y = s * sum(weight partials) + sum(adapter partials), in list order.
+// Hand-over between CTAs, without fences or grid barriers (the launch is cooperative, all CTAs are
+// resident): a partial-sum slot holds a reserved NaN pattern while empty; its one reader polls it,
+// takes the value and marks it empty again.
+//   T = X R^T:   service warps (three per CTA) sum the partials of a 16-column piece in list order,
+//                round to bf16 and publish {two columns, call number} as one 64-bit word; the call
+//                number comes from a counter every CTA increments when it leaves.  The same warps then
+//                bring all of T into shared memory while the weight phase runs, and arrive on a barrier
+//                the consumers wait on before L.
+//   Y:           the warp that holds the first L slot of a group of rows finishes those output tiles
+//                when it leaves them:  Y = s * sum(weight partials) + sum(adapter partials), in list
+//                order (without adapters: a last pass over the tiles).
 // All polls are bounded; an expired one sets SLIM_ERR_TIMEOUT and the kernel runs on.
 // Reductions have a fixed order: results are bit-identical from run to run.
 #include <cuda.h>
@@ -47,12 +52,17 @@ constexpr int kCW = 8;                                  // consumer warps
 constexpr int kProducerWarp = kCW;                      // one warp requests every slot of the CTA
 constexpr int kSW = 3;                                  // service warps
 constexpr int kThreads = (kCW + 1 + kSW) * 32;
-constexpr int kBlockBytes = 1536;                       // one 16-row x 256-column block of the tiled weight
+constexpr int kWT = 4;                                  // row tiles of a weight slot (a group of the tiled layout)
+constexpr int kAT = 3;                                  // row tiles of an adapter slot (48 rows)
+constexpr int kACols = 64;                              // columns of an adapter slot (two steps of 32)
+constexpr int kSlotBytes = 6144;
+constexpr int kBlockBytes = 1536;                       // one 16-row x 256-column piece of the tiled weight
 constexpr int kMaxRing = 8;                             // slots per warp
-constexpr int kDCols = 128;                             // adapter columns per slot
 constexpr int kMaxRank = 3072;
+constexpr int kMaxKS = 64;                              // k-slices the shared-memory tables hold
 constexpr size_t kSmemBudget = 227 * 1024;
-constexpr uint32_t kPollLimit = 1u << 22;
+constexpr uint32_t kPollLimit = 1u << 20;
+constexpr uint32_t kPollPause = 400;                    // ns between two polls of a slot: waiting warps must not flood the L2
 constexpr uint32_t kMbarSpinLimit = 1u << 26;
 constexpr uint32_t kEmpty = 0xFFFFFFFFu;                // "no value yet" in a partial-sum slot
 constexpr uint32_t kNanBits = 0x7FFFFFFFu;              // what a computed all-ones NaN is stored as
@@ -69,18 +79,18 @@ struct Params {
     int b, r, d_out, d_in;
     int KS, G;                           // k-slices; CTAs per slice
     int nblk;                            // 256-column blocks of a row
-    int NB;                              // blocks per weight slot (MT * NB = 4)
-    int unitsW, tilesW, tilesR, nqL;     // ceil(tilesW / MT); d_out / 16; r / 16; ceil(r / 128)
+    int tilesW, tilesR;                  // d_out / 16; r / 16
+    int unitsW, unitsR, unitsL;          // groups of kWT weight tiles; of kAT tiles of R; of kAT tiles of L
+    int nqL;                             // adapter slots along r: ceil(r / 64)
     int wnR;                             // workers per slice in the R phase (<= G * kCW)
     int muW, muR, muL;                   // partial slots a worker owns in each phase
-    int ring, slot_bytes;                // ring slots per warp; bytes between slots (a multiple of 1024)
+    int ring;                            // ring slots per warp
     int x_bytes;                         // activation slice region
 };
 
 // Optional timeline: built with -DSLIM_TILED_TRACE, lane 0 of consumer warp 0 (entries 0-7) and of service
 // warp 0 (entries 8-9) of every CTA record the global timer (read back with slim_debug_read_tiled_trace).
 #ifdef SLIM_TILED_TRACE
-__device__ unsigned long long g_tiled_dbg[16];
 __device__ unsigned long long g_tiled_trace[256 * 16];
 #define TSTAMP(w, i) do { if (warp == (w) && lane == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_tiled_trace[blockIdx.x * 16 + (i)] = t_; } } while (0)
 #else
@@ -136,6 +146,14 @@ __device__ __forceinline__ unsigned long long ld_gpu64(const unsigned long long*
 __device__ __forceinline__ void st_gpu64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" :: "l"(p), "l"(v) : "memory");
 }
+__device__ __forceinline__ uint4 ld_gpu_v4(const uint32_t* p) {
+    uint4 v;
+    asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_gpu_v4(uint32_t* p, uint4 v) {
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 __device__ __forceinline__ uint32_t slot_bits(float v) {    // fp32 bits that never equal kEmpty
     const uint32_t u = __float_as_uint(v);
     return u == kEmpty ? kNanBits : u;
@@ -147,10 +165,6 @@ struct Split { int len, rem; };
 __host__ __device__ __forceinline__ Split make_split(int S, int Wn) { Split sp; sp.len = S / Wn; sp.rem = S % Wn; return sp; }
 __host__ __device__ __forceinline__ int split_start(const Split& sp, int w) { return w * sp.len + (w < sp.rem ? w : sp.rem); }
 __host__ __device__ __forceinline__ int split_count(const Split& sp, int w) { return sp.len + (w < sp.rem ? 1 : 0); }
-__host__ __device__ __forceinline__ int split_owner(const Split& sp, int pos) {
-    const int edge = sp.rem * (sp.len + 1);
-    return pos < edge ? pos / (sp.len + 1) : sp.rem + (pos - edge) / sp.len;   // pos >= edge implies len > 0
-}
 
 // Blocks [b0, b1) of k-slice ks.
 __host__ __device__ __forceinline__ void slice_blocks(int ks, int KS, int nblk, int* b0, int* b1) {
@@ -158,21 +172,45 @@ __host__ __device__ __forceinline__ void slice_blocks(int ks, int KS, int nblk, 
     *b1 = (int)((long long)(ks + 1) * nblk / KS);
 }
 
+// One list as its readers need it, kept in shared memory: nq slots per unit, divided among the workers as
+// `len` slots each plus one more for the first `rem`; reciprocals for division by multiplication (a
+// hardware integer division is a long chain of dependent instructions).
+struct ListTab { int nq, len, rem, edge; float r_nq, r_len, r_len1; };
+__device__ __forceinline__ ListTab make_tab(int units, int nq, int Wn) {
+    ListTab t;
+    const Split sp = make_split(units * nq, Wn);
+    t.nq = nq; t.len = sp.len; t.rem = sp.rem; t.edge = sp.rem * (sp.len + 1);
+    t.r_nq = nq > 0 ? 1.f / (float)nq : 0.f; t.r_len = sp.len > 0 ? 1.f / (float)sp.len : 0.f; t.r_len1 = 1.f / (float)(sp.len + 1);
+    return t;
+}
+// n / d for 0 <= n < 2^22, d > 0, rd = 1 / d: the float product is off by less than one, fixed up exactly.
+__device__ __forceinline__ int fdiv(int n, int d, float rd) {
+    int q = __float2int_rz(__int2float_rn(n) * rd);
+    const int r = n - q * d;
+    if (r < 0) --q; else if (r >= d) ++q;
+    return q;
+}
+__device__ __forceinline__ int tab_owner(const ListTab& t, int pos) {
+    return pos < t.edge ? fdiv(pos, t.len + 1, t.r_len1) : t.rem + fdiv(pos - t.edge, t.len, t.r_len);
+}
+__device__ __forceinline__ int tab_first_unit(const ListTab& t, int w) {      // first unit the range of worker w meets
+    return fdiv(w * t.len + min(w, t.rem), t.nq, t.r_nq);
+}
+
 // Walks, in list order, the partial-sum slots that the workers of one phase left for one list
 // unit: every worker whose range meets the unit's positions owns `mu` slots of `stride` words,
 // the unit's being number (unit - first unit of the worker's range).
 struct PartWalk {
-    const Split sp; const int nq, mu, unit; const size_t stride; uint32_t* const base;
+    const ListTab& t; const int mu, unit; const size_t stride; uint32_t* const base;
     int w, w_last;
-    __device__ PartWalk(uint32_t* base_, const Split& sp_, int nq_, int mu_, int unit_, size_t stride_, int worker0)
-        : sp(sp_), nq(nq_), mu(mu_), unit(unit_), stride(stride_), base(base_ + (size_t)worker0 * mu_ * stride_) {
-        w = nq > 0 ? split_owner(sp, unit * nq) : 0;
-        w_last = nq > 0 ? split_owner(sp, unit * nq + nq - 1) : -1;
+    __device__ PartWalk(uint32_t* base_, const ListTab& t_, int mu_, int unit_, size_t stride_, int worker0)
+        : t(t_), mu(mu_), unit(unit_), stride(stride_), base(base_ + (size_t)worker0 * mu_ * stride_) {
+        w = t.nq > 0 ? tab_owner(t, unit * t.nq) : 0;
+        w_last = t.nq > 0 ? tab_owner(t, unit * t.nq + t.nq - 1) : -1;
     }
     __device__ uint32_t* next() {
         if (w > w_last) return nullptr;
-        const int u0 = split_start(sp, w) / nq;
-        uint32_t* p = base + ((size_t)w * mu + (unit - u0)) * stride;
+        uint32_t* p = base + ((size_t)w * mu + (unit - tab_first_unit(t, w))) * stride;
         ++w;
         return p;
     }
@@ -202,6 +240,7 @@ __device__ __forceinline__ bool take_batch(PartWalk& pw, int off, int lane, floa
                 if (v[k][e] == kEmpty) { v[k][e] = ld_gpu(ptr[k] + off + e * 32 + lane); all = false; }
         if (all) break;
         if (spins > kPollLimit) { *ok = false; break; }
+        __nanosleep(kPollPause);
     }
 #pragma unroll
     for (int k = 0; k < kBatch; ++k)
@@ -215,6 +254,87 @@ __device__ __forceinline__ bool take_batch(PartWalk& pw, int off, int lane, floa
     return ptr[kBatch - 1] != nullptr;
 }
 
+constexpr int kFinishers = kCW + kSW;      // warps of a CTA that finish output tiles once their other work is done
+
+// Finishes the output tiles of finisher `fid` of `n_fin`: Y = s * (weight partials of every k-slice, in list
+// order) + (adapter partials, in list order), rounded to bf16.  Tiles are dealt out in order; a tile's
+// partials are complete once every consumer warp has walked past its rows.
+template <int NT>
+__device__ __forceinline__ void finish_tiles(const Params& p, const ListTab* tabW, const ListTab* tabL, int fid, int n_fin,
+                                             const LaneCtx& lc, uint32_t* expired) {
+    constexpr int frag = NT * 128, E = NT * 4;
+    constexpr int kFB = 8;                              // partials requested together (this code runs once per call and
+                                                        // comes cold from the L2: it is kept small)
+    const int lane = lc.lane;
+    const Split spF = make_split(p.tilesW, n_fin);
+    const int f0 = split_start(spF, fid), f1 = f0 + split_count(spF, fid);
+    for (int tile = f0; tile < f1; ++tile) {
+        float psum[E], asum[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) { psum[e] = 0.f; asum[e] = 0.f; }
+        const int uW = tile / kWT, mW = tile % kWT, uL = tile / kAT, mL = tile % kAT;
+        // walk state: k-slice of the weight partials being walked (p.KS = the adapter partials, then the end)
+        int k2 = -1, w = 0, w_last = -1;
+        auto next_part = [&](bool* is_adapter) -> uint32_t* {
+            while (w > w_last) {
+                ++k2;
+                if (k2 > p.KS || (k2 == p.KS && p.r == 0)) return nullptr;
+                const ListTab& t = k2 < p.KS ? tabW[k2] : tabL[0];
+                const int u = k2 < p.KS ? uW : uL;
+                w = tab_owner(t, u * t.nq); w_last = tab_owner(t, u * t.nq + t.nq - 1);
+            }
+            uint32_t* ptr;
+            if (k2 < p.KS) ptr = p.Ppart + (((size_t)(k2 * p.G * kCW + w) * p.muW + (uW - tab_first_unit(tabW[k2], w))) * kWT + mW) * frag;
+            else           ptr = p.Apart + (((size_t)w * p.muL + (uL - tab_first_unit(tabL[0], w))) * kAT + mL) * frag;
+            *is_adapter = k2 == p.KS;
+            ++w;
+            return ptr;
+        };
+        for (bool more = true; more;) {
+            uint32_t* ptr[kFB];
+            bool adapter[kFB];
+#pragma unroll
+            for (int k = 0; k < kFB; ++k) { adapter[k] = false; ptr[k] = more ? next_part(&adapter[k]) : nullptr; if (!ptr[k]) more = false; }
+            uint4 v[kFB][NT];
+#pragma unroll
+            for (int k = 0; k < kFB; ++k)
+#pragma unroll
+                for (int h = 0; h < NT; ++h) v[k][h] = ptr[k] ? ld_gpu_v4(ptr[k] + lane * E + 4 * h) : make_uint4(0, 0, 0, 0);
+            for (uint32_t spins = 0;; ++spins) {
+                bool all = true;
+#pragma unroll
+                for (int k = 0; k < kFB; ++k)
+#pragma unroll
+                    for (int h = 0; h < NT; ++h)
+                        if (v[k][h].x == kEmpty || v[k][h].y == kEmpty || v[k][h].z == kEmpty || v[k][h].w == kEmpty) {
+                            v[k][h] = ld_gpu_v4(ptr[k] + lane * E + 4 * h); all = false;
+                        }
+                if (all) break;
+                if (spins > kPollLimit) { *expired |= 16u; break; }
+                __nanosleep(kPollPause);
+            }
+#pragma unroll
+            for (int k = 0; k < kFB; ++k)
+                if (ptr[k]) {
+#pragma unroll
+                    for (int h = 0; h < NT; ++h) {
+                        float* dstsum = adapter[k] ? asum : psum;
+                        dstsum[4 * h + 0] += __uint_as_float(v[k][h].x); dstsum[4 * h + 1] += __uint_as_float(v[k][h].y);
+                        dstsum[4 * h + 2] += __uint_as_float(v[k][h].z); dstsum[4 * h + 3] += __uint_as_float(v[k][h].w);
+                        st_gpu_v4(ptr[k] + lane * E + 4 * h, make_uint4(kEmpty, kEmpty, kEmpty, kEmpty));
+                    }
+                }
+        }
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int h = e >> 2, q = e & 3;
+            const int n = tile * 16 + lc.g + 8 * (q >> 1);
+            const int tok = 8 * h + 2 * lc.t + (q & 1);
+            if (tok < p.b) p.Y[(size_t)tok * p.d_out + n] = __float2bfloat16_rn(fmaf(psum[e], p.s, asum[e]));
+        }
+    }
+}
+
 // The jobs of one consumer warp: nR slots of the R list from sR, nW of the weight list, nL of the L list.
 struct Jobs { int nR, sR, nW, sW, nL, sL, total; };
 struct SliceGeo { bool in_slice; int ks, grp, blk0, blk1, nqW, nqR; };
@@ -225,14 +345,14 @@ __device__ __forceinline__ SliceGeo make_geo(const Params& p, int cta) {
     g.ks = g.in_slice ? cta % p.KS : 0;
     g.grp = g.in_slice ? cta / p.KS : 0;
     slice_blocks(g.ks, p.KS, p.nblk, &g.blk0, &g.blk1);
-    g.nqW = ceil_div(g.blk1 - g.blk0, p.NB);              // weight slots per unit in this slice
-    g.nqR = (g.blk1 - g.blk0) * 2;                        // adapter slots per R tile in this slice
+    g.nqW = g.blk1 - g.blk0;                              // weight slots per group of rows in this slice
+    g.nqR = (g.blk1 - g.blk0) * (256 / kACols);           // adapter slots per group of R rows in this slice
     return g;
 }
 __device__ __forceinline__ Jobs make_jobs(const Params& p, const SliceGeo& g, int cta, int n_ctas, int cwarp) {
-    const Split spR = make_split(p.tilesR * g.nqR, p.wnR);
+    const Split spR = make_split(p.unitsR * g.nqR, p.wnR);
     const Split spW = make_split(p.unitsW * g.nqW, p.G * kCW);
-    const Split spL = make_split(p.tilesW * p.nqL, n_ctas * kCW);
+    const Split spL = make_split(p.unitsL * p.nqL, n_ctas * kCW);
     const int wi = g.grp * kCW + cwarp;                   // worker number inside the slice
     const int wl = cta * kCW + cwarp;                     // worker number in the grid
     Jobs jb;
@@ -243,7 +363,7 @@ __device__ __forceinline__ Jobs make_jobs(const Params& p, const SliceGeo& g, in
     return jb;
 }
 
-template <int NT, int MT>
+template <int NT>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmL)
 {
@@ -252,17 +372,19 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
     extern __shared__ unsigned char smem_raw[];
     // layout (1024-byte aligned for the swizzle): rings | X slice | T | barriers
     unsigned char* rings = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char* xs = rings + (size_t)kCW * p.ring * p.slot_bytes;
+    unsigned char* xs = rings + (size_t)kCW * p.ring * kSlotBytes;
     unsigned char* ts = xs + p.x_bytes;
-    const int t_bytes = p.nqL * 4 * p.b * 64;
+    const int t_bytes = p.nqL * 2 * p.b * 64;
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(ts + t_bytes);      // [kCW][kMaxRing]
     uint64_t* empty_bar = full_bar + kCW * kMaxRing;                     // [kCW][kMaxRing]
     uint64_t* t_bar = empty_bar + kCW * kMaxRing;
+    ListTab* tabW = reinterpret_cast<ListTab*>(t_bar + 1);              // [KS] weight list of every k-slice
+    ListTab* tabR = tabW + kMaxKS;                                       // [KS] R list of every k-slice
+    ListTab* tabL = tabR + kMaxKS;                                       // [1]  L list
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_ctas = gridDim.x, cta = blockIdx.x;
     const LaneCtx lc = make_lane_ctx(lane);
-    const int NB = p.NB;
     const SliceGeo geo = make_geo(p, cta);
     const int blk0 = geo.blk0, blk1 = geo.blk1, nqW = geo.nqW, nqR = geo.nqR, ks = geo.ks;
 
@@ -271,6 +393,13 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
         mbar_init(t_bar, kSW);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    for (int k2 = threadIdx.x; k2 < p.KS; k2 += kThreads) {
+        int c0, c1;
+        slice_blocks(k2, p.KS, p.nblk, &c0, &c1);
+        tabW[k2] = make_tab(p.unitsW, c1 - c0, p.G * kCW);
+        tabR[k2] = make_tab(p.unitsR, (c1 - c0) * (256 / kACols), p.wnR);
+    }
+    if (threadIdx.x == kThreads - 1) tabL[0] = make_tab(p.unitsL, p.nqL, gridDim.x * kCW);
     __syncthreads();
 
     // which kind of wait expired, if any: reported in bits 16-23 of the status word beside SLIM_ERR_TIMEOUT
@@ -283,28 +412,21 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
 #endif
     if (warp == kProducerWarp) {
         // ================================ producer warp ================================
-        // Lane w < kCW requests the slots of consumer warp w, in that warp's job order, as its ring
-        // slots come free.  A request is held until the copy engine has room for it (with full rings
-        // that is most of the time), so it must not sit in the warps that compute.
+        // Every lane walks the job list of its consumer warp at its own pace: in each round a lane whose
+        // next ring slot is free (a test that does not wait) requests its next job, the others sit the
+        // round out; the requests of a round start with one instruction per list kind.
         const bool serves = lane < kCW;
         const Jobs jb = make_jobs(p, geo, cta, n_ctas, serves ? lane : 0);
         const int total = serves ? jb.total : 0;
-        int longest = total;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) longest = max(longest, __shfl_xor_sync(0xffffffffu, longest, o));
         uint64_t* fbar = full_bar + (serves ? lane : 0) * kMaxRing;
         uint64_t* ebar = empty_bar + (serves ? lane : 0) * kMaxRing;
-        const uint32_t ring0 = smem_u32(rings + (size_t)(serves ? lane : 0) * p.ring * p.slot_bytes);
-        // running (unit, slot in unit) of this lane's position in each list
-        int r_tile = nqR > 0 ? jb.sR / nqR : 0, r_q = nqR > 0 ? jb.sR % nqR : 0;
+        const uint32_t ring0 = smem_u32(rings + (size_t)(serves ? lane : 0) * p.ring * kSlotBytes);
+        // running (group of rows, slot in group) of this lane's position in each list
+        int r_u = nqR > 0 ? jb.sR / nqR : 0, r_q = nqR > 0 ? jb.sR % nqR : 0;
         int w_u = jb.sW / nqW, w_q = jb.sW % nqW;
-        int l_tile = p.nqL > 0 ? jb.sL / p.nqL : 0, l_q = p.nqL > 0 ? jb.sL % p.nqL : 0;
-        // Every lane walks its own job list at its own pace: in each round a lane whose next ring slot is
-        // free (a test that does not wait) requests its next job, the others sit the round out, so one slow
-        // consumer does not hold up the requests of the other seven.
+        int l_u = p.nqL > 0 ? jb.sL / p.nqL : 0, l_q = p.nqL > 0 ? jb.sL % p.nqL : 0;
         int j = 0, slot = 0;
         uint32_t parity = 0;                                // phase of the "slot left" barrier awaited in the second lap; flips per lap
-        (void)longest;
         for (uint32_t idle = 0;;) {
             const bool has = j < total;
             if (!__any_sync(0xffffffffu, has)) break;
@@ -317,26 +439,21 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
             }
             if (can) {
                 uint64_t* bar = &fbar[slot];
-                const uint32_t dst = ring0 + slot * p.slot_bytes;
+                const uint32_t dst = ring0 + slot * kSlotBytes;
                 if (j < jb.nR) {
-                    mbar_arrive_expect_tx(bar, 4096);
-                    tma_tile(dst, &tmR, blk0 * 256 + r_q * kDCols, r_tile * 16, bar);
-                    tma_tile(dst + 2048, &tmR, blk0 * 256 + r_q * kDCols + 64, r_tile * 16, bar);
-                    if (++r_q == nqR) { r_q = 0; ++r_tile; }
+                    mbar_arrive_expect_tx(bar, kSlotBytes);
+                    tma_tile(dst, &tmR, blk0 * 256 + r_q * kACols, r_u * (16 * kAT), bar);
+                    if (++r_q == nqR) { r_q = 0; ++r_u; }
                 } else if (j < jb.nR + jb.nW) {
-                    const int nb = min(NB, blk1 - blk0 - w_q * NB), mt = min(MT, p.tilesW - w_u * MT);
-                    mbar_arrive_expect_tx(bar, (uint32_t)(mt * nb * kBlockBytes));
-#pragma unroll
-                    for (int m = 0; m < MT; ++m)
-                        if (m < mt)
-                            bulk_copy(dst + m * NB * kBlockBytes,
-                                      p.W + ((size_t)(w_u * MT + m) * p.nblk + blk0 + w_q * NB) * kBlockBytes, (uint32_t)(nb * kBlockBytes), bar);
+                    const int tg = min(kWT, p.tilesW - w_u * kWT);                  // tiles of this group
+                    mbar_arrive_expect_tx(bar, (uint32_t)(tg * kBlockBytes));
+                    bulk_copy(dst, p.W + ((size_t)w_u * kWT * p.nblk + (size_t)(blk0 + w_q) * tg) * kBlockBytes,
+                              (uint32_t)(tg * kBlockBytes), bar);
                     if (++w_q == nqW) { w_q = 0; ++w_u; }
                 } else {
-                    mbar_arrive_expect_tx(bar, 4096);
-                    tma_tile(dst, &tmL, l_q * kDCols, l_tile * 16, bar);
-                    tma_tile(dst + 2048, &tmL, l_q * kDCols + 64, l_tile * 16, bar);
-                    if (++l_q == p.nqL) { l_q = 0; ++l_tile; }
+                    mbar_arrive_expect_tx(bar, kSlotBytes);
+                    tma_tile(dst, &tmL, l_q * kACols, l_u * (16 * kAT), bar);
+                    if (++l_q == p.nqL) { l_q = 0; ++l_u; }
                 }
                 if (++slot == p.ring) { slot = 0; if (j >= p.ring) parity ^= 1u; }
                 ++j;
@@ -351,11 +468,10 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
         // ================================ consumer warps ================================
         const Jobs jb = make_jobs(p, geo, cta, n_ctas, warp);
         const int nR = jb.nR, sR = jb.sR, nW = jb.nW, sW = jb.sW, nL = jb.nL, sL = jb.sL;
-        const Split spL = make_split(p.tilesW * p.nqL, n_ctas * kCW);
         const int wi = geo.grp * kCW + warp, wl = cta * kCW + warp;
         uint64_t* my_full = full_bar + warp * kMaxRing;
         uint64_t* my_empty = empty_bar + warp * kMaxRing;
-        const uint32_t my_ring = smem_u32(rings + (size_t)warp * p.ring * p.slot_bytes);
+        const uint32_t my_ring = smem_u32(rings + (size_t)warp * p.ring * kSlotBytes);
 
         // ---- the CTA's slice of the activations into shared memory, fragment order.  A thread
         // requests several 16-byte pieces before it stores the first (one global round trip per batch).
@@ -390,129 +506,64 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
         TSTAMP(0, 1);
 
         const uint32_t xs_addr = smem_u32(xs), ts_addr = smem_u32(ts);
-        uint32_t* const Pmine = p.Ppart + ((size_t)(ks * p.G * kCW + wi) * p.muW) * (MT * frag);
-        uint32_t* const Tmine = p.Tpart + ((size_t)(ks * p.wnR + wi) * p.muR) * frag;
-        uint32_t* const Amine = p.Apart + ((size_t)wl * p.muL) * frag;
+        uint32_t* const Pmine = p.Ppart + ((size_t)(ks * p.G * kCW + wi) * p.muW) * (kWT * frag);
+        uint32_t* const Tmine = p.Tpart + ((size_t)(ks * p.wnR + wi) * p.muR) * (kAT * frag);
+        uint32_t* const Amine = p.Apart + ((size_t)wl * p.muL) * (kAT * frag);
 
-        float acc[MT][NT][4];
+        float acc[kWT][NT][4];                              // weight phase: four row tiles; adapter phases: the first three
         auto zero_acc = [&]() {
 #pragma unroll
-            for (int m = 0; m < MT; ++m)
+            for (int m = 0; m < kWT; ++m)
 #pragma unroll
                 for (int h = 0; h < NT; ++h)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) acc[m][h][e] = 0.f;
         };
+        // a partial tile in the workspace: lane-major, word lane * E + 4 h + e (every word is its own "empty" flag)
         auto store_tile = [&](uint32_t* dst, const float (&a)[NT][4]) {
 #pragma unroll
             for (int h = 0; h < NT; ++h)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) st_gpu(dst + (h * 4 + e) * 32 + lane, slot_bits(a[h][e]));
-        };
-
-        // Finishes output tile `tile`: s * (weight partials of every k-slice, in list order) + (own[] +
-        // the adapter partials of the workers from first_w on, in list order), rounded to bf16.
-        auto finish_tile = [&](int tile, const float (&own)[NT][4], int first_w) {
-            float psum[E], asum[E];
-#pragma unroll
-            for (int h = 0; h < NT; ++h)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) { psum[h * 4 + e] = 0.f; asum[h * 4 + e] = own[h][e]; }
-            const int u = tile / MT, m = tile % MT;
-            // walk state: k-slice of the weight partials being walked (p.KS = the adapter partials, then the end)
-            int k2 = -1, w = 0, w_last = -1, nq2 = 1;
-            Split sp2 = spL;
-            auto next_part = [&](bool* is_adapter) -> uint32_t* {
-                while (w > w_last) {
-                    ++k2;
-                    if (k2 > p.KS || (k2 == p.KS && p.r == 0)) return nullptr;
-                    if (k2 < p.KS) {
-                        int c0, c1;
-                        slice_blocks(k2, p.KS, p.nblk, &c0, &c1);
-                        nq2 = ceil_div(c1 - c0, NB);
-                        sp2 = make_split(p.unitsW * nq2, p.G * kCW);
-                        w = split_owner(sp2, u * nq2); w_last = split_owner(sp2, u * nq2 + nq2 - 1);
-                    } else {
-                        nq2 = p.nqL; sp2 = spL;
-                        w = first_w; w_last = split_owner(sp2, tile * nq2 + nq2 - 1);
-                    }
-                }
-                const int u0 = split_start(sp2, w) / nq2;
-                uint32_t* ptr;
-                if (k2 < p.KS) ptr = p.Ppart + (((size_t)(k2 * p.G * kCW + w) * p.muW + (u - u0)) * MT + m) * frag;
-                else           ptr = p.Apart + ((size_t)w * p.muL + (tile - u0)) * frag;
-                *is_adapter = k2 == p.KS;
-                ++w;
-                return ptr;
-            };
-            constexpr int kFB = NT == 1 ? 16 : 8;           // partials requested together: one round trip for most tiles
-            for (bool more = true; more;) {
-                uint32_t* ptr[kFB];
-                bool adapter[kFB];
-#pragma unroll
-                for (int k = 0; k < kFB; ++k) { adapter[k] = false; ptr[k] = more ? next_part(&adapter[k]) : nullptr; if (!ptr[k]) more = false; }
-                uint32_t v[kFB][E];
-#pragma unroll
-                for (int k = 0; k < kFB; ++k)
-#pragma unroll
-                    for (int e = 0; e < E; ++e) v[k][e] = ptr[k] ? ld_gpu(ptr[k] + e * 32 + lane) : 0u;
-                for (uint32_t spins = 0;; ++spins) {
-                    bool all = true;
-#pragma unroll
-                    for (int k = 0; k < kFB; ++k)
-#pragma unroll
-                        for (int e = 0; e < E; ++e)
-                            if (v[k][e] == kEmpty) { v[k][e] = ld_gpu(ptr[k] + e * 32 + lane); all = false; }
-                    if (all) break;
-                    if (spins > kPollLimit) { expired |= 16u; break; }
-                }
-#pragma unroll
-                for (int k = 0; k < kFB; ++k)
-                    if (ptr[k]) {
-#pragma unroll
-                        for (int e = 0; e < E; ++e) {
-                            if (adapter[k]) asum[e] += __uint_as_float(v[k][e]); else psum[e] += __uint_as_float(v[k][e]);
-                            st_gpu(ptr[k] + e * 32 + lane, kEmpty);
-                        }
-                    }
-            }
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const int h = e >> 2, q = e & 3;
-                const int n = tile * 16 + lc.g + 8 * (q >> 1);
-                const int tok = 8 * h + 2 * lc.t + (q & 1);
-                if (tok < p.b) p.Y[(size_t)tok * p.d_out + n] = __float2bfloat16_rn(fmaf(psum[e], p.s, asum[e]));
-            }
+                st_gpu_v4(dst + lane * E + 4 * h, make_uint4(slot_bits(a[h][0]), slot_bits(a[h][1]), slot_bits(a[h][2]), slot_bits(a[h][3])));
         };
 
         zero_acc();
-        // Walk of the three lists with running (unit, slot in unit) pairs and a running ring position:
-        // no division inside the loops (a division is a long chain of dependent instructions, and a warp
-        // has only one or two others on its scheduler to hide it behind).
+        // Walk of the three lists with running (group of rows, slot in group) pairs and a running ring
+        // position: no division inside the loops (a division is a long chain of dependent instructions, and
+        // a warp has only one or two others on its scheduler to hide it behind).
         int slot = 0; uint32_t parity = 0;
         auto next_slot = [&]() { if (++slot == p.ring) { slot = 0; parity ^= 1u; } };
         const int r_first = nqR > 0 ? sR / nqR : 0, w_first = sW / nqW, l_first = p.nqL > 0 ? sL / p.nqL : 0;
 
         // ---------------------------------------------------------------- R slots
         {
-            int tile = r_first, q = nqR > 0 ? sR % nqR : 0;
+            int u = r_first, q = nqR > 0 ? sR % nqR : 0;
             for (int j = 0; j < nR; ++j) {
-                const uint32_t src = my_ring + slot * p.slot_bytes;
+                const uint32_t src = my_ring + slot * kSlotBytes;
+                const int mt = min(kAT, p.tilesR - u * kAT);
                 if (!mbar_wait(&my_full[slot], parity)) expired |= 1u;
                 if (j == 0) TSTAMP(0, 2);
 #pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
+                for (int jj = 0; jj < 2; ++jj) {
                     uint4 xb[NT];
-                    load_x_step<NT>(xb, xs_addr, q * 4 + jj, p.b, lc);
-                    dense_step<NT>(acc[0], src + (jj >> 1) * 2048, jj & 1, xb, lc);
+                    load_x_step<NT>(xb, xs_addr, q * 2 + jj, p.b, lc);
+                    if (mt == kAT) {
+#pragma unroll
+                        for (int m = 0; m < kAT; ++m) dense_step<NT>(acc[m], src + m * 2048, jj, xb, lc);
+                    } else {
+#pragma unroll
+                        for (int m = 0; m < kAT; ++m)
+                            if (m < mt) dense_step<NT>(acc[m], src + m * 2048, jj, xb, lc);
+                    }
                 }
                 __syncwarp();                               // every lane is done reading the slot
                 if (lane == 0) mbar_arrive(&my_empty[slot]);
                 next_slot();
-                if (++q == nqR || j + 1 == nR) {            // leaving the tile: its partial goes to the workspace
-                    store_tile(Tmine + (size_t)(tile - r_first) * frag, acc[0]);
+                if (++q == nqR || j + 1 == nR) {            // leaving the rows: their partials go to the workspace
+#pragma unroll
+                    for (int m = 0; m < kAT; ++m)
+                        if (m < mt) store_tile(Tmine + ((size_t)(u - r_first) * kAT + m) * frag, acc[m]);
                     zero_acc();
-                    q = 0; ++tile;
+                    q = 0; ++u;
                 }
             }
         }
@@ -520,8 +571,8 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
         {
             int u = w_first, q = sW % nqW;
             for (int j = 0; j < nW; ++j) {
-                const uint32_t src = my_ring + slot * p.slot_bytes;
-                const int nb = min(NB, blk1 - blk0 - q * NB), mt = min(MT, p.tilesW - u * MT);
+                const uint32_t src = my_ring + slot * kSlotBytes;
+                const int mt = min(kWT, p.tilesW - u * kWT);
 #ifdef SLIM_TILED_TRACE
                 const long long w0_ = clock64();
 #endif
@@ -531,14 +582,16 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
                 if (warp == 0 && lane == 0) { g_tiled_trace[blockIdx.x * 16 + 11] += c0_ - w0_; g_tiled_trace[blockIdx.x * 16 + 12] += 1; }
 #endif
                 if (j == 0) TSTAMP(0, 3);
+                {
+                    uint4 xf[8][NT];
+                    load_x_block<NT>(xf, xs_addr, q * 8, p.b, lc);
+                    if (mt == kWT) {                          // the usual case, free of branches between the tiles
 #pragma unroll
-                for (int bi = 0; bi < 4 / MT; ++bi) {
-                    if (bi < nb) {
-                        uint4 xf[8][NT];
-                        load_x_block<NT>(xf, xs_addr, (q * NB + bi) * 8, p.b, lc);
+                        for (int m = 0; m < kWT; ++m) sparse_block<NT>(acc[m], src + m * kBlockBytes, xf, lc);
+                    } else {
 #pragma unroll
-                        for (int m = 0; m < MT; ++m)
-                            if (m < mt) sparse_block<NT>(acc[m], src + (m * NB + bi) * kBlockBytes, xf, lc);
+                        for (int m = 0; m < kWT; ++m)
+                            if (m < mt) sparse_block<NT>(acc[m], src + m * kBlockBytes, xf, lc);
                     }
                 }
 #ifdef SLIM_TILED_TRACE
@@ -549,7 +602,8 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
                 next_slot();
                 if (++q == nqW || j + 1 == nW) {
 #pragma unroll
-                    for (int m = 0; m < MT; ++m) store_tile(Pmine + ((size_t)(u - w_first) * MT + m) * frag, acc[m]);
+                    for (int m = 0; m < kWT; ++m)
+                        if (m < mt) store_tile(Pmine + ((size_t)(u - w_first) * kWT + m) * frag, acc[m]);
                     zero_acc();
                     q = 0; ++u;
                 }
@@ -560,46 +614,46 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
             TSTAMP(0, 4);
             if (!mbar_wait(t_bar, 0)) expired |= 4u;        // all of T is in shared memory
             TSTAMP(0, 5);
-            int tile = l_first, q = sL % p.nqL;
-            bool head = q == 0;                             // this worker holds the first slot of the tile
+            int u = l_first, q = sL % p.nqL;
             for (int j = 0; j < nL; ++j) {
-                const uint32_t src = my_ring + slot * p.slot_bytes;
+                const uint32_t src = my_ring + slot * kSlotBytes;
+                const int mt = min(kAT, p.tilesW - u * kAT);
                 if (!mbar_wait(&my_full[slot], parity)) expired |= 8u;
 #pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
+                for (int jj = 0; jj < 2; ++jj) {
                     uint4 tb[NT];
-                    load_x_step<NT>(tb, ts_addr, q * 4 + jj, p.b, lc);
-                    dense_step<NT>(acc[0], src + (jj >> 1) * 2048, jj & 1, tb, lc);
+                    load_x_step<NT>(tb, ts_addr, q * 2 + jj, p.b, lc);
+                    if (mt == kAT) {
+#pragma unroll
+                        for (int m = 0; m < kAT; ++m) dense_step<NT>(acc[m], src + m * 2048, jj, tb, lc);
+                    } else {
+#pragma unroll
+                        for (int m = 0; m < kAT; ++m)
+                            if (m < mt) dense_step<NT>(acc[m], src + m * 2048, jj, tb, lc);
+                    }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&my_empty[slot]);
                 next_slot();
-                if (++q == p.nqL || j + 1 == nL) {
-                    // The worker that holds a tile's first slot finishes the tile (the workers after it have long
-                    // written their partials: a range is walked front to back, so the tile a range ends in is the
-                    // first thing the next worker does); any other worker leaves its partial.
-                    if (head) finish_tile(tile, acc[0], wl + 1);
-                    else store_tile(Amine + (size_t)(tile - l_first) * frag, acc[0]);
+                if (++q == p.nqL || j + 1 == nL) {            // leaving the rows: their partials go to the workspace
+#pragma unroll
+                    for (int m = 0; m < kAT; ++m)
+                        if (m < mt) store_tile(Amine + ((size_t)(u - l_first) * kAT + m) * frag, acc[m]);
                     zero_acc();
-                    q = 0; ++tile; head = true;
+                    q = 0; ++u;
                 }
             }
         }
         TSTAMP(0, 6);
-
-        // ---------------------------------------------------------------- output tiles without adapters
-        if (p.r == 0) {
-            const Split spF = make_split(p.tilesW, n_ctas * kCW);
-            const int f0 = split_start(spF, wl), f1 = f0 + split_count(spF, wl);
-            for (int tile = f0; tile < f1; ++tile) finish_tile(tile, acc[0], 0);      // acc is zero here
-        }
+        finish_tiles<NT>(p, tabW, tabL, cta * kFinishers + warp, n_ctas * kFinishers, lc, &expired);
         TSTAMP(0, 7);
 #ifdef SLIM_TILED_TRACE
         if (warp == 0 && lane == 0) g_tiled_trace[blockIdx.x * 16 + 13] = clock64() - g_tiled_trace[blockIdx.x * 16 + 13];
 #endif
-    } else if (p.r > 0) {
+    } else {
         // ================================ service warps ================================
         const int sw = warp - kProducerWarp - 1;
+        if (p.r > 0) {
         const uint32_t call = (uint32_t)(ld_gpu64(p.departures) / (unsigned)n_ctas) + 1u;
         const int pairs = p.r / 2;
         bool ok = true;
@@ -609,11 +663,8 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
             const int jt = it / E, e = it % E;
             float sum[1] = {0.f};
             for (int k2 = 0; k2 < p.KS; ++k2) {
-                int c0, c1;
-                slice_blocks(k2, p.KS, p.nblk, &c0, &c1);
-                const int nq2 = (c1 - c0) * 2;
-                PartWalk pw(p.Tpart, make_split(p.tilesR * nq2, p.wnR), nq2, p.muR, jt, (size_t)frag, k2 * p.wnR);
-                while (take_batch<1>(pw, e * 32, lane, sum, &ok)) { }
+                PartWalk pw(p.Tpart, tabR[k2], p.muR, jt / kAT, (size_t)kAT * frag, k2 * p.wnR);
+                while (take_batch<1>(pw, (jt % kAT) * frag + e, lane * E, sum, &ok)) { }
                 if (!ok) expired |= 64u;
             }
             // element (h, q, lane) of the fragment is T[token 8h + 2(lane%4) + (q&1)][16 jt + lane/4 + 8(q>>1)]:
@@ -650,6 +701,7 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
                     if ((uint32_t)(v[k] >> 32) != call) { v[k] = ld_gpu64(p.Tfinal + e0 + k * kSW * 32); all = false; }
                 if (all) break;
                 if (spins > kPollLimit) { expired |= 128u; break; }
+                __nanosleep(kPollPause);
             }
 #pragma unroll
             for (int k = 0; k < kFetch; ++k) {
@@ -665,6 +717,10 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
         __syncwarp();
         if (lane == 0) mbar_arrive(t_bar);
         TSTAMP(kProducerWarp + 1, 9);
+        }
+        TSTAMP(kProducerWarp + 1, 10);
+        finish_tiles<NT>(p, tabW, tabL, cta * kFinishers + kCW + sw, n_ctas * kFinishers, lc, &expired);
+        TSTAMP(kProducerWarp + 1, 15);
     }
 
     if (expired && p.status) atomicOr(p.status, (1u << SLIM_ERR_TIMEOUT) | (expired << 16));
@@ -674,8 +730,8 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
 
 // ------------------------------------------------------------------ host side
 struct Plan {
-    int nt, mt, nb, KS, G, nblk, ring, slot_bytes;
-    int unitsW, tilesW, tilesR, nqL, wnR, muW, muR, muL;
+    int nt, KS, G, nblk, ring;
+    int tilesW, tilesR, unitsW, unitsR, unitsL, nqL, wnR, muW, muR, muL;
     int x_bytes;
     size_t smem, p_bytes, a_bytes, t_bytes;
 };
@@ -698,89 +754,72 @@ bool make_plan(int b, int d_out, int d_in, int r, int ctas, Plan* pl) {
     pl->nblk = d_in / 256;
     pl->tilesW = d_out / 16;
     pl->tilesR = r / 16;
-    pl->nqL = ceil_div(r, kDCols);
+    pl->unitsW = ceil_div(pl->tilesW, kWT);
+    pl->unitsR = ceil_div(pl->tilesR, kAT);
+    pl->unitsL = ceil_div(pl->tilesW, kAT);
+    pl->nqL = ceil_div(r, kACols);
     const int workers = ctas * kCW;
-    // Row tiles per weight slot: wide slots share the activation fragments of a block among more
-    // rows (the activation reads are what loads shared memory), but leave fewer, larger list
-    // units; take the widest one that still gives every warp a few slots.
-    const long long tile_blocks = (long long)pl->tilesW * pl->nblk;
-    pl->mt = 1;
-    if (tile_blocks >= 6LL * workers && pl->tilesW >= 2) pl->mt = 2;
-    if (tile_blocks >= 8LL * workers && pl->tilesW >= 4) pl->mt = 4;
-    pl->nb = 4 / pl->mt;
-    if (tile_blocks < 4LL * workers) pl->nb = pl->nb > 2 ? 2 : pl->nb;      // small problems: finer slots
-    if (tile_blocks < 2LL * workers) pl->nb = 1;
-#ifdef SLIM_DECODE_TUNE
-    // experiments only: the environment overrides the slot shape
-    if (const char* e = getenv("SLIM_MT")) { const int v = atoi(e); if ((v == 1 || v == 2 || v == 4) && pl->tilesW >= v) { pl->mt = v; pl->nb = 4 / v; } }
-    if (const char* e = getenv("SLIM_NB")) { const int v = atoi(e); if (v >= 1 && v * pl->mt <= 4) pl->nb = v; }
-#endif
-    pl->unitsW = ceil_div(pl->tilesW, pl->mt);
     // shared memory: T, the rings, and the activation slice (b tokens x 2 bytes per column).  The rings want
-    // to hold what HBM delivers during one round trip (about 18 KB per warp); the slice wants to be wide,
+    // to hold what HBM delivers during one round trip (18 KB or more per warp); the slice wants to be wide,
     // because every k-slice adds a set of partial sums.  Take the deepest ring (up to kMaxRing slots)
     // that still leaves the whole row to one slice, else three slots, else two.
-    const size_t t_smem = (size_t)pl->nqL * 4 * b * 64;
-    const size_t fixed = 1024 + t_smem + (2 * kCW * kMaxRing + 1) * 8 + 64;
-    int slot = pl->mt * pl->nb * kBlockBytes;
-    if (r > 0 && slot < 4096) slot = 4096;
-    slot = (slot + 1023) / 1024 * 1024;
-    pl->slot_bytes = slot;
+    const size_t t_smem = (size_t)pl->nqL * 2 * b * 64;
+    const size_t fixed = 1024 + t_smem + (2 * kCW * kMaxRing + 1) * 8 + (2 * kMaxKS + 1) * sizeof(ListTab) + 64;
     const size_t row_bytes = (size_t)pl->nblk * 512 * b;
     auto left_with = [&](int ring) -> size_t {
-        const size_t used = fixed + (size_t)kCW * ring * slot;
+        const size_t used = fixed + (size_t)kCW * ring * kSlotBytes;
         return kSmemBudget > used ? kSmemBudget - used : 0;
     };
     pl->ring = 2;
     for (int ring = kMaxRing; ring >= 3; --ring)
         if (left_with(ring) >= row_bytes || (ring == 3 && left_with(3) >= (size_t)b * 512 * 4)) { pl->ring = ring; break; }
 #ifdef SLIM_DECODE_TUNE
+    // experiments only: the environment overrides the ring depth
     if (const char* e = getenv("SLIM_RING")) { const int v = atoi(e); if (v >= 2 && v <= kMaxRing && left_with(v) >= (size_t)b * 512) pl->ring = v; }
 #endif
     const size_t left = left_with(pl->ring);
     const int max_blocks = (int)(left / ((size_t)b * 512));
     if (max_blocks < 1) return false;
     pl->KS = ceil_div(pl->nblk, max_blocks);
-    if (pl->KS > ctas) return false;
+    if (pl->KS > ctas || pl->KS > kMaxKS) return false;
     pl->G = ctas / pl->KS;
-    int widest = 0, nq_min = 1 << 30, nqr_min = 1 << 30, muW = 1, muR = 1;
+    int widest = 0, muW = 1, muR = 1;
     const int slice_workers = pl->G * kCW;
-    // R phase: at least two slots per worker, so that a piece of T has fewer partials to collect
+    // R phase: eight slots or more per worker, so that a piece of T has few partials to collect (the adapter
+    // arithmetic is light: a fraction of the warps keeps up with the stream, the others start on the weight)
     {
         int b0, b1;
         slice_blocks(0, pl->KS, pl->nblk, &b0, &b1);
-        const int S = pl->tilesR * (b1 - b0) * 2;
-        int wn = S / 2;
+        const int S = pl->unitsR * (b1 - b0) * (256 / kACols);
+        int wn = S / 8;
         pl->wnR = wn < 1 ? 1 : (wn > slice_workers ? slice_workers : wn);
     }
     for (int ks = 0; ks < pl->KS; ++ks) {
         int b0, b1;
         slice_blocks(ks, pl->KS, pl->nblk, &b0, &b1);
         if (b1 - b0 > widest) widest = b1 - b0;
-        const int nq = ceil_div(b1 - b0, pl->nb), nqr = (b1 - b0) * 2;
-        if (nq < nq_min) nq_min = nq;
-        if (nqr < nqr_min) nqr_min = nqr;
-        const int mw = slots_per_worker(pl->unitsW * nq, slice_workers, nq), mr = slots_per_worker(pl->tilesR * nqr, pl->wnR, nqr);
+        const int nq = b1 - b0, nqr = (b1 - b0) * (256 / kACols);
+        const int mw = slots_per_worker(pl->unitsW * nq, slice_workers, nq), mr = slots_per_worker(pl->unitsR * nqr, pl->wnR, nqr);
         if (mw > muW) muW = mw;
         if (mr > muR) muR = mr;
     }
     pl->muW = muW; pl->muR = muR;
-    pl->muL = slots_per_worker(pl->tilesW * pl->nqL, workers, pl->nqL);
+    pl->muL = slots_per_worker(pl->unitsL * pl->nqL, workers, pl->nqL);
     pl->x_bytes = widest * 512 * b;
-    pl->smem = fixed + (size_t)kCW * pl->ring * pl->slot_bytes + pl->x_bytes;
+    pl->smem = fixed + (size_t)kCW * pl->ring * kSlotBytes + pl->x_bytes;
     const size_t frag_bytes = (size_t)pl->nt * 128 * sizeof(float);
-    pl->p_bytes = (size_t)pl->KS * slice_workers * pl->muW * pl->mt * frag_bytes;
-    pl->a_bytes = r > 0 ? (size_t)workers * pl->muL * frag_bytes : 0;
-    pl->t_bytes = r > 0 ? (size_t)pl->KS * pl->wnR * pl->muR * frag_bytes : 0;
+    pl->p_bytes = (size_t)pl->KS * slice_workers * pl->muW * kWT * frag_bytes;
+    pl->a_bytes = r > 0 ? (size_t)workers * pl->muL * kAT * frag_bytes : 0;
+    pl->t_bytes = r > 0 ? (size_t)pl->KS * pl->wnR * pl->muR * kAT * frag_bytes : 0;
     return pl->smem <= kSmemBudget;
 }
 
-template <int NT, int MT>
+template <int NT>
 int query_residency() {
     int n = 0;
-    if (cudaFuncSetAttribute(decode_tiled_kernel<NT, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+    if (cudaFuncSetAttribute(decode_tiled_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
         return 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_tiled_kernel<NT, MT>, kThreads, kSmemBudget) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_tiled_kernel<NT>, kThreads, kSmemBudget) != cudaSuccess) return 0;
     return n > 0 ? 1 : 0;
 }
 
@@ -795,13 +834,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// Row-major bf16 matrix [rows][cols], tiles of 16 rows x 64 columns (128 bytes), 128-byte swizzle.
+// Row-major bf16 matrix [rows][cols], boxes of 48 rows x 64 columns (128-byte rows), 128-byte swizzle.
 bool make_tile_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows) {
     EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(tensor_map_encoder());
     if (!fn) return false;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {64, 16};
+    cuuint32_t box[2] = {kACols, 16 * kAT};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -810,10 +849,7 @@ bool make_tile_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t r
 
 }  // namespace
 
-int decode_tiled_query_residency() {
-    return query_residency<1, 1>() && query_residency<1, 2>() && query_residency<1, 4>() && query_residency<2, 1>() &&
-           query_residency<2, 2>() && query_residency<2, 4>();
-}
+int decode_tiled_query_residency() { return query_residency<1>() && query_residency<2>(); }
 
 bool decode_tiled_supports(int b, int d_out, int d_in, int r) {
     Plan pl;
@@ -848,10 +884,10 @@ slim_status_t launch_decode_tiled(const __nv_bfloat16* X, int b, const uint8_t* 
     p.Tpart = reinterpret_cast<uint32_t*>(base + SLIM_WORKSPACE_SYNC_BYTES + kTfinalBytes + pl.p_bytes + pl.a_bytes);
     p.status = status_dev;
     p.s = s; p.b = b; p.r = r; p.d_out = d_out; p.d_in = d_in;
-    p.KS = pl.KS; p.G = pl.G; p.nblk = pl.nblk; p.NB = pl.nb;
-    p.unitsW = pl.unitsW; p.tilesW = pl.tilesW; p.tilesR = pl.tilesR; p.nqL = pl.nqL;
-    p.wnR = pl.wnR; p.muW = pl.muW; p.muR = pl.muR; p.muL = pl.muL;
-    p.ring = pl.ring; p.slot_bytes = pl.slot_bytes; p.x_bytes = pl.x_bytes;
+    p.KS = pl.KS; p.G = pl.G; p.nblk = pl.nblk;
+    p.tilesW = pl.tilesW; p.tilesR = pl.tilesR; p.unitsW = pl.unitsW; p.unitsR = pl.unitsR; p.unitsL = pl.unitsL;
+    p.nqL = pl.nqL; p.wnR = pl.wnR; p.muW = pl.muW; p.muR = pl.muR; p.muL = pl.muL;
+    p.ring = pl.ring; p.x_bytes = pl.x_bytes;
     CUtensorMap tmR, tmL;
     if (r > 0) {
         if (!make_tile_map(&tmR, R, (uint64_t)d_in, (uint64_t)r) || !make_tile_map(&tmL, L, (uint64_t)r, (uint64_t)d_out))
@@ -861,11 +897,7 @@ slim_status_t launch_decode_tiled(const __nv_bfloat16* X, int b, const uint8_t* 
     }
     void* args[] = {&p, &tmR, &tmL};
     const dim3 grid(ctas), block(kThreads);
-    const void* fn = nullptr;
-    if (pl.nt == 1) fn = pl.mt == 1 ? (const void*)decode_tiled_kernel<1, 1> : pl.mt == 2 ? (const void*)decode_tiled_kernel<1, 2>
-                                                                                : (const void*)decode_tiled_kernel<1, 4>;
-    else fn = pl.mt == 1 ? (const void*)decode_tiled_kernel<2, 1> : pl.mt == 2 ? (const void*)decode_tiled_kernel<2, 2>
-                                                                                : (const void*)decode_tiled_kernel<2, 4>;
+    const void* fn = pl.nt == 1 ? (const void*)decode_tiled_kernel<1> : (const void*)decode_tiled_kernel<2>;
     const cudaError_t e = cudaLaunchCooperativeKernel(fn, grid, block, args, pl.smem, st);
     count_launch(1);
     return e == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
@@ -874,9 +906,6 @@ slim_status_t launch_decode_tiled(const __nv_bfloat16* X, int b, const uint8_t* 
 }  // namespace slim
 
 #ifdef SLIM_TILED_TRACE
-extern "C" int slim_debug_read_tiled_dbg(unsigned long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, slim::g_tiled_dbg, sizeof(slim::g_tiled_dbg));
-}
 extern "C" int slim_debug_read_tiled_trace(unsigned long long* out) {
     return (int)cudaMemcpyFromSymbol(out, slim::g_tiled_trace, sizeof(slim::g_tiled_trace));
 }
