@@ -101,10 +101,10 @@ def unpack(vals: np.ndarray, meta: np.ndarray):
 
 
 def repack_tiled(vals: np.ndarray, meta: np.ndarray) -> np.ndarray:
-    """(vals, meta) -> the decode-tiled copy, uint8 [d_out * d_in * 3 / 8]."""
+    """(vals, meta) -> the decode-tiled copy, uint8 [ceil(d_out / 64) * 64 * d_in * 3 / 8]."""
     vals, meta = _c(vals, np.uint8), _c(meta, np.uint8)
     d_out, d_in = vals.shape[0], vals.shape[1] * 4
-    out = np.zeros(d_out * d_in * 3 // 8, np.uint8)
+    out = np.zeros((d_out + 63) // 64 * 64 * d_in * 3 // 8, np.uint8)
     rc = _load().oracle_repack_tiled(_p(vals), _p(meta), d_out, d_in, _p(out))
     if rc != OK:
         raise OracleError(rc)

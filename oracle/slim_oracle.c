@@ -160,11 +160,13 @@ int oracle_unpack(const uint8_t *vals, const uint8_t *meta, int d_out, int d_in,
  *
  * d_out % 16 == 0, d_in % 256 == 0.  The matrix is cut into tiles of 16 rows and
  * blocks of 256 columns; (tile, block) occupies 1536 bytes.  Tiles are taken in groups
- * of four (the last group may have fewer): group g = tile / 4 has T = min(4, d_out/16 - 4 g)
- * tiles and starts at 4 g * (d_in/256) * 1536; inside a group the blocks follow each
- * other, and inside a block the group's tiles: (tile, block) sits at
- *     (4 g * (d_in/256) + block * T + (tile - 4 g)) * 1536,
+ * of four: group g = tile / 4 starts at 4 g * (d_in/256) * 1536; inside a group the
+ * blocks follow each other, and inside a block the group's four tiles: (tile, block) sits at
+ *     (4 g * (d_in/256) + block * 4 + (tile - 4 g)) * 1536,
  * so the 64 rows x 256 columns a group holds of one block are 6144 contiguous bytes.
+ * When d_out/16 is not a multiple of four the last group is completed with padding
+ * pieces: value words 0 and every index nibble 4 (positions 0 and 1), i.e. rows of
+ * stored zeros.
  * Inside a (tile, block) piece, a "step" j = 0..7 is 32
  * columns (8 groups of four), a "lane" is (g, t) = (lane / 4, lane % 4):
  *   value words, bytes [0, 1024):  word (j, lane) at (j / 4) * 512 + lane * 16 + (j % 4) * 4.
@@ -176,7 +178,7 @@ int oracle_unpack(const uint8_t *vals, const uint8_t *meta, int d_out, int d_in,
  *     16 tile + g for 16 of the step's 32 columns (the first 16 when t is even, the
  *     last 16 when t is odd), as a little-endian 16-bit number; bits 16-31 the same
  *     for row 16 tile + g + 8.
- * Words are stored little-endian.  out: d_out * d_in * 3 / 8 bytes.
+ * Words are stored little-endian.  out: ceil(d_out / 64) * 64 * d_in * 3 / 8 bytes.
  */
 int oracle_repack_tiled(const uint8_t *vals, const uint8_t *meta, int d_out, int d_in, uint8_t *out)
 {
@@ -184,11 +186,17 @@ int oracle_repack_tiled(const uint8_t *vals, const uint8_t *meta, int d_out, int
         return ORACLE_BAD_ARG;
     const int nblk = d_in / 256, tiles = d_out / 16;
     const size_t vrow = (size_t)d_in / 4, mrow = (size_t)d_in / 8;
+    const int tiles4 = (tiles + 3) / 4 * 4;
+    for (int tile = tiles; tile < tiles4; ++tile)               /* padding pieces of the last group */
+        for (int blk = 0; blk < nblk; ++blk) {
+            uint8_t *base = out + ((size_t)(4 * (tile / 4)) * nblk + (size_t)blk * 4 + tile % 4) * 1536;
+            memset(base, 0, 1024);
+            memset(base + 1024, 0x44, 512);
+        }
     for (int tile = 0; tile < tiles; ++tile) {
         const int g4 = 4 * (tile / 4);                          /* first tile of the group */
-        const int T = tiles - g4 < 4 ? tiles - g4 : 4;          /* tiles in the group */
         for (int blk = 0; blk < nblk; ++blk) {
-            uint8_t *base = out + ((size_t)g4 * nblk + (size_t)blk * T + (tile - g4)) * 1536;
+            uint8_t *base = out + ((size_t)g4 * nblk + (size_t)blk * 4 + (tile - g4)) * 1536;
             for (int j = 0; j < 8; ++j) {
                 for (int lane = 0; lane < 32; ++lane) {
                     const int g = lane / 4, t = lane % 4;

@@ -233,7 +233,9 @@ def test_repack_tiled_bytes_by_hand():
     vals[9, 5] = 0xA3
     meta[9, 2] = 0xE4
     out = oracle.repack_tiled(vals, meta)
-    assert out.size == 1536
+    assert out.size == 4 * 1536              # one group of four pieces: the tile and three padding pieces
+    assert not out[1536:].reshape(3, 1536)[:, :1024].any() and (out[1536:].reshape(3, 1536)[:, 1024:] == 0x44).all()
+    out = out[:1536]
     expect = np.zeros(1536, np.uint8)
     expect[5 * 16 + 0: 5 * 16 + 4] = [0x00, 0x30, 0x00, 0xA0]           # 0xA0003000 little-endian
     expect[1024 + 5 * 16 + 0: 1024 + 5 * 16 + 4] = [0x00, 0x00, 0xE4, 0x00]
@@ -244,7 +246,7 @@ def test_repack_tiled_bytes_by_hand():
     meta[:] = 0
     vals[3, 8 * 6 + 2] = 0x7C
     meta[3, 4 * 6 + 1] = 0x9D        # columns 8-15 of step 6: first half -> lane t even of steps 4-7: t = 2
-    out = oracle.repack_tiled(vals, meta)
+    out = oracle.repack_tiled(vals, meta)[:1536]
     expect = np.zeros(1536, np.uint8)
     lane = 3 * 4 + 2
     expect[512 + lane * 16 + 2 * 4: 512 + lane * 16 + 2 * 4 + 4] = [0x0C, 0x00, 0x07, 0x00]
@@ -257,12 +259,13 @@ def dense_from_tiled(buf, d_out, d_in):
     value slots, index half-words from the lane that holds them) and rebuild the dense
     code matrix.  Written from the layout's description, not from the oracle's loops."""
     nblk, tiles = d_in // 256, d_out // 16
-    pieces = buf.view("<u4").reshape(tiles * nblk, 384)         # 1536-byte pieces in storage order
-    dense = np.zeros((d_out, d_in), np.int64)
+    tiles4 = (tiles + 3) // 4 * 4
+    pieces = buf.view("<u4").reshape(tiles4 * nblk, 384)        # 1536-byte pieces in storage order
+    dense = np.zeros((16 * tiles4, d_in), np.int64)
     sext = lambda n: n - 16 if n >= 8 else n
-    # storage order: groups of four tiles; in a group block after block; in a block the group's tiles
-    order = [(g4 + t, blk) for g4 in range(0, tiles, 4) for blk in range(nblk) for t in range(min(4, tiles - g4))]
-    assert len(order) == tiles * nblk
+    # storage order: groups of four tiles; in a group block after block; in a block the group's four tiles
+    order = [(g4 + t, blk) for g4 in range(0, tiles4, 4) for blk in range(nblk) for t in range(4)]
+    assert len(order) == tiles4 * nblk
     for piece, (tile, blk) in enumerate(order):
         if True:
             wv = pieces[piece, :256].reshape(2, 32, 4)          # [half of the steps][lane][word]
@@ -293,24 +296,29 @@ def test_repack_tiled_keeps_every_code_and_position():
     mask = inputs.top2_mask(rng.standard_normal((d_out, d_in)).astype(np.float32))
     vals, meta = oracle.pack(codes, mask)
     tiled = oracle.repack_tiled(vals, meta)
-    assert tiled.size == d_out * d_in * 3 // 8
-    assert np.array_equal(dense_from_tiled(tiled, d_out, d_in), codes.astype(np.int64) * mask)
-    # a permutation of the input bits: same population of set bits
-    assert int(np.unpackbits(tiled).sum()) == int(np.unpackbits(vals).sum() + np.unpackbits(meta).sum())
+    assert tiled.size == 128 * d_in * 3 // 8                     # seven tiles are stored as two groups of four
+    dense = dense_from_tiled(tiled, d_out, d_in)
+    assert np.array_equal(dense[:d_out], codes.astype(np.int64) * mask)
+    assert not dense[d_out:].any()                               # the padding tile holds stored zeros
+    # a permutation of the input bits plus the padding tile's index nibbles (one set bit each)
+    pad_bits = 16 * d_in // 4
+    assert int(np.unpackbits(tiled).sum()) == int(np.unpackbits(vals).sum() + np.unpackbits(meta).sum()) + pad_bits
 
 
 def test_repack_tiled_group_order_by_hand():
     """Where whole pieces go: 6 tiles x 2 blocks.  Group 0 (tiles 0-3) holds block 0 of tiles 0..3, then
-    block 1 of tiles 0..3; group 1 (tiles 4, 5; two tiles) holds block 0 of tiles 4, 5, then block 1."""
+    block 1 of tiles 0..3; group 1 (tiles 4, 5 and two padding tiles) holds block 0 of its four tiles, then block 1."""
     d_out, d_in = 96, 512
     vals = np.zeros((d_out, d_in // 4), np.uint8)
     meta = np.zeros((d_out, d_in // 8), np.uint8)
     for tile in range(6):
         for blk in range(2):
             vals[16 * tile, 64 * blk] = 0x10 * tile + blk + 1      # row g = 0, group 0 of the block: lane 0, step 0, slot 0
-    out = oracle.repack_tiled(vals, meta).reshape(12, 1536)
+    out = oracle.repack_tiled(vals, meta).reshape(16, 1536)
     where = {(0, 0): 0, (1, 0): 1, (2, 0): 2, (3, 0): 3, (0, 1): 4, (1, 1): 5, (2, 1): 6, (3, 1): 7,
-             (4, 0): 8, (5, 0): 9, (4, 1): 10, (5, 1): 11}
+             (4, 0): 8, (5, 0): 9, (4, 1): 12, (5, 1): 13}
+    for piece in (10, 11, 14, 15):                               # padding: stored zeros at positions (0, 1)
+        assert not out[piece, :1024].any() and (out[piece, 1024:] == 0x44).all()
     for (tile, blk), piece in where.items():
         B = 0x10 * tile + blk + 1
         w = int(out[piece, :4].view("<u4")[0])
