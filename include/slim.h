@@ -151,12 +151,14 @@ slim_status_t slim_linear_fwd_ex(const void* X, int b, const uint8_t* vals, cons
  * layout (the paper leaves storage to a third-party kernel).  Layout SLIM_LAYOUT_DECODE_TILED,
  * for d_out % 16 == 0 and d_in % 256 == 0:
  *   the matrix is cut into tiles of 16 rows and blocks of 256 columns; (tile, block) occupies
- *   1536 bytes.  Tiles are stored in groups of four (the last group may have fewer): group
- *   g = tile / 4 has T = min(4, d_out / 16 - 4 g) tiles and starts at 4 g * (d_in / 256) * 1536;
- *   inside a group the blocks follow each other and inside a block the group's tiles, so (tile, block)
- *   sits at (4 g * (d_in / 256) + block * T + (tile - 4 g)) * 1536 and the 64 rows x 256 columns a
- *   group holds of one block are 6144 contiguous bytes (one copy request of the streaming kernel: a
- *   request costs the same issue time whatever its size).  Inside a (tile, block) piece a "step"
+ *   1536 bytes.  Tiles are stored in groups of four: group g = tile / 4 starts at
+ *   4 g * (d_in / 256) * 1536; inside a group the blocks follow each other and inside a block the
+ *   group's four tiles, so (tile, block) sits at (4 g * (d_in / 256) + block * 4 + (tile - 4 g)) * 1536
+ *   and the 64 rows x 256 columns a group holds of one block are 6144 contiguous bytes (one copy
+ *   request of the streaming kernel: a request costs the same issue time whatever its size).  When
+ *   d_out / 16 is not a multiple of four, the last group is completed with padding pieces (value words
+ *   0, every index nibble 4: stored zeros), so the buffer holds ceil(d_out / 64) * 64 rows.
+ *   Inside a (tile, block) piece a "step"
  *   j = 0..7 is 32 columns (8 groups of four) and a "lane" is (g, t) = (lane / 4, lane % 4), lane = 0..31.
  *   Value words, bytes [0, 1024): the 32-bit word of (j, lane) sits at
  *   (j / 4) * 512 + lane * 16 + (j % 4) * 4 and holds four value bytes B_i, i = 0..3, of row
@@ -169,7 +171,7 @@ slim_status_t slim_linear_fwd_ex(const void* X, int b, const uint8_t* vals, cons
  */
 #define SLIM_LAYOUT_DECODE_TILED 1
 
-/* Bytes of the tiled copy (d_out * d_in * 3 / 8), or 0 when the layout cannot hold the shape. */
+/* Bytes of the tiled copy (ceil(d_out / 64) * 64 * d_in * 3 / 8), or 0 when the layout cannot hold the shape. */
 size_t slim_tiled_bytes(int d_out, int d_in, int layout_id);
 
 /*

@@ -186,7 +186,7 @@ slim_status_t slim_linear_fwd(const void* X, int b, const uint8_t* vals, const u
 size_t slim_tiled_bytes(int d_out, int d_in, int layout_id)
 {
     if (layout_id != SLIM_LAYOUT_DECODE_TILED || d_out < 16 || d_in < 256 || d_out % 16 != 0 || d_in % 256 != 0) return 0;
-    return (size_t)d_out * (size_t)d_in / 8 * 3;
+    return (size_t)((d_out + 63) / 64 * 64) * (size_t)d_in / 8 * 3;       // whole groups of four 16-row tiles
 }
 
 slim_status_t slim_repack_tiled(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in, int layout_id,

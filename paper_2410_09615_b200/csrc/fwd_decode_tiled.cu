@@ -63,7 +63,8 @@ constexpr int kMaxKS = 64;                              // k-slices the shared-m
 constexpr size_t kSmemBudget = 227 * 1024;
 constexpr uint32_t kPollLimit = 1u << 20;
 constexpr uint32_t kPollPause = 400;                    // ns between two polls of a slot: waiting warps must not flood the L2
-constexpr uint32_t kMbarSpinLimit = 1u << 26;
+constexpr unsigned long long kWaitNs = 250ull * 1000 * 1000;   // longest wait on a shared-memory barrier
+constexpr uint32_t kIdleLimit = 1u << 21;               // rounds of 64 ns in which the producer warp found nothing to request
 constexpr uint32_t kEmpty = 0xFFFFFFFFu;                // "no value yet" in a partial-sum slot
 constexpr uint32_t kNanBits = 0x7FFFFFFFu;              // what a computed all-ones NaN is stored as
 constexpr size_t kTfinalBytes = kDecodeTfinalBytes;
@@ -107,9 +108,17 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Waits for a phase of a shared-memory barrier, for kWaitNs at most (a try may itself suspend the thread for
+// a while, so the bound is on time and not on tries); false when it gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t it = 0; it < kMbarSpinLimit; ++it) {
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -117,8 +126,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done) : "r"(addr), "r"(parity) : "memory");
         if (done) return true;
+        if ((it & 63u) == 63u) {
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitNs) return false;
+        }
     }
-    return false;
 }
 __device__ __forceinline__ void tma_tile(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -445,10 +458,8 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
                     tma_tile(dst, &tmR, blk0 * 256 + r_q * kACols, r_u * (16 * kAT), bar);
                     if (++r_q == nqR) { r_q = 0; ++r_u; }
                 } else if (j < jb.nR + jb.nW) {
-                    const int tg = min(kWT, p.tilesW - w_u * kWT);                  // tiles of this group
-                    mbar_arrive_expect_tx(bar, (uint32_t)(tg * kBlockBytes));
-                    bulk_copy(dst, p.W + ((size_t)w_u * kWT * p.nblk + (size_t)(blk0 + w_q) * tg) * kBlockBytes,
-                              (uint32_t)(tg * kBlockBytes), bar);
+                    mbar_arrive_expect_tx(bar, kSlotBytes);                     // groups are whole: the last one is padded
+                    bulk_copy(dst, p.W + ((size_t)w_u * p.nblk + (size_t)(blk0 + w_q)) * kSlotBytes, kSlotBytes, bar);
                     if (++w_q == nqW) { w_q = 0; ++w_u; }
                 } else {
                     mbar_arrive_expect_tx(bar, kSlotBytes);
@@ -460,7 +471,7 @@ decode_tiled_kernel(const Params p, const __grid_constant__ CUtensorMap tmR, con
             }
             if (__any_sync(0xffffffffu, can)) idle = 0;
             else {
-                if (++idle > kMbarSpinLimit) { expired |= 32u; break; }
+                if (++idle > kIdleLimit) { expired |= 32u; break; }
                 __nanosleep(64);
             }
         }

@@ -10,18 +10,12 @@ __global__ void repack_tiled_kernel(const uint8_t* __restrict__ vals, const uint
     const size_t wi = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (wi >= n_words) return;
     const int k = (int)(wi % 384);                       // word inside the 1536-byte piece
-    // pieces are stored by groups of four tiles: in a group block after block, in a block the group's tiles
-    const size_t piece = wi / 384, full = (size_t)(tiles / 4) * 4 * nblk;
-    int tile, blk;
-    if (piece < full) {
-        const int rem = (int)(piece % (size_t)(4 * nblk));
-        tile = 4 * (int)(piece / (size_t)(4 * nblk)) + (rem & 3);
-        blk = rem >> 2;
-    } else {
-        const int T = tiles % 4, rem = (int)(piece - full);
-        tile = tiles - T + rem % T;
-        blk = rem / T;
-    }
+    // pieces are stored by groups of four tiles: in a group block after block, in a block the group's four
+    // tiles; tiles past d_out / 16 are padding (stored zeros at positions 0 and 1)
+    const size_t piece = wi / 384;
+    const int rem = (int)(piece % (size_t)(4 * nblk));
+    const int tile = 4 * (int)(piece / (size_t)(4 * nblk)) + (rem & 3), blk = rem >> 2;
+    if (tile >= tiles) { out[wi] = k < 256 ? 0u : 0x44444444u; return; }
     const size_t vrow = (size_t)d_in / 4, mrow = (size_t)d_in / 8;
     uint32_t w = 0;
     if (k < 256) {
@@ -48,7 +42,7 @@ __global__ void repack_tiled_kernel(const uint8_t* __restrict__ vals, const uint
 
 slim_status_t launch_repack_tiled(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in, uint8_t* out, cudaStream_t st)
 {
-    const size_t n_words = (size_t)d_out * (size_t)d_in / 8 * 3 / 4;
+    const size_t n_words = (size_t)((d_out + 63) / 64 * 64) * (size_t)d_in / 8 * 3 / 4;
     const unsigned blocks = (unsigned)((n_words + 255) / 256);
     repack_tiled_kernel<<<blocks, 256, 0, st>>>(vals, meta, d_in, d_in / 256, d_out / 16, n_words, reinterpret_cast<uint32_t*>(out));
     count_launch(1);

@@ -65,6 +65,7 @@ def test_host_side_argument_checks_need_no_device(lib):
 
 def test_tiled_entry_points_host_logic(lib):
     assert binding.slim_tiled_bytes(4096, 4096) == 4096 * 4096 * 3 // 8
+    assert binding.slim_tiled_bytes(48, 256) == 64 * 256 * 3 // 8      # whole groups of 64 rows
     assert binding.slim_tiled_bytes(4096, 4096, 2) == 0           # unknown layout
     assert binding.slim_tiled_bytes(4100, 4096) == 0 and binding.slim_tiled_bytes(4096, 4160) == 0
     one = 16

@@ -121,6 +121,36 @@ def test_tiled_zero_scale_and_zero_rank():
     assert parity.compare(inputs.bf16_bits_to_f64(K.bits_from_bf16(Y)), y_ref)["ok"]
 
 
+@pytest.mark.parametrize("d_in,d_out,r,b", [
+    (8192, 8192, 1648, 16),     # two ring slots per warp, four k-slices
+    (8192, 8192, 832, 16),
+    (4096, 11008, 416, 3),
+    (8192, 1024, 112, 16),
+    (2048, 2064, 3072, 16),     # the largest rank
+])
+def test_tiled_calls_repeat_bit_for_bit(d_in, d_out, r, b):
+    """Every partial sum is added in list order, so a call's bits do not depend on which warp was
+    first: forty calls back to back on one workspace (random weight bytes, nothing to compare but
+    the calls with one another) give one result."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(5)
+    tiled = torch.randint(0, 256, (K.slim_tiled_bytes(d_out, d_in),), dtype=torch.uint8, device="cuda", generator=g)
+    tiled.view(-1, 1536)[:, 1024:] = 0x44        # index bytes must name two different positions per group
+    L = torch.randn(d_out, r, device="cuda", generator=g).mul_(0.02).bfloat16()
+    R = torch.randn(r, d_in, device="cuda", generator=g).mul_(0.02).bfloat16()
+    X = torch.randn(b, d_in, device="cuda", generator=g).bfloat16()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = K.new_workspace(b, d_out, d_in, r)
+    first = K.slim_linear_fwd_tiled(X, tiled, d_out, 0.01, L, R, workspace=ws, status=status).clone()
+    assert torch.isfinite(first.float()).all()
+    differ = 0
+    for _ in range(40):
+        Y = K.slim_linear_fwd_tiled(X, tiled, d_out, 0.01, L, R, workspace=ws, status=status)
+        differ += int(not torch.equal(Y.view(torch.int16), first.view(torch.int16)))
+    torch.cuda.synchronize()
+    assert K.read_status(status) == 0 and differ == 0, (differ, K.read_status(status))
+
+
 def test_one_workspace_serves_every_kernel_and_shape_in_turn():
     """Decode calls of different shapes and batch sizes (both tiled and packed-format kernels), a
     prefill call and a CUDA-core call share one workspace; every result is checked against the
