@@ -6,8 +6,10 @@
 Workload: the LLaMA-2-70B decode layer set, the largest configuration that fits one GPU.  One
 step = the seven linears of one transformer block (2 x 8192->8192, 2 x 8192->1024 grouped-query
 k/v, 2 x 8192->28672, 1 x 28672->8192; int4 2:4 weights, per-layer fp32 scale, bf16 adapters of
-rank 0.1 x the smaller dimension) run once at batch 1 and once at batch 16: 14 calls of
-slim_linear_fwd_tiled on the decode-tiled weights (repacked once, outside the timed region).
+rank 0.1 x the smaller dimension) run once at batch 1 and once at batch 16: 14 small-batch calls,
+each on the weight copy slim_decode_layout_hint names for its shape and batch (the packed format
+through slim_linear_fwd, or the decode-tiled copy through slim_linear_fwd_tiled; both made once,
+outside the timed region).
 Every linear has its own copy of weight and adapters; the set is 563 MB, so each call reads its
 operands from HBM (the L2 holds 126 MB).  The step is captured in a CUDA graph and replayed; time
 is taken with CUDA events on the launching stream, max over ranks.  Prints one JSON line, which
@@ -229,6 +231,31 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------ GPU arm
+KERNEL_OF = {"slim_linear_fwd": "decode_kernel", "slim_linear_fwd_tiled": "decode_tiled_kernel"}
+
+
+def weight_copy(ly):
+    """One more copy of a layer's device tensors, in both weight formats."""
+    return {"tiled": ly["tiled"].clone(), "vals": ly["vals"].clone(), "meta": ly["meta"].clone(),
+            "L": ly["Ld"].clone(), "R": ly["Rd"].clone()}
+
+
+def decode_call(K, lib, ly, b, c, ws, ws_bytes, status, tiled=None):
+    """(C function, arguments without the stream, name) of one small-batch call on the copy `c`: the
+    decode-tiled weight through slim_linear_fwd_tiled when slim_decode_layout_hint says so (or `tiled`
+    forces it), else the packed weight through slim_linear_fwd."""
+    import ctypes
+    P = ctypes.c_void_p
+    if tiled is None:
+        tiled = K.slim_decode_layout_hint(b, ly["d_out"], ly["d_in"], ly["r"]) == K.LAYOUT_DECODE_TILED
+    head = (P(ly["Xd"][b].data_ptr()), b)
+    tail = (ctypes.c_float(ly["s"]), P(c["L"].data_ptr()), P(c["R"].data_ptr()), ly["r"], ly["d_out"], ly["d_in"],
+            P(ly["Yd"][b].data_ptr()), P(ws.data_ptr()), ws_bytes, P(status.data_ptr()))
+    if tiled:
+        return lib.slim_linear_fwd_tiled, head + (P(c["tiled"].data_ptr()), K.LAYOUT_DECODE_TILED) + tail, "slim_linear_fwd_tiled"
+    return lib.slim_linear_fwd, head + (P(c["vals"].data_ptr()), P(c["meta"].data_ptr())) + tail, "slim_linear_fwd"
+
+
 def run_ours(args):
     import ctypes
     import torch
@@ -259,31 +286,24 @@ def run_ours(args):
         ly["Ld"], ly["Rd"] = K.bf16_from_bits(ly["L"], dev), K.bf16_from_bits(ly["R"], dev)
         ly["Xd"] = {b: K.bf16_from_bits(ly["X"][b], dev) for b in BATCHES}
         ly["Yd"] = {b: torch.empty((b, ly["d_out"]), dtype=torch.bfloat16, device=dev) for b in BATCHES}
-        ly["copies"] = [(ly["tiled"].clone(), ly["Ld"].clone(), ly["Rd"].clone()) for _ in range(ly["count"])]
+        ly["copies"] = [weight_copy(ly) for _ in range(ly["count"])]
     ws_bytes = max(K.slim_workspace_bytes(b, ly["d_out"], ly["d_in"], ly["r"]) for ly in layers for b in BATCHES)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     K.slim_workspace_reset(ws)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    set_bytes = sum(c[0].numel() + 2 * c[1].numel() + 2 * c[2].numel() for ly in layers for c in ly["copies"])
+    set_bytes = sum(c["tiled"].numel() + 2 * c["L"].numel() + 2 * c["R"].numel() for ly in layers for c in ly["copies"])
     torch.cuda.synchronize()
 
-    fwd = lib.slim_linear_fwd_tiled
-
-    def call_args(ly, b, copy):
-        tiled, L, R = copy
-        return (P(ly["Xd"][b].data_ptr()), b, P(tiled.data_ptr()), K.LAYOUT_DECODE_TILED, ctypes.c_float(ly["s"]),
-                P(L.data_ptr()), P(R.data_ptr()), ly["r"], ly["d_out"], ly["d_in"], P(ly["Yd"][b].data_ptr()),
-                P(ws.data_ptr()), ws_bytes, P(status.data_ptr()))
-
-    # the 14 calls of one step: the block at batch 1, then the block at batch 16
-    step_calls = [(ly, b, call_args(ly, b, copy)) for b in BATCHES for ly in layers for copy in ly["copies"]]
+    # the 14 calls of one step: the block at batch 1, then the block at batch 16; every call goes to the
+    # weight copy and entry point slim_decode_layout_hint names for its shape and batch
+    step_calls = [(ly, b, decode_call(K, lib, ly, b, copy, ws, ws_bytes, status)) for b in BATCHES for ly in layers for copy in ly["copies"]]
     assert len(step_calls) == CALLS_PER_STEP
 
     def issue_step(stream_ptr):
-        for _ly, _b, a in step_calls:
-            rc = fwd(*a, stream_ptr)
+        for _ly, _b, (fn, a, name) in step_calls:
+            rc = fn(*a, stream_ptr)
             if rc != 0:
-                raise RuntimeError(f"slim_linear_fwd_tiled failed: {K.strerror(rc)}")
+                raise RuntimeError(f"{name} failed: {K.strerror(rc)}")
 
     stream = torch.cuda.Stream(device=dev)
     sp = P(stream.cuda_stream)
@@ -291,8 +311,8 @@ def run_ours(args):
         issue_step(sp)                      # first call fills the per-device cache outside any capture
     stream.synchronize()
     launches_per_step = 0
-    for _ly, _b, a in step_calls:
-        fwd(*a, sp)
+    for _ly, _b, (fn, a, _name) in step_calls:
+        fn(*a, sp)
         launches_per_step += lib.slim_last_launch_count()
     stream.synchronize()
 
@@ -348,10 +368,11 @@ def run_ours(args):
 
     # ---- roofline of the dominant kernel over the timed region
     step_bytes = sum(algorithmic_bytes(ly["d_in"], ly["d_out"], ly["r"], b) for ly, b, _ in step_calls)
+    kernels = sorted({KERNEL_OF[name] for _ly, _b, (_fn, _a, name) in step_calls})
     peak, peak_kind = measured_peaks()
     achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
     traffic = None if NCU_TRAFFIC is None else NCU_TRAFFIC["ratio"] * step_bytes / len(step_calls)
-    roofline = {"bound": "hbm", "kernel": "decode_tiled_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": "+".join(kernels), "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "traffic": traffic,
                 "traffic_kind": None if NCU_TRAFFIC is None else
@@ -363,7 +384,10 @@ def run_ours(args):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "batches": list(BATCHES), "calls_per_step": CALLS_PER_STEP,
                        "layers": [[ly["name"], ly["d_in"], ly["d_out"], ly["r"], ly["count"]] for ly in layers],
-                       "weight_format": "decode-tiled (slim_repack_tiled, once, outside the timed region)",
+                       "weight_format": "per call the copy slim_decode_layout_hint names (slim_pack / slim_repack_tiled once, "
+                                        "outside the timed region): " + ", ".join(sorted({
+                                            f"{ly['name']}@b{b}:{'tiled' if name.endswith('tiled') else 'packed'}"
+                                            for ly, b, (_f, _a, name) in step_calls})),
                        "l2": f"inputs larger than L2: every linear has its own copy, {set_bytes / 1e6:.0f} MB per step pass",
                        "launch": launch_mode, "parallelism": f"replicas x{world}"},
             "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
@@ -428,33 +452,38 @@ def time_graph_of_calls(fn, calls, stream, replays=10):
 
 
 def per_case_table(K, lib, layers, model, ws, ws_bytes, status, stream, peak):
-    """Per (layer, batch): us/call of slim_linear_fwd_tiled over rotating copies (> 2x L2 between
-    reuses), algorithmic GB/s and fraction of the HBM roofline."""
-    import ctypes
+    """Per (layer, batch): us/call of both small-batch kernels over rotating copies (> 2x L2 between
+    reuses); `us` is the one slim_decode_layout_hint names, with its algorithmic GB/s and fraction of
+    the HBM roofline."""
     import torch
-    P = ctypes.c_void_p
     rows = []
     for ly in layers:
         per_copy = ly["tiled"].numel() + 2 * ly["Ld"].numel() + 2 * ly["Rd"].numel()
         n_copies = int(np.ceil(2 * L2_BYTES / per_copy)) + 1
-        copies = [(ly["tiled"].clone(), ly["Ld"].clone(), ly["Rd"].clone()) for _ in range(n_copies)]
+        copies = [weight_copy(ly) for _ in range(n_copies)]
         torch.cuda.synchronize()
         for b in BATCHES:
-            calls = [(P(ly["Xd"][b].data_ptr()), b, P(c[0].data_ptr()), K.LAYOUT_DECODE_TILED, ctypes.c_float(ly["s"]),
-                      P(c[1].data_ptr()), P(c[2].data_ptr()), ly["r"], ly["d_out"], ly["d_in"],
-                      P(ly["Yd"][b].data_ptr()), P(ws.data_ptr()), ws_bytes, P(status.data_ptr()))
-                     for c in copies] * 3
-            try:
-                med, best = time_graph_of_calls(lib.slim_linear_fwd_tiled, calls, stream)
-            except Exception as e:
-                rows.append({"model": model, "layer": ly["name"], "b": b, "error": str(e)[:80]})
+            hint_tiled = K.slim_decode_layout_hint(b, ly["d_out"], ly["d_in"], ly["r"]) == K.LAYOUT_DECODE_TILED
+            t = {}
+            for tiled in (False, True):
+                trip = [decode_call(K, lib, ly, b, c, ws, ws_bytes, status, tiled=tiled) for c in copies] * 3
+                try:
+                    t[tiled] = time_graph_of_calls(trip[0][0], [a for _f, a, _n in trip], stream)
+                except Exception as e:
+                    t[tiled] = None
+                    sys.stderr.write(f"[bench] {model} {ly['name']} b={b} tiled={tiled}: {str(e)[:80]}\n")
+            if t[hint_tiled] is None:
+                rows.append({"model": model, "layer": ly["name"], "b": b, "error": "call failed"})
                 continue
+            med, best = t[hint_tiled]
             nbytes = algorithmic_bytes(ly["d_in"], ly["d_out"], ly["r"], b)
             gbs = nbytes / (med * 1e-6) / 1e9
             rows.append({"model": model, "layer": ly["name"], "d_in": ly["d_in"], "d_out": ly["d_out"], "r": ly["r"], "b": b,
+                         "kernel": "decode_tiled_kernel" if hint_tiled else "decode_kernel",
                          "us": round(med, 3), "us_min": round(best, 3), "GBs": round(gbs, 1),
                          "frac_measured": round(gbs / peak, 4), "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
-                         "roofline_us": round(nbytes / peak / 1e3, 3)})
+                         "roofline_us": round(nbytes / peak / 1e3, 3),
+                         "us_other_kernel": None if t[not hint_tiled] is None else round(t[not hint_tiled][0], 3)})
         del copies
     return rows
 
@@ -544,7 +573,7 @@ def time_pack(K, ly, stream):
 
 
 def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, world, barrier):
-    """Same step through slim_linear_fwd_tiled_host: X comes from pinned host memory
+    """Same step through the host-buffer entry points: X comes from pinned host memory
     and Y goes back to pinned host memory inside every call."""
     import ctypes
     import torch
@@ -557,11 +586,12 @@ def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, wor
             yh = torch.empty((b, ly["d_out"]), dtype=torch.bfloat16).pin_memory()
             host[(ly["name"], b)] = (xh, yh)
     calls, h2d, d2h = [], 0, 0
-    for ly, b, a in step_calls:
+    for ly, b, (_fn, a, name) in step_calls:
         xh, yh = host[(ly["name"], b)]
-        # (X_host, b, tiled, layout, s, L, R, r, d_out, d_in, Y_host, x_dev, y_dev, ws, ws_bytes, status)
-        calls.append((P(xh.data_ptr()), b, a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], P(yh.data_ptr()),
-                      P(ly["Xd"][b].data_ptr()), P(ly["Yd"][b].data_ptr()), a[11], a[12], a[13]))
+        # (X_host, b, weight (two arguments), s, L, R, r, d_out, d_in, Y_host, x_dev, y_dev, ws, ws_bytes, status)
+        fn = lib.slim_linear_fwd_tiled_host if name == "slim_linear_fwd_tiled" else lib.slim_linear_fwd_host
+        calls.append((fn, (P(xh.data_ptr()), b, a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], P(yh.data_ptr()),
+                           P(ly["Xd"][b].data_ptr()), P(ly["Yd"][b].data_ptr()), a[11], a[12], a[13])))
         h2d += xh.numel() * 2
         d2h += yh.numel() * 2
     sp = P(stream.cuda_stream)
@@ -569,10 +599,10 @@ def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, wor
 
     def run(n):
         for _ in range(n):
-            for c in calls:
-                rc = lib.slim_linear_fwd_tiled_host(*c, sp)
+            for fn, c in calls:
+                rc = fn(*c, sp)
                 if rc != 0:
-                    raise RuntimeError(f"slim_linear_fwd_tiled_host failed: {K.strerror(rc)}")
+                    raise RuntimeError(f"host-buffer call failed: {K.strerror(rc)}")
 
     run(min(args.warmup, 10))
     barrier()
@@ -584,7 +614,7 @@ def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, wor
     ms = e0.elapsed_time(e1)
     ms = replicas.max_over_ranks(ms, "cuda")
     return {"value": replicas.whole_job_us_per_call(ms / steps, CALLS_PER_STEP, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h, "steps": steps, "api": "slim_linear_fwd_tiled_host"}
+            "d2h_bytes_per_step": d2h, "steps": steps, "api": "slim_linear_fwd_host / slim_linear_fwd_tiled_host"}
 
 
 def time_cpu_baseline(layers, repeats=2):
@@ -626,7 +656,7 @@ def time_cpu_baseline(layers, repeats=2):
 
 def run_single_case(args):
     """Plain stream launches of one (d_in, d_out, r, b) case, L2 flushed between them: the command a
-    profiler captures.  b <= 16: slim_linear_fwd_tiled; above: slim_linear_fwd on the packed weight."""
+    profiler captures.  b <= 16: the copy --layout names; above: slim_linear_fwd on the packed weight."""
     import torch
     from paper_2410_09615_b200 import binding as K, build
     build.build()
@@ -634,7 +664,9 @@ def run_single_case(args):
     s, codes, mask = inputs.make_weights(d_out, d_in, 1)
     L, R = inputs.make_adapters(d_out, d_in, r, 1)
     vals, meta = K.slim_pack(torch.from_numpy(codes).cuda(), torch.from_numpy(mask).cuda())
-    tiled = K.slim_repack_tiled(vals, meta) if b <= 16 else None
+    use_tiled = b <= 16 and (args.layout == "tiled" or (args.layout == "hint" and
+                             K.slim_decode_layout_hint(b, d_out, d_in, r) == K.LAYOUT_DECODE_TILED))
+    tiled = K.slim_repack_tiled(vals, meta) if use_tiled else None
     Ld = K.bf16_from_bits(L) if r else None
     Rd = K.bf16_from_bits(R) if r else None
     X = K.bf16_from_bits(inputs.make_activations(b, d_in, 1))
@@ -664,6 +696,8 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", default=None, help="d_in,d_out,r,b: run plain launches of one case (for profilers)")
     ap.add_argument("--calls", type=int, default=5)
+    ap.add_argument("--layout", choices=["hint", "packed", "tiled"], default="hint",
+                    help="with --case and b <= 16: which weight copy (default: what slim_decode_layout_hint names)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)

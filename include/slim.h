@@ -191,6 +191,18 @@ slim_status_t slim_linear_fwd_tiled(const void* X, int b, const void* tiled, int
                                     const void* R, int r, int d_out, int d_in, void* Y, void* workspace,
                                     size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream);
 
+/*
+ * Which copy of a weight serves small-batch calls of this shape faster on the current device:
+ * 0 = the packed format (slim_linear_fwd), SLIM_LAYOUT_DECODE_TILED = the decode-tiled copy
+ * (slim_linear_fwd_tiled).  The tiled kernel streams large weights at a higher rate but has a
+ * longer fixed start and end, and its two-token-tile form (b > 8) does more tensor work per byte:
+ * the rule is "tiled when b <= 8 and the packed weight has 64 MiB or more", from timings of both
+ * kernels on the LLaMA-2 layer shapes.  Returns 0 as well for shapes the tiled kernel does not take
+ * and for illegal arguments.  (Storage layout is the implementation's choice: Sec. 4 "Speedup"
+ * measures the layer, the paper fixes no format.)
+ */
+int slim_decode_layout_hint(int b, int d_out, int d_in, int r);
+
 /* Host-buffer form of slim_linear_fwd_tiled (see slim_linear_fwd_host). */
 slim_status_t slim_linear_fwd_tiled_host(const void* X_host, int b, const void* tiled, int layout_id, float s,
                                          const void* L, const void* R, int r, int d_out, int d_in, void* Y_host,

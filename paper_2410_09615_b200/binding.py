@@ -41,6 +41,7 @@ SIGNATURES = {
     "slim_linear_fwd_tiled_host": (_I, [_P, _I, _P, _I, _F, _P, _P, _I, _I, _I, _P, _P, _P, _P, _SZ, _P, _P]),
     "slim_noalloc_scratch_needed": (_SZ, [_I, _I, _I, _I]),
     "slim_select_kernel": (_I, [_I, _I, _I, _I]),
+    "slim_decode_layout_hint": (_I, [_I, _I, _I, _I]),
     "slim_last_launch_count": (_I, []),
     "slim_last_token_tile": (_I, []),
     "slim_strerror": (ctypes.c_char_p, [_I]),
@@ -150,6 +151,10 @@ def slim_noalloc_scratch_needed(b: int, d_out: int, d_in: int, r: int) -> int:
 
 def slim_select_kernel(b: int, d_out: int, d_in: int, r: int) -> int:
     return int(lib().slim_select_kernel(b, d_out, d_in, r))
+
+
+def slim_decode_layout_hint(b: int, d_out: int, d_in: int, r: int) -> int:
+    return int(lib().slim_decode_layout_hint(b, d_out, d_in, r))
 
 
 def slim_last_launch_count() -> int:

@@ -127,6 +127,16 @@ slim_status_t slim_workspace_reset(void* workspace, size_t workspace_bytes_, voi
     return cudaMemsetAsync(workspace, 0, SLIM_WORKSPACE_SYNC_BYTES, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
 }
 
+int slim_decode_layout_hint(int b, int d_out, int d_in, int r)
+{
+    if (b < 1 || b > 8 || r < 0 || r % 16 != 0 || check_weight_shape(d_out, d_in) != SLIM_OK) return 0;
+    if ((size_t)d_out * (size_t)d_in * 3 / 8 < ((size_t)64 << 20)) return 0;
+    slim_status_t err;
+    const DeviceInfo* di = device_info(&err);
+    if (!di || !di->decode_tiled_ok || !decode_tiled_supports(b, d_out, d_in, r)) return 0;
+    return SLIM_LAYOUT_DECODE_TILED;
+}
+
 slim_kernel_t slim_select_kernel(int b, int d_out, int d_in, int r)
 {
     if (b < 1 || r < 0 || r % 16 != 0 || check_weight_shape(d_out, d_in) != SLIM_OK) return SLIM_KERNEL_AUTO;
