@@ -54,7 +54,14 @@ L2_BYTES = 126e6
 # DRAM traffic of one launch of the dominant kernel relative to the call's algorithmic bytes, from an
 # ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) whose summary is kept with the other
 # profiler summaries.  None = no capture of the current kernel: the bench then reports traffic null.
-NCU_TRAFFIC = None     # e.g. {"ratio": 1.0, "source": "profiles/<file>", "case": "d_in,d_out,r,b"}
+# DRAM bytes / algorithmic bytes of one launch, from the ncu captures summarised under profiles/ (one
+# case per kernel; traffic grows with the bytes streamed, so other cases are scaled by their bytes).
+# Set an entry to None when its kernel changes after the capture.
+NCU_TRAFFIC = {
+    "decode_kernel": {"ratio": 1.007, "case": "8192,8192,832,16"},
+    "decode_tiled_kernel": {"ratio": 1.035, "case": "8192,28672,832,1"},
+    "source": "profiles/decode_kernels_llama2_70b_decode_layer_set.md",
+}
 
 
 def algorithmic_bytes(d_in, d_out, r, b):
@@ -371,12 +378,16 @@ def run_ours(args):
     kernels = sorted({KERNEL_OF[name] for _ly, _b, (_fn, _a, name) in step_calls})
     peak, peak_kind = measured_peaks()
     achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
-    traffic = None if NCU_TRAFFIC is None else NCU_TRAFFIC["ratio"] * step_bytes / len(step_calls)
+    ratios = {k: NCU_TRAFFIC.get(k) for k in kernels}
+    traffic = None if any(v is None for v in ratios.values()) else sum(
+        ratios[KERNEL_OF[name]]["ratio"] * algorithmic_bytes(ly["d_in"], ly["d_out"], ly["r"], b)
+        for ly, b, (_fn, _a, name) in step_calls) / len(step_calls)
     roofline = {"bound": "hbm", "kernel": "+".join(kernels), "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "traffic": traffic,
-                "traffic_kind": None if NCU_TRAFFIC is None else
-                f"scaled by bytes from {NCU_TRAFFIC['source']}, case {NCU_TRAFFIC['case']}",
+                "traffic_kind": None if traffic is None else
+                "per launch, scaled by algorithmic bytes from the captures in " + NCU_TRAFFIC["source"] + ": " +
+                ", ".join(f"{k} x{v['ratio']} (case {v['case']})" for k, v in ratios.items()),
                 "bytes_per_launch": step_bytes / len(step_calls), "avg_launch_us": 1e3 * ms_per_step / len(step_calls)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -415,6 +426,22 @@ def run_ours(args):
             prefill_rows += prefill_table(K, small, model, stream, 2048)
             del small
         line["per_case"] = tables
+        # the step's two kernels apart: bytes and time of the 70B rows each of them serves, weighted by
+        # the number of such linears in the block
+        count = {ly["name"]: ly["count"] for ly in host70}
+        by = {}
+        for row in tables:
+            if row.get("model") == "70b" and "us" in row:
+                k = by.setdefault(row["kernel"], {"bytes": 0.0, "us": 0.0, "launches": 0})
+                n = count[row["layer"]]
+                k["bytes"] += n * algorithmic_bytes(row["d_in"], row["d_out"], row["r"], row["b"])
+                k["us"] += n * row["us"]
+                k["launches"] += n
+        line["roofline"]["by_kernel"] = {
+            name: {"launches_per_step": k["launches"], "avg_launch_us": round(k["us"] / k["launches"], 3),
+                   "achieved": round(k["bytes"] / k["us"] / 1e3, 1), "frac": round(k["bytes"] / k["us"] / 1e3 / peak, 4),
+                   "share_of_step_time": round(k["us"] / sum(v["us"] for v in by.values()), 4)}
+            for name, k in by.items()}
         line["prefill"] = prefill_rows
         line["roofline_prefill"] = prefill_roofline(prefill_rows)
         line["pack"] = time_pack(K, host70[0], stream)
