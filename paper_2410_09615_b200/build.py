@@ -25,9 +25,11 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False, defines=(), out: str | None = None) -> str:
     """Compile every CUDA source into ``libslim.so`` next to this file.
 
-    ``defines``: extra ``-D`` macros (the kernels' optional hooks: ``SLIM_DECODE_TUNE`` lets the
-    environment override the decode plan, ``SLIM_DECODE_TRACE`` records a per-CTA timeline); such a
-    build goes to ``out`` (required then), never to the library the package loads by default."""
+    ``defines``: extra ``-D`` macros, the kernels' optional hooks: ``SLIM_DECODE_TUNE`` (the environment
+    variable SLIM_RING overrides the tiled decode kernel's ring depth), ``SLIM_DECODE_TRACE``,
+    ``SLIM_TILED_TRACE`` and ``SLIM_PREFILL_TRACE`` (per-CTA timelines of the three kernels, read back
+    with the ``slim_debug_read_*`` functions such a build exports).  A build with hooks goes to ``out``
+    (required then), never to the library the package loads by default."""
     if defines and not out:
         raise ValueError("a build with extra defines needs its own output path")
     if not defines and not force and not _stale():
