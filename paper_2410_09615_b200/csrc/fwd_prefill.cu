@@ -25,6 +25,9 @@
 // selector bit of the instruction descriptor picks the column.  A 32-bit word of the
 // packed index array is one row's 32 columns, so a converter thread swaps one
 // half-word with the thread eight rows away and stores the result.
+// Source of the layout: PTX ISA, "tcgen05.mma.sp" -- "Sparse matrices" / "Sparsity selector" for
+// kind::f16 (which bits of the metadata columns in tensor memory describe which chunk of A, and
+// how the selector picks a column of a pair); the one-hot and exact-integer tests check it.
 //
 // Pipeline.  A ring of stages {B: token rows x 128 bytes, A: 8 KB (16 KB in the dense-only
 // launch)}; a sparse stage is 64 weight columns (two MMAs of K = 32), a dense stage 32 columns
