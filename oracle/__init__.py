@@ -55,6 +55,13 @@ def _load():
         lib.oracle_linear_fwd_dense.argtypes = [P, ctypes.c_int, P, P, ctypes.c_float, P, P,
                                                 ctypes.c_int, ctypes.c_int, ctypes.c_int, P, P]
         lib.oracle_linear_fwd_dense.restype = ctypes.c_int
+        lib.oracle_quant_adapter.argtypes = [P, ctypes.c_int, ctypes.c_int, P, P]
+        lib.oracle_quant_adapter.restype = ctypes.c_int
+        lib.oracle_dequant_adapter.argtypes = [P, P, ctypes.c_int, ctypes.c_int, P]
+        lib.oracle_dequant_adapter.restype = ctypes.c_int
+        lib.oracle_linear_fwd_q.argtypes = [P, ctypes.c_int, P, P, ctypes.c_float, P, P, P, P, ctypes.c_int,
+                                            ctypes.c_int, ctypes.c_int, P, ctypes.c_int, P]
+        lib.oracle_linear_fwd_q.restype = ctypes.c_int
         lib.oracle_flop_reduction.argtypes = [ctypes.c_double] * 5
         lib.oracle_flop_reduction.restype = ctypes.c_double
         lib.oracle_num_threads.argtypes = []
@@ -127,6 +134,48 @@ def linear_fwd(X, vals, meta, s, L, R, rows=None) -> np.ndarray:
     rc = _load().oracle_linear_fwd(_p(X), b, _p(vals), _p(meta), float(s),
                                    _p(L) if r else None, _p(R) if r else None, r, d_out, d_in,
                                    _p(rows_a), nm, _p(Y))
+    if rc != OK:
+        raise OracleError(rc)
+    return Y
+
+
+def quant_adapter(A: np.ndarray):
+    """bf16 bit patterns A[rows][cols] -> (codes uint8 [rows][cols / 2], scales uint16 [rows][ceil(cols / 128)])."""
+    A = _c(A, np.uint16)
+    rows, cols = A.shape
+    codes = np.zeros((rows, cols // 2), np.uint8)
+    scales = np.zeros((rows, (cols + 127) // 128), np.uint16)
+    rc = _load().oracle_quant_adapter(_p(A), rows, cols, _p(codes), _p(scales))
+    if rc != OK:
+        raise OracleError(rc)
+    return codes, scales
+
+
+def dequant_adapter(codes: np.ndarray, scales: np.ndarray) -> np.ndarray:
+    """The fp64 values (code x scale) a quantized adapter stands for."""
+    codes, scales = _c(codes, np.uint8), _c(scales, np.uint16)
+    rows, cols = codes.shape[0], codes.shape[1] * 2
+    assert scales.shape == (rows, (cols + 127) // 128)
+    out = np.empty((rows, cols), np.float64)
+    rc = _load().oracle_dequant_adapter(_p(codes), _p(scales), rows, cols, _p(out))
+    if rc != OK:
+        raise OracleError(rc)
+    return out
+
+
+def linear_fwd_q(X, vals, meta, s, Lq, Ls, Rq, Rs, rows=None) -> np.ndarray:
+    """Factored fp64 forward with quantized adapters (codes and scales of L and of R)."""
+    X, vals, meta = _c(X, np.uint16), _c(vals, np.uint8), _c(meta, np.uint8)
+    Lq, Ls, Rq, Rs = _c(Lq, np.uint8), _c(Ls, np.uint16), _c(Rq, np.uint8), _c(Rs, np.uint16)
+    b, d_in = X.shape
+    d_out, r = vals.shape[0], Lq.shape[1] * 2
+    assert Lq.shape == (d_out, r // 2) and Rq.shape == (r, d_in // 2)
+    assert Ls.shape == (d_out, (r + 127) // 128) and Rs.shape == (r, (d_in + 127) // 128)
+    rows_a = None if rows is None else _c(np.asarray(rows, np.int32), np.int32)
+    nm = b if rows_a is None else len(rows_a)
+    Y = np.empty((nm, d_out), np.float64)
+    rc = _load().oracle_linear_fwd_q(_p(X), b, _p(vals), _p(meta), float(s), _p(Lq), _p(Ls), _p(Rq), _p(Rs), r,
+                                     d_out, d_in, _p(rows_a), nm, _p(Y))
     if rc != OK:
         raise OracleError(rc)
     return Y

@@ -38,6 +38,7 @@
  * that do not come from this file (hand-computed bytes and sums, an
  * independent float64 matrix product, closed forms, invariants).
  */
+#include <math.h>
 #include <stddef.h>
 #include <stdint.h>
 #include <stdlib.h>
@@ -328,6 +329,140 @@ double oracle_flop_reduction(double d, double n, double a, double V, double rr)
     double comp = n * (4.0 * d * d / 2.0 + 4.0 * 2.0 * d * d * rr + 2.0 * d * d * a / 2.0 +
                        2.0 * (d * d * rr + d * d * rr * a)) + d * V;
     return dense / comp;
+}
+
+/* ------------------------------------------------------------------------
+ * Quantized adapters  [Sec. 3.3 "Low-rank Adapter Quantization": 4-bit AbsMax
+ * group quantization, groups of 128 elements share one quantization parameter;
+ * the symmetric uniform grid is that of Sec. 3.1, Eq. 2 and Eq. 5].
+ *
+ * The paper fixes neither the axis of the groups, nor the type of the
+ * parameter, nor which of the 17 levels of Eq. 2 are kept.  Readings taken
+ * here: an adapter is a row-major bf16 matrix A[rows][cols] whose rows run
+ * along the contraction axis of the product it enters (R[r][d_in]: along d_in;
+ * L[d_out][r]: along r); a group is 128 consecutive elements of a row (the last
+ * group of a row may be shorter); the parameter of a group is stored as a bf16
+ * scale = absmax / 7, so that codes are int4 in [-7, 7] (-8 never produced, but
+ * decoded); the value of an element is code * scale.
+ *
+ * Floating point decides the codes, so the decision is taken in one stated
+ * precision on both sides: scale = bf16_rne(fp32(absmax) / 7.0f) and
+ * code = clamp(rint_even(fp32(a) / fp32(scale)), -8, 7), both divisions in IEEE
+ * binary32; a group whose absmax is 0 gets scale 0 and codes 0.
+ *
+ * Storage: codes[rows][cols / 2], two per byte, the even column in the low
+ * nibble, two's complement; scales[rows][ceil(cols / 128)] bf16 bit patterns.
+ * 4 + 16/128 = 4.125 bits per element.
+ * ---------------------------------------------------------------------- */
+static float bf16_to_float(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+/* binary32 -> bfloat16, round to nearest even (finite inputs). */
+static uint16_t float_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+int oracle_quant_adapter(const uint16_t *A, int rows, int cols, uint8_t *codes, uint16_t *scales)
+{
+    if (!A || !codes || !scales || rows < 1 || cols < 2 || cols % 2 != 0) return ORACLE_BAD_ARG;
+    const int groups = (cols + 127) / 128;
+    for (int i = 0; i < rows; ++i) {
+        for (int g = 0; g < groups; ++g) {
+            const int c0 = g * 128, c1 = c0 + 128 < cols ? c0 + 128 : cols;
+            float absmax = 0.0f;
+            for (int c = c0; c < c1; ++c) {
+                float v = bf16_to_float(A[(size_t)i * cols + c]);
+                if (v < 0.0f) v = -v;
+                if (v > absmax) absmax = v;
+            }
+            const uint16_t sb = absmax > 0.0f ? float_to_bf16_rne(absmax / 7.0f) : 0;
+            const float sc = bf16_to_float(sb);
+            scales[(size_t)i * groups + g] = sb;
+            for (int c = c0; c < c1; ++c) {
+                int q = 0;
+                if (sc > 0.0f) {
+                    const float t = bf16_to_float(A[(size_t)i * cols + c]) / sc;
+                    q = (int)nearbyintf(t);               /* default rounding mode: to nearest even */
+                    if (q > 7) q = 7;
+                    if (q < -8) q = -8;
+                }
+                uint8_t *byte = &codes[(size_t)i * (cols / 2) + c / 2];
+                if (c % 2 == 0) *byte = (uint8_t)((*byte & 0xF0u) | ((unsigned)q & 0xFu));
+                else            *byte = (uint8_t)((*byte & 0x0Fu) | (((unsigned)q & 0xFu) << 4));
+            }
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* The values a quantized adapter stands for: out[i][c] = code * scale, exact in fp64. */
+int oracle_dequant_adapter(const uint8_t *codes, const uint16_t *scales, int rows, int cols, double *out)
+{
+    if (!codes || !scales || !out || rows < 1 || cols < 2 || cols % 2 != 0) return ORACLE_BAD_ARG;
+    const int groups = (cols + 127) / 128;
+    for (int i = 0; i < rows; ++i)
+        for (int c = 0; c < cols; ++c) {
+            const uint8_t byte = codes[(size_t)i * (cols / 2) + c / 2];
+            const int q = sext4(c % 2 == 0 ? byte & 0xFu : byte >> 4);
+            out[(size_t)i * cols + c] = (double)q * bf16_to_double(scales[(size_t)i * groups + c / 128]);
+        }
+    return ORACLE_OK;
+}
+
+/*
+ * The layer with quantized adapters: the definition of oracle_linear_fwd with L and R replaced
+ * by the values their codes and scales stand for  [Sec. 3.2: W ~ W^C + L R; Sec. 3.3].
+ * Lq/Ls: codes and scales of L[d_out][r]; Rq/Rs: of R[r][d_in].
+ */
+int oracle_linear_fwd_q(const uint16_t *X, int b, const uint8_t *vals, const uint8_t *meta, float s,
+                        const uint8_t *Lq, const uint16_t *Ls, const uint8_t *Rq, const uint16_t *Rs, int r,
+                        int d_out, int d_in, const int32_t *rows, int n_rows, double *Y)
+{
+    if (!X || !vals || !meta || !Y || b < 1 || d_out < 1 || d_in < 8 || d_in % 8 != 0 || r < 2 || r % 2 != 0)
+        return ORACLE_BAD_ARG;
+    if (!Lq || !Ls || !Rq || !Rs) return ORACLE_BAD_ARG;
+    const int nm = rows ? n_rows : b;
+    int8_t *Wd = (int8_t *)malloc((size_t)d_out * d_in);
+    double *Ld = (double *)malloc(sizeof(double) * (size_t)d_out * r);
+    double *Rd = (double *)malloc(sizeof(double) * (size_t)r * d_in);
+    int rc = (Wd && Ld && Rd) ? ORACLE_OK : ORACLE_BAD_ARG;
+    if (rc == ORACLE_OK) rc = oracle_unpack(vals, meta, d_out, d_in, Wd, NULL);
+    if (rc == ORACLE_OK) rc = oracle_dequant_adapter(Lq, Ls, d_out, r, Ld);
+    if (rc == ORACLE_OK) rc = oracle_dequant_adapter(Rq, Rs, r, d_in, Rd);
+    if (rc != ORACLE_OK) { free(Wd); free(Ld); free(Rd); return rc; }
+    const double sd = (double)s;
+#pragma omp parallel for schedule(static)
+    for (int mi = 0; mi < nm; ++mi) {
+        const int m = rows ? rows[mi] : mi;
+        double *xrow = (double *)malloc(sizeof(double) * (size_t)d_in);
+        double *t = (double *)malloc(sizeof(double) * (size_t)r);
+        for (int k = 0; k < d_in; ++k) xrow[k] = bf16_to_double(X[(size_t)m * d_in + k]);
+        for (int j = 0; j < r; ++j) {
+            double acc = 0.0;
+            for (int k = 0; k < d_in; ++k) acc += xrow[k] * Rd[(size_t)j * d_in + k];
+            t[j] = acc;
+        }
+        for (int n = 0; n < d_out; ++n) {
+            double acc = 0.0;
+            for (int k = 0; k < d_in; ++k) acc += xrow[k] * (sd * (double)Wd[(size_t)n * d_in + k]);
+            double lr = 0.0;
+            for (int j = 0; j < r; ++j) lr += t[j] * Ld[(size_t)n * r + j];
+            Y[(size_t)mi * d_out + n] = acc + lr;
+        }
+        free(xrow);
+        free(t);
+    }
+    free(Wd); free(Ld); free(Rd);
+    return ORACLE_OK;
 }
 
 /* Number of OpenMP threads oracle_linear_fwd will use (1 without OpenMP). */

@@ -331,3 +331,122 @@ def test_repack_tiled_rejects_shapes_it_cannot_tile():
         oracle.repack_tiled(np.zeros((8, 64), np.uint8), np.zeros((8, 32), np.uint8))
     with pytest.raises(oracle.OracleError):
         oracle.repack_tiled(np.zeros((16, 32), np.uint8), np.zeros((16, 16), np.uint8))
+
+
+# ---------------------------------------------------------------- quantized adapters (Sec. 3.3)
+def np_dequant(codes, scales):
+    """Reader-side decode of the adapter storage, written with numpy bit operations only."""
+    lo = (codes & 0xF).astype(np.int16)
+    hi = (codes >> 4).astype(np.int16)
+    q = np.stack([lo, hi], axis=-1).reshape(codes.shape[0], -1)
+    q = np.where(q > 7, q - 16, q).astype(np.float64)
+    sc = inputs.bf16_bits_to_f64(scales)
+    return q * np.repeat(sc, 128, axis=1)[:, :q.shape[1]]
+
+
+def test_quant_adapter_groups_by_hand():
+    cols = 128 + 16                      # a full group and a short one per row
+    A = np.zeros((3, cols), np.float32)
+    # row 0, group 0: absmax 1.75 -> scale 0.25 exactly; 0.3 -> bf16 0.30078 / 0.25 = 1.203 -> 1;
+    #   ties go to even: 0.375 / 0.25 = 1.5 -> 2, 0.625 / 0.25 = 2.5 -> 2, -0.375 -> -2 (= -1.5 to even)
+    A[0, :8] = [0.5, -1.75, 0.25, 0.0, 0.3, 0.375, 0.625, -0.375]
+    # row 0, group 1 (16 elements): its largest magnitude is negative: -3.5 -> scale 0.5, code -7
+    A[0, 128:132] = [-3.5, 1.0, 0.26, -0.74]       # 2, 0.26 -> bf16 0.2598 / 0.5 = 0.52 -> 1, -0.74 -> -1.48 -> -1
+    # row 1: all zeros -> scale 0, codes 0
+    # row 2, group 0: absmax 1 -> 1/7 = 0.142857 -> bf16 0x3E12 = 0.142578125; 1 / 0.142578125 = 7.01 -> 7
+    A[2, :4] = [1.0, -1.0, 0.5, 0.07]               # 0.5 / 0.142578 = 3.507 -> 4 ; 0.07 -> bf16 0.06982 / 0.142578 = 0.49 -> 0
+    codes, scales = oracle.quant_adapter(bf(A))
+    assert codes.shape == (3, cols // 2) and scales.shape == (3, 2)
+    assert scales.tolist() == [[0x3E80, 0x3F00], [0, 0], [0x3E12, 0]]
+    # two codes per byte, the even column in the low nibble, two's complement
+    assert codes[0, :4].tolist() == [0x92, 0x01, 0x21, 0xE2]          # (2,-7) (1,0) (1,2) (2,-2)
+    assert codes[0, 64:66].tolist() == [0x29, 0xF1]                    # (-7,2) (1,-1)
+    assert not codes[0, 4:64].any() and not codes[0, 66:].any() and not codes[1].any()
+    assert codes[2, :2].tolist() == [0x97, 0x04] and not codes[2, 2:].any()   # (7,-7) (4,0)
+    # the values they stand for
+    val = oracle.dequant_adapter(codes, scales)
+    assert val[0, :8].tolist() == [0.5, -1.75, 0.25, 0.0, 0.25, 0.5, 0.5, -0.5]
+    assert val[0, 128:132].tolist() == [-3.5, 1.0, 0.5, -0.5]
+    assert val[2, :4].tolist() == [7 * 0.142578125, -7 * 0.142578125, 4 * 0.142578125, 0.0]
+    assert not val[1].any()
+
+
+def test_dequant_adapter_decodes_minus_eight_and_every_nibble():
+    codes = np.array([[0x10 * h + l for l in range(16)] for h in range(16)], np.uint8).reshape(2, 128)
+    scales = bf(np.array([[0.5, 2.0], [1.0, 0.25]], np.float32))
+    val = oracle.dequant_adapter(codes, scales)
+    assert np.array_equal(val, np_dequant(codes, scales))
+    assert val[0, 16] == -8 * 0.5 and val[0, 17] == 0.0           # byte 0x08: nibble 8 is -8, even column low
+    assert val.min() == -8 * 2.0 and val.max() == 7 * 2.0
+
+
+@pytest.mark.parametrize("rows,cols,seed", [(5, 256, 1), (7, 144, 2), (3, 16, 3), (2, 1000, 4)])
+def test_quant_adapter_round_trip_bound_and_invariants(rows, cols, seed):
+    rng = np.random.default_rng(seed)
+    A = bf(rng.standard_t(3, (rows, cols)).astype(np.float32) * 0.02)        # long-tailed, like adapters
+    a = inputs.bf16_bits_to_f64(A)
+    codes, scales = oracle.quant_adapter(A)
+    val = oracle.dequant_adapter(codes, scales)
+    assert np.array_equal(val, np_dequant(codes, scales))
+    sc = np.repeat(inputs.bf16_bits_to_f64(scales), 128, axis=1)[:, :cols]
+    # AbsMax: the scale is the group's largest magnitude over 7, to bf16 precision
+    for i in range(rows):
+        for g in range((cols + 127) // 128):
+            m = np.abs(a[i, g * 128:(g + 1) * 128]).max()
+            assert abs(sc[i, g * 128] - m / 7) <= m / 7 * 2.0 ** -8
+    # nearest code: the error is at most half a step (a hair more where the rounded scale makes 7.0x -> 7)
+    assert np.all(np.abs(val - a) <= sc * (0.5 + 2.0 ** -6))
+    q = np.rint(val / np.where(sc > 0, sc, 1))
+    assert q.min() >= -7 and q.max() <= 7
+    # the element with the group's largest magnitude gets code +-7
+    for i in range(rows):
+        k = np.abs(a[i, :min(cols, 128)]).argmax()
+        assert abs(q[i, k]) == 7
+
+
+def test_quant_adapter_rejects_bad_shapes():
+    with pytest.raises(oracle.OracleError):
+        oracle.quant_adapter(np.zeros((2, 7), np.uint16))
+
+
+def test_linear_fwd_q_matches_numpy_float64_from_decoded_storage():
+    d_in, d_out, r, b = 272, 24, 48, 5                 # short last groups on both adapters
+    s, codes, mask = inputs.make_weights(d_out, d_in, 71)
+    vals, meta = oracle.pack(codes, mask)
+    L, R = inputs.make_adapters(d_out, d_in, r, 71)
+    X = inputs.make_activations(b, d_in, 71)
+    Lq, Ls = oracle.quant_adapter(L)
+    Rq, Rs = oracle.quant_adapter(R)
+    got = oracle.linear_fwd_q(X, vals, meta, s, Lq, Ls, Rq, Rs)
+    x = inputs.bf16_bits_to_f64(X)
+    W = np.float64(np.float32(s)) * (codes.astype(np.float64) * mask)
+    want = x @ W.T + (x @ np_dequant(Rq, Rs).T) @ np_dequant(Lq, Ls).T
+    assert got.shape == (b, d_out)
+    assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()
+    # it is not the unquantized layer: the adapters' rounding shows
+    plain = oracle.linear_fwd(X, vals, meta, s, L, R)
+    assert np.abs(got - plain).max() > 1e-6
+    # rows subset
+    sub = oracle.linear_fwd_q(X, vals, meta, s, Lq, Ls, Rq, Rs, rows=[4, 0])
+    assert np.array_equal(sub, got[[4, 0]])
+
+
+def test_linear_fwd_q_reduces_to_the_plain_layer_for_adapters_on_the_grid():
+    """Adapters whose entries are already code x power-of-two scale survive quantization unchanged,
+    so the quantized layer equals the pinned bf16-adapter layer."""
+    d_in, d_out, r, b = 256, 16, 32, 3
+    rng = np.random.default_rng(9)
+    s, codes, mask = inputs.make_weights(d_out, d_in, 72)
+    vals, meta = oracle.pack(codes, mask)
+    def on_grid(rows, cols):
+        q = rng.integers(-7, 8, (rows, cols)).astype(np.float32)
+        q[:, ::128] = 7                                  # every group reaches +7, so its scale is what was meant
+        sc = 2.0 ** rng.integers(-9, -3, (rows, (cols + 127) // 128)).astype(np.float32)
+        return bf(q * np.repeat(sc, 128, axis=1)[:, :cols])
+    L, R = on_grid(d_out, r), on_grid(r, d_in)
+    X = inputs.make_activations(b, d_in, 72)
+    Lq, Ls = oracle.quant_adapter(L)
+    Rq, Rs = oracle.quant_adapter(R)
+    assert np.array_equal(oracle.dequant_adapter(Lq, Ls), inputs.bf16_bits_to_f64(L))
+    assert np.array_equal(oracle.dequant_adapter(Rq, Rs), inputs.bf16_bits_to_f64(R))
+    assert np.array_equal(oracle.linear_fwd_q(X, vals, meta, s, Lq, Ls, Rq, Rs), oracle.linear_fwd(X, vals, meta, s, L, R))
