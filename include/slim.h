@@ -225,6 +225,42 @@ slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* val
                                    uint32_t* status_dev, void* cuda_stream);
 
 /*
+ * Quantized adapters (Sec. 3.3 "Low-rank Adapter Quantization": 4-bit AbsMax group quantization,
+ * groups of 128 elements share one quantization parameter; grid of Sec. 3.1 Eq. 2 / Eq. 5).
+ * An adapter is a row-major bf16 matrix A[rows][cols] whose rows run along the contraction axis
+ * of its product (R[r][d_in]; L[d_out][r]); a group is 128 consecutive elements of a row (the last
+ * group of a row may be shorter).  Storage, 4.125 bits per element:
+ *   codes[rows][cols / 2]             two int4 codes per byte, even column in the low nibble;
+ *   scales[rows][ceil(cols / 128)]    bf16, scale = absmax / 7 (binary32 division, nearest-even).
+ * code = clamp(rint(a / scale), -8, 7), division in binary32, ties to even; a group of zeros has
+ * scale 0 and codes 0; the value of an element is code * scale.  cols must be even; all pointers
+ * are DEVICE pointers, 16-byte aligned.  (Magnitudes below the smallest normal binary32 number are
+ * handled as the device's flush-to-zero arithmetic handles them.)
+ */
+size_t slim_adapter_code_bytes(int rows, int cols);     /* 0 for illegal arguments */
+size_t slim_adapter_scale_bytes(int rows, int cols);
+/* Quantize: bit-exact with the definition above. */
+slim_status_t slim_pack_adapter(const void* A, int rows, int cols, uint8_t* codes, void* scales, void* cuda_stream);
+/* The bf16 matrix nearest to the values the codes and scales stand for. */
+slim_status_t slim_unpack_adapter(const uint8_t* codes, const void* scales, int rows, int cols, void* A_out,
+                                  void* cuda_stream);
+
+/*
+ * The layer forward with quantized adapters (SLiM-LoRA^Q; Sec. 3.3, with the layer of Sec. 3.2):
+ * slim_linear_fwd with L and R given as codes and scales (Lq/Ls for L[d_out][r], Rq/Rs for
+ * R[r][d_in]).  r >= 16.  The adapters are expanded to bf16 (each value rounded once, nearest
+ * even) into the tail of the workspace, then the kernel slim_linear_fwd would pick runs on them:
+ * what is saved is the resident size of the adapters, not the bytes a call moves.  The workspace
+ * must have slim_workspace_bytes_q bytes (its first slim_workspace_bytes bytes are the ordinary
+ * workspace, prepared by slim_workspace_reset as usual).
+ */
+size_t slim_workspace_bytes_q(int b, int d_out, int d_in, int r);
+slim_status_t slim_linear_fwd_q(const void* X, int b, const uint8_t* vals, const uint8_t* meta, float s,
+                                const uint8_t* Lq, const void* Ls, const uint8_t* Rq, const void* Rs, int r,
+                                int d_out, int d_in, void* Y, void* workspace, size_t workspace_bytes,
+                                uint32_t* status_dev, void* cuda_stream);
+
+/*
  * Small-batch forward that allocates nothing.  (The paper has no counterpart:
  * this entry point exists for the deployment constraint described here.)
  *

@@ -40,6 +40,12 @@ SIGNATURES = {
     "slim_linear_fwd_tiled": (_I, [_P, _I, _P, _I, _F, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P]),
     "slim_linear_fwd_tiled_host": (_I, [_P, _I, _P, _I, _F, _P, _P, _I, _I, _I, _P, _P, _P, _P, _SZ, _P, _P]),
     "slim_noalloc_scratch_needed": (_SZ, [_I, _I, _I, _I]),
+    "slim_adapter_code_bytes": (_SZ, [_I, _I]),
+    "slim_adapter_scale_bytes": (_SZ, [_I, _I]),
+    "slim_pack_adapter": (_I, [_P, _I, _I, _P, _P, _P]),
+    "slim_unpack_adapter": (_I, [_P, _P, _I, _I, _P, _P]),
+    "slim_workspace_bytes_q": (_SZ, [_I, _I, _I, _I]),
+    "slim_linear_fwd_q": (_I, [_P, _I, _P, _P, _F, _P, _P, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P]),
     "slim_select_kernel": (_I, [_I, _I, _I, _I]),
     "slim_decode_layout_hint": (_I, [_I, _I, _I, _I]),
     "slim_last_launch_count": (_I, []),
@@ -288,4 +294,53 @@ def slim_linear_fwd_noalloc(X, vals, meta, s: float, L, R, Y, status=None):
     _check(lib().slim_linear_fwd_noalloc(_ptr(X), b, _ptr(vals), _ptr(meta), float(s), _ptr(L) if r else None,
                                          _ptr(R) if r else None, r, d_out, d_in, _ptr(Y), _ptr(status), _stream()),
            "slim_linear_fwd_noalloc")
+    return Y
+
+
+def slim_pack_adapter(A: torch.Tensor):
+    """bf16 adapter [rows, cols] -> (codes uint8 [rows, cols / 2], scales bf16 [rows, ceil(cols / 128)])."""
+    _dev(A, torch.bfloat16, "A")
+    rows, cols = A.shape
+    if lib().slim_adapter_code_bytes(rows, cols) == 0:
+        raise SlimError(SLIM_ERR_INVALID_ARG, "slim_pack_adapter", "illegal adapter shape")
+    codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=A.device)
+    scales = torch.empty((rows, (cols + 127) // 128), dtype=torch.bfloat16, device=A.device)
+    _check(lib().slim_pack_adapter(_ptr(A), rows, cols, _ptr(codes), _ptr(scales), _stream()), "slim_pack_adapter")
+    return codes, scales
+
+
+def slim_unpack_adapter(codes: torch.Tensor, scales: torch.Tensor) -> torch.Tensor:
+    """The bf16 matrix nearest to what codes and scales stand for."""
+    _dev(codes, torch.uint8, "codes"), _dev(scales, torch.bfloat16, "scales")
+    rows, cols = codes.shape[0], codes.shape[1] * 2
+    out = torch.empty((rows, cols), dtype=torch.bfloat16, device=codes.device)
+    _check(lib().slim_unpack_adapter(_ptr(codes), _ptr(scales), rows, cols, _ptr(out), _stream()), "slim_unpack_adapter")
+    return out
+
+
+def slim_workspace_bytes_q(b: int, d_out: int, d_in: int, r: int) -> int:
+    return int(lib().slim_workspace_bytes_q(b, d_out, d_in, r))
+
+
+def slim_linear_fwd_q(X, vals, meta, s: float, Lq, Ls, Rq, Rs, Y=None, workspace=None, status=None):
+    """Layer forward with quantized adapters.  Returns Y (bf16 [b, d_out])."""
+    _dev(X, torch.bfloat16, "X"), _dev(vals, torch.uint8, "vals"), _dev(meta, torch.uint8, "meta")
+    for name, t, dt in (("Lq", Lq, torch.uint8), ("Ls", Ls, torch.bfloat16), ("Rq", Rq, torch.uint8), ("Rs", Rs, torch.bfloat16)):
+        _dev(t, dt, name)
+    b, d_in = X.shape
+    d_out, r = vals.shape[0], Lq.shape[1] * 2
+    if tuple(Lq.shape) != (d_out, r // 2) or tuple(Rq.shape) != (r, d_in // 2):
+        raise ValueError("adapter code shapes do not match the weight")
+    if Y is None:
+        Y = torch.empty((b, d_out), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        n = slim_workspace_bytes_q(b, d_out, d_in, r)
+        if n == 0:
+            raise SlimError(SLIM_ERR_UNSUPPORTED_SHAPE, "slim_workspace_bytes_q", "illegal shape")
+        workspace = torch.empty(n, dtype=torch.uint8, device=X.device)
+        with torch.cuda.device(X.device):
+            slim_workspace_reset(workspace)
+    _check(lib().slim_linear_fwd_q(_ptr(X), b, _ptr(vals), _ptr(meta), float(s), _ptr(Lq), _ptr(Ls), _ptr(Rq), _ptr(Rs), r,
+                                   d_out, d_in, _ptr(Y), _ptr(workspace), workspace.numel(), _ptr(status), _stream()),
+           "slim_linear_fwd_q")
     return Y

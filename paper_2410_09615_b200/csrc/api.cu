@@ -193,6 +193,69 @@ slim_status_t slim_linear_fwd(const void* X, int b, const uint8_t* vals, const u
                               status_dev, cuda_stream, SLIM_KERNEL_AUTO);
 }
 
+size_t slim_adapter_code_bytes(int rows, int cols)
+{
+    return rows < 1 || cols < 2 || cols % 2 != 0 ? 0 : (size_t)rows * (size_t)(cols / 2);
+}
+
+size_t slim_adapter_scale_bytes(int rows, int cols)
+{
+    return rows < 1 || cols < 2 || cols % 2 != 0 ? 0 : (size_t)rows * (size_t)((cols + 127) / 128) * 2;
+}
+
+slim_status_t slim_pack_adapter(const void* A, int rows, int cols, uint8_t* codes, void* scales, void* cuda_stream)
+{
+    reset_launch_count();
+    if (!A || !codes || !scales || slim_adapter_code_bytes(rows, cols) == 0) return SLIM_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(codes) || !aligned16(scales)) return SLIM_ERR_INVALID_ARG;
+    return launch_pack_adapter(static_cast<const __nv_bfloat16*>(A), rows, cols, codes, static_cast<__nv_bfloat16*>(scales),
+                               (cudaStream_t)cuda_stream);
+}
+
+slim_status_t slim_unpack_adapter(const uint8_t* codes, const void* scales, int rows, int cols, void* A_out, void* cuda_stream)
+{
+    reset_launch_count();
+    if (!A_out || !codes || !scales || slim_adapter_code_bytes(rows, cols) == 0) return SLIM_ERR_INVALID_ARG;
+    if (!aligned16(A_out) || !aligned16(codes) || !aligned16(scales)) return SLIM_ERR_INVALID_ARG;
+    return launch_unpack_adapter(codes, static_cast<const __nv_bfloat16*>(scales), rows, cols, static_cast<__nv_bfloat16*>(A_out),
+                                 (cudaStream_t)cuda_stream);
+}
+
+static size_t align256(size_t n) { return (n + 255) / 256 * 256; }
+
+size_t slim_workspace_bytes_q(int b, int d_out, int d_in, int r)
+{
+    const size_t base = slim_workspace_bytes(b, d_out, d_in, r);
+    if (base == 0 || r < 16) return 0;
+    return align256(base) + align256((size_t)d_out * r * 2) + align256((size_t)r * d_in * 2);
+}
+
+slim_status_t slim_linear_fwd_q(const void* X, int b, const uint8_t* vals, const uint8_t* meta, float s,
+                                const uint8_t* Lq, const void* Ls, const uint8_t* Rq, const void* Rs, int r,
+                                int d_out, int d_in, void* Y, void* workspace, size_t workspace_bytes_,
+                                uint32_t* status_dev, void* cuda_stream)
+{
+    reset_launch_count();
+    if (!Lq || !Ls || !Rq || !Rs || r < 16 || r % 16 != 0) return SLIM_ERR_INVALID_ARG;
+    if (!aligned16(Lq) || !aligned16(Ls) || !aligned16(Rq) || !aligned16(Rs) || !aligned16(workspace)) return SLIM_ERR_INVALID_ARG;
+    const size_t need = slim_workspace_bytes_q(b, d_out, d_in, r);
+    if (need == 0) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    if (!workspace || workspace_bytes_ < need) return SLIM_ERR_WORKSPACE;
+    const size_t base = align256(slim_workspace_bytes(b, d_out, d_in, r));
+    char* w = static_cast<char*>(workspace);
+    __nv_bfloat16* Ld = reinterpret_cast<__nv_bfloat16*>(w + base);
+    __nv_bfloat16* Rd = reinterpret_cast<__nv_bfloat16*>(w + base + align256((size_t)d_out * r * 2));
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    slim_status_t rc = launch_unpack_adapter(Lq, static_cast<const __nv_bfloat16*>(Ls), d_out, r, Ld, st);
+    if (rc == SLIM_OK) rc = launch_unpack_adapter(Rq, static_cast<const __nv_bfloat16*>(Rs), r, d_in, Rd, st);
+    if (rc != SLIM_OK) return rc;
+    const int dequant_launches = slim_last_launch_count();
+    rc = slim_linear_fwd_ex(X, b, vals, meta, s, Ld, Rd, r, d_out, d_in, Y, workspace, base, status_dev, cuda_stream,
+                            SLIM_KERNEL_AUTO);
+    count_launch(dequant_launches);
+    return rc;
+}
+
 size_t slim_tiled_bytes(int d_out, int d_in, int layout_id)
 {
     if (layout_id != SLIM_LAYOUT_DECODE_TILED || d_out < 16 || d_in < 256 || d_out % 16 != 0 || d_in % 256 != 0) return 0;

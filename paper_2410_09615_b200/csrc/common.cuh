@@ -64,6 +64,10 @@ int decode_tiled_query_residency();
 
 slim_status_t launch_repack_tiled(const uint8_t* vals, const uint8_t* meta, int d_out, int d_in, uint8_t* out, cudaStream_t st);
 
+slim_status_t launch_pack_adapter(const __nv_bfloat16* A, int rows, int cols, uint8_t* codes, __nv_bfloat16* scales, cudaStream_t st);
+slim_status_t launch_unpack_adapter(const uint8_t* codes, const __nv_bfloat16* scales, int rows, int cols, __nv_bfloat16* out,
+                                    cudaStream_t st);
+
 bool prefill_supports(int b, int d_out, int d_in, int r);
 size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r);
 slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
