@@ -70,6 +70,12 @@ def algorithmic_bytes(d_in, d_out, r, b):
     return 0.375 * d_out * d_in + 2.0 * r * (d_in + d_out) + 2.0 * b * (d_in + d_out) + 4.0
 
 
+def algorithmic_bytes_q(d_in, d_out, r, b):
+    """The same with quantized adapters: 4 bits per adapter element plus one bf16 scale per 128."""
+    groups = r * (d_in // 128) + d_out * ((r + 127) // 128)
+    return 0.375 * d_out * d_in + 0.5 * r * (d_in + d_out) + 2.0 * groups + 2.0 * b * (d_in + d_out) + 4.0
+
+
 def executed_flops(d_in, d_out, r, b):
     return 2.0 * b * d_out * d_in / 2.0 + 2.0 * b * r * (d_in + d_out)
 
@@ -445,6 +451,7 @@ def run_ours(args):
         line["prefill"] = prefill_rows
         line["roofline_prefill"] = prefill_roofline(prefill_rows)
         line["pack"] = time_pack(K, host70[0], stream)
+        line["quantized_adapters"] = quantized_adapter_table(K, lib, host70, stream, peak)
     if rank == 0 and world == 1 and not args.skip_cpu:
         line["cpu_baseline"] = time_cpu_baseline(layers)
     if rank == 0:
@@ -511,6 +518,54 @@ def per_case_table(K, lib, layers, model, ws, ws_bytes, status, stream, peak):
                          "frac_measured": round(gbs / peak, 4), "frac_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
                          "roofline_us": round(nbytes / peak / 1e3, 3),
                          "us_other_kernel": None if t[not hint_tiled] is None else round(t[not hint_tiled][0], 3)})
+        del copies
+    return rows
+
+
+def quantized_adapter_table(K, lib, layers, stream, peak):
+    """The 70B layers at batch 1 and 16 through slim_linear_fwd_q (adapters as int4 codes with a bf16
+    scale per 128 elements) beside slim_linear_fwd on the same packed weight with bf16 adapters:
+    bytes per call, us per call over rotating copies, fraction of the HBM roofline on the smaller bytes."""
+    import ctypes
+    import torch
+    P = ctypes.c_void_p
+    rows = []
+    for ly in layers:
+        d_in, d_out, r = ly["d_in"], ly["d_out"], ly["r"]
+        Lq, Ls = K.slim_pack_adapter(ly["Ld"])
+        Rq, Rs = K.slim_pack_adapter(ly["Rd"])
+        per_copy = ly["vals"].numel() + ly["meta"].numel() + 2 * ly["Ld"].numel() + 2 * ly["Rd"].numel()
+        n_copies = int(np.ceil(2 * L2_BYTES / per_copy)) + 1
+        copies = [dict(vals=ly["vals"].clone(), meta=ly["meta"].clone(), L=ly["Ld"].clone(), R=ly["Rd"].clone(),
+                       Lq=Lq.clone(), Ls=Ls.clone(), Rq=Rq.clone(), Rs=Rs.clone()) for _ in range(n_copies)]
+        wsq = torch.empty(max(K.slim_workspace_bytes_q(b, d_out, d_in, r) for b in BATCHES), dtype=torch.uint8, device=Lq.device)
+        K.slim_workspace_reset(wsq)
+        status = torch.zeros(1, dtype=torch.int32, device=Lq.device)
+        torch.cuda.synchronize()
+        for b in BATCHES:
+            head = (P(ly["Xd"][b].data_ptr()), b)
+            tail = (r, d_out, d_in, P(ly["Yd"][b].data_ptr()), P(wsq.data_ptr()), wsq.numel(), P(status.data_ptr()))
+            plain = [head + (P(c["vals"].data_ptr()), P(c["meta"].data_ptr()), ctypes.c_float(ly["s"]), P(c["L"].data_ptr()),
+                             P(c["R"].data_ptr())) + tail for c in copies] * 3
+            quant = [head + (P(c["vals"].data_ptr()), P(c["meta"].data_ptr()), ctypes.c_float(ly["s"]), P(c["Lq"].data_ptr()),
+                             P(c["Ls"].data_ptr()), P(c["Rq"].data_ptr()), P(c["Rs"].data_ptr())) + tail for c in copies] * 3
+            try:
+                t_plain, _ = time_graph_of_calls(lib.slim_linear_fwd, plain, stream)
+                t_q, _ = time_graph_of_calls(lib.slim_linear_fwd_q, quant, stream)
+            except Exception as e:
+                rows.append({"layer": ly["name"], "b": b, "error": str(e)[:80]})
+                continue
+            lib.slim_linear_fwd_q(*quant[0], P(stream.cuda_stream))
+            launches = lib.slim_last_launch_count()
+            nb, nq = algorithmic_bytes(d_in, d_out, r, b), algorithmic_bytes_q(d_in, d_out, r, b)
+            rows.append({"layer": ly["name"], "d_in": d_in, "d_out": d_out, "r": r, "b": b,
+                         "path": "decode kernel on codes and scales" if launches == 1 else "adapters expanded to bf16 first",
+                         "bytes_bf16_adapters": nb, "bytes_quantized": nq, "bytes_ratio": round(nb / nq, 3),
+                         "us_bf16_adapters": round(t_plain, 3), "us_quantized": round(t_q, 3),
+                         "speedup": round(t_plain / t_q, 3), "frac_measured_quantized": round(nq / (t_q * 1e-6) / 1e9 / peak, 4)})
+        torch.cuda.synchronize()
+        if K.read_status(status) != 0:
+            raise RuntimeError(f"device status {K.read_status(status):#x}")
         del copies
     return rows
 

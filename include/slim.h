@@ -248,9 +248,13 @@ slim_status_t slim_unpack_adapter(const uint8_t* codes, const void* scales, int 
 /*
  * The layer forward with quantized adapters (SLiM-LoRA^Q; Sec. 3.3, with the layer of Sec. 3.2):
  * slim_linear_fwd with L and R given as codes and scales (Lq/Ls for L[d_out][r], Rq/Rs for
- * R[r][d_in]).  r >= 16.  The adapters are expanded to bf16 (each value rounded once, nearest
- * even) into the tail of the workspace, then the kernel slim_linear_fwd would pick runs on them:
- * what is saved is the resident size of the adapters, not the bytes a call moves.  The workspace
+ * R[r][d_in]).  r >= 16.  For b <= 16, shapes the decode kernel takes and r % 32 == 0 (the rows of
+ * L's codes must be 16-byte multiples) the decode kernel reads codes and scales as they are: it
+ * multiplies the exact integer codes and scales its accumulator once per group, and a call moves
+ * 4.125 bits per adapter element instead of 16 (Sec. 4 "Speedup": quantized adapters cut the
+ * adapters' share of the layer's time).  Otherwise the adapters are expanded to bf16 (each value
+ * rounded once, nearest even) into the tail of the workspace and the kernel slim_linear_fwd would
+ * pick runs on them: what is saved then is the resident size of the adapters only.  The workspace
  * must have slim_workspace_bytes_q bytes (its first slim_workspace_bytes bytes are the ordinary
  * workspace, prepared by slim_workspace_reset as usual).
  */

@@ -242,10 +242,21 @@ slim_status_t slim_linear_fwd_q(const void* X, int b, const uint8_t* vals, const
     if (need == 0) return SLIM_ERR_UNSUPPORTED_SHAPE;
     if (!workspace || workspace_bytes_ < need) return SLIM_ERR_WORKSPACE;
     const size_t base = align256(slim_workspace_bytes(b, d_out, d_in, r));
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // small batches: the decode kernel reads the codes and scales as they are
+    if (b <= 16 && decode_supports_q(b, d_out, d_in, r)) {
+        if (!X || !vals || !meta || !Y || !std::isfinite(s)) return SLIM_ERR_INVALID_ARG;
+        if (!aligned16(X) || !aligned16(vals) || !aligned16(meta) || !aligned16(Y)) return SLIM_ERR_INVALID_ARG;
+        if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return SLIM_ERR_INVALID_ARG;
+        slim_status_t derr;
+        if (!device_info(&derr)) return derr;
+        return launch_decode_q(static_cast<const __nv_bfloat16*>(X), b, vals, meta, s, Lq, static_cast<const __nv_bfloat16*>(Ls), Rq,
+                               static_cast<const __nv_bfloat16*>(Rs), r, d_out, d_in, static_cast<__nv_bfloat16*>(Y), workspace,
+                               status_dev, st);
+    }
     char* w = static_cast<char*>(workspace);
     __nv_bfloat16* Ld = reinterpret_cast<__nv_bfloat16*>(w + base);
     __nv_bfloat16* Rd = reinterpret_cast<__nv_bfloat16*>(w + base + align256((size_t)d_out * r * 2));
-    cudaStream_t st = (cudaStream_t)cuda_stream;
     slim_status_t rc = launch_unpack_adapter(Lq, static_cast<const __nv_bfloat16*>(Ls), d_out, r, Ld, st);
     if (rc == SLIM_OK) rc = launch_unpack_adapter(Rq, static_cast<const __nv_bfloat16*>(Rs), r, d_in, Rd, st);
     if (rc != SLIM_OK) return rc;

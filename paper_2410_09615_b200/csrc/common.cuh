@@ -53,6 +53,10 @@ slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, 
                             float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
                             int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
                             cudaStream_t st);
+bool decode_supports_q(int b, int d_out, int d_in, int r);
+slim_status_t launch_decode_q(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta, float s,
+                              const uint8_t* Lq, const __nv_bfloat16* Ls, const uint8_t* Rq, const __nv_bfloat16* Rs, int r,
+                              int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev, cudaStream_t st);
 int decode_query_residency(int nt);
 
 bool decode_tiled_supports(int b, int d_out, int d_in, int r);

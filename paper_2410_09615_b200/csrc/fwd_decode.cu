@@ -69,6 +69,7 @@ constexpr uint32_t kNanBits = 0x7FFFFFFFu;                 // what a computed al
 struct DecodeParams {
     const __nv_bfloat16* X; const uint8_t* vals; const uint8_t* meta;
     const __nv_bfloat16* L; const __nv_bfloat16* R; __nv_bfloat16* Y;
+    const __nv_bfloat16* Ls; const __nv_bfloat16* Rs;     // quantized adapters: scales [d_out][ceil(r/128)], [r][d_in/128]
     uint32_t* Ppart;              // [KS][tilesW][frag]      fp32 bits or kEmpty
     uint32_t* Tpart;              // [tilesR][QT][frag]      fp32 bits or kEmpty
     uint2* Tfinal;                // [NT*8][r_pad/2]         {bf16 pair, call number}
@@ -213,6 +214,27 @@ __device__ __forceinline__ uint32_t word_of(const uint4& v, int i) {
     return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
 }
 
+// Quantized adapters.  Two int4 codes at bits 0-3 and 16-19 of `x` (other bits arbitrary) as an exact bf16x2.
+__device__ __forceinline__ uint32_t nib_pair(uint32_t x) {
+    uint32_t y;
+    asm("lop3.b32 %0, %1, %2, %3, 0x6a;" : "=r"(y) : "r"(x), "r"(0x000F000Fu), "r"(0x43084308u));
+    __nv_bfloat162 v = *reinterpret_cast<__nv_bfloat162*>(&y);
+    const uint32_t bias_bits = 0x43084308u;
+    v = __hsub2(v, *reinterpret_cast<const __nv_bfloat162*>(&bias_bits));
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// A word of eight codes c0..c7 (two per byte, even column low) gives, shifted by 4 i, the pair (c_i, c_{i+4}):
+// the dense operand of a quantized adapter pairs columns four apart, and the other operand's eight
+// consecutive bf16 values (c0 c1 | c2 c3 | c4 c5 | c6 c7) are put in the same order.
+__device__ __forceinline__ uint4 pair_four_apart(const uint4& v) {
+    uint4 o;
+    asm("prmt.b32 %0, %1, %2, 0x5410;" : "=r"(o.x) : "r"(v.x), "r"(v.z));
+    asm("prmt.b32 %0, %1, %2, 0x7632;" : "=r"(o.y) : "r"(v.x), "r"(v.z));
+    asm("prmt.b32 %0, %1, %2, 0x5410;" : "=r"(o.z) : "r"(v.y), "r"(v.w));
+    asm("prmt.b32 %0, %1, %2, 0x7632;" : "=r"(o.w) : "r"(v.y), "r"(v.w));
+    return o;
+}
+
 // ------------------------------------------------------------ work split
 // Computed identically by every warp role.
 struct Share {
@@ -335,7 +357,11 @@ __device__ __forceinline__ float take_slots(uint32_t* first, size_t stride, int 
     return slots_finish(sb, first, stride, n, ok);
 }
 
-template <int NT>
+// QA: the adapters are quantized (int4 codes with one bf16 scale per 128 elements of a row, layout in
+// include/slim.h): tmR / tmL then describe the code bytes, a chunk of 512 columns is two tiles of 256
+// codes, a warp's 64 columns lie inside one group, so the warp multiplies exact integer codes and
+// scales its accumulator rows once per chunk.
+template <int NT, bool QA = false>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
 decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
               const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmM,
@@ -391,11 +417,13 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
         for (int u = sh.r_begin; u < sh.r_begin + sh.r_count; ++u) {
             const int tile = u / sh.Qk, q = u % sh.Qk;
             const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
-            const int n_sub = cols / 64;
+            const int n_sub = QA ? cols / 256 : cols / 64;
             const int slot = acquire((uint32_t)n_sub * kSubTile);
-            if (lane < n_sub)
-                tma_tile(ring + (size_t)slot * kSlotBytes + lane * kSubTile, &tmR,
-                         sh.blk_begin * 256 + q * kRChunkCols + 64 * lane, tile * 16, &full_bar[slot]);
+            if (lane < n_sub) {
+                const int x = QA ? (sh.blk_begin * 256 + q * kRChunkCols) / 2 + 128 * lane      // bytes of codes
+                                 : sh.blk_begin * 256 + q * kRChunkCols + 64 * lane;
+                tma_tile(ring + (size_t)slot * kSlotBytes + lane * kSubTile, &tmR, x, tile * 16, &full_bar[slot]);
+            }
         }
         // ---- weight tiles: value bytes (128 per tile row = 2 blocks), then index bytes (4 blocks)
         const int v_sub = (sh.nb + 1) / 2, m_sub = (sh.nb + 3) / 4;
@@ -411,11 +439,11 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
         for (int tile = blockIdx.x; tile < tilesW && p.r > 0; tile += n_ctas) {
             for (int lc = 0; lc < l_chunks; ++lc) {
                 const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
-                const int n_sub = ceil_div(cols, 64);
+                const int n_sub = QA ? ceil_div(cols, 256) : ceil_div(cols, 64);
                 const int slot = acquire((uint32_t)n_sub * kSubTile);
                 if (lane < n_sub)
                     tma_tile(ring + (size_t)slot * kSlotBytes + lane * kSubTile, &tmL,
-                             lc * kLChunkCols + 64 * lane, tile * 16, &full_bar[slot]);
+                             QA ? lc * (kLChunkCols / 2) + 128 * lane : lc * kLChunkCols + 64 * lane, tile * 16, &full_bar[slot]);
             }
         }
         if (lane == 0 && !ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
@@ -503,11 +531,18 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
                     const int tile64 = q * 8 + warp;        // 64-column tile of the slice
                     xd[q][jj][h] = tile64 < sh.nb * 4 ? lds128(xs + tile64 * x_sub + swz(g + 8 * h, jj * 64 + t * 16))
                                                       : make_uint4(0, 0, 0, 0);
+                    if (QA) xd[q][jj][h] = pair_four_apart(xd[q][jj][h]);
                 }
         for (int u = sh.r_begin; u < sh.r_begin + sh.r_count; ++u) {
             const int tile = u / sh.Qk, q = u % sh.Qk;
             const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
             const bool active = warp * 64 < cols;
+            float sc0 = 1.f, sc1 = 1.f;                   // quantized R: scales of rows g and g + 8 in the warp's group
+            if (QA && active) {
+                const size_t grp = (size_t)((sh.blk_begin * 256 + q * kRChunkCols + warp * 64) >> 7), per_row = (size_t)(p.d_in >> 7);
+                sc0 = __bfloat162float(p.Rs[(size_t)(tile * 16 + g) * per_row + grp]);
+                sc1 = __bfloat162float(p.Rs[(size_t)(tile * 16 + g + 8) * per_row + grp]);
+            }
             const unsigned char* base = wait_full();
             if (u == sh.r_begin) STAMP(2);
             float acc[NT][4];
@@ -515,7 +550,29 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
             for (int h = 0; h < NT; ++h)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
-            if (active) {
+            if (QA && active) {
+                // warp w owns 64 columns = 32 bytes of codes in the 256-column tile w / 4
+                const unsigned char* sub = base + (warp >> 2) * kSubTile;
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {
+                    const uint32_t wa = lds32(sub + swz(g, (warp & 3) * 32 + jj * 16 + t * 4));
+                    const uint32_t wb = lds32(sub + swz(g + 8, (warp & 3) * 32 + jj * 16 + t * 4));
+                    uint32_t a[4], c[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { a[i] = nib_pair(wa >> (4 * i)); c[i] = nib_pair(wb >> (4 * i)); }
+#pragma unroll
+                    for (int h = 0; h < NT; ++h) {
+                        uint4 xb = xd[0][jj][h];
+                        if (q == 1) xb = xd[1][jj][h];
+                        if (q == 2) xb = xd[2][jj][h];
+                        if (q == 3) xb = xd[3][jj][h];
+                        mma_16816(acc[h], a[0], c[0], a[1], c[1], xb.x, xb.y);
+                        mma_16816(acc[h], a[2], c[2], a[3], c[3], xb.z, xb.w);
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < NT; ++h) { acc[h][0] *= sc0; acc[h][1] *= sc0; acc[h][2] *= sc1; acc[h][3] *= sc1; }
+            } else if (active) {
                 // warp w owns the 64-column tile w of the chunk
                 const unsigned char* sub = base + warp * kSubTile;
                 uint4 ra[2], rb[2];
@@ -673,6 +730,12 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
         float ysum = 0.f;
         for (int lc = 0; lc < l_chunks; ++lc) {
             const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
+            float sc0 = 1.f, sc1 = 1.f;                   // quantized L: scales of rows g and g + 8 in the warp's group
+            if (QA && warp * 64 < cols) {
+                const size_t grp = (size_t)((lc * kLChunkCols + warp * 64) >> 7), per_row = (size_t)((p.r + 127) >> 7);
+                sc0 = __bfloat162float(p.Ls[(size_t)(tile * 16 + g) * per_row + grp]);
+                sc1 = __bfloat162float(p.Ls[(size_t)(tile * 16 + g + 8) * per_row + grp]);
+            }
             const unsigned char* base = wait_full();
             float acc[NT][4];
 #pragma unroll
@@ -680,7 +743,26 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
             // warp w owns the 64-column tile w of the chunk (two 32-column blocks)
-            if (warp * 64 < cols) {
+            if (QA && warp * 64 < cols) {
+                const unsigned char* sub = base + (warp >> 2) * kSubTile;   // codes past r read as zero
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int kk = warp * 64 + jj * 32 + 8 * t;
+                    const uint32_t wa = lds32(sub + swz(g, (warp & 3) * 32 + jj * 16 + t * 4));
+                    const uint32_t wb = lds32(sub + swz(g + 8, (warp & 3) * 32 + jj * 16 + t * 4));
+                    uint32_t a[4], c[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { a[i] = nib_pair(wa >> (4 * i)); c[i] = nib_pair(wb >> (4 * i)); }
+#pragma unroll
+                    for (int h = 0; h < NT; ++h) {
+                        const uint4 tb = pair_four_apart(lds128(Ts + (size_t)(g + 8 * h) * p.r_pad + lc * kLChunkCols + kk));
+                        mma_16816(acc[h], a[0], c[0], a[1], c[1], tb.x, tb.y);
+                        mma_16816(acc[h], a[2], c[2], a[3], c[3], tb.z, tb.w);
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < NT; ++h) { acc[h][0] *= sc0; acc[h][1] *= sc0; acc[h][2] *= sc1; acc[h][3] *= sc1; }
+            } else if (warp * 64 < cols) {
                 const unsigned char* sub = base + warp * kSubTile;
 #pragma unroll
                 for (int jj = 0; jj < 2; ++jj) {
@@ -768,6 +850,10 @@ int decode_query_residency(int nt) {
         e2 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_kernel<2>, kDecodeThreads, kSmemBudget);
     }
     if (e1 != cudaSuccess || e2 != cudaSuccess) return 0;
+    // the quantized-adapter instances use the same resources
+    if (nt == 1) e1 = cudaFuncSetAttribute(decode_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+    else         e1 = cudaFuncSetAttribute(decode_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+    if (e1 != cudaSuccess) return 0;
     return n > 1 ? 1 : n;      // one CTA per SM: the plan sizes the grid for that
 }
 
@@ -776,6 +862,11 @@ static int decode_ctas(int nt) {
     const DeviceInfo* di = device_info(&err);
     if (!di) return 148;       // sizing queries without a device assume a full B200
     return di->sm_count * (di->decode_ctas_per_sm[nt - 1] > 0 ? 1 : 0);
+}
+
+// Quantized adapters: the rows of L's codes (r / 2 bytes) must be 16-byte multiples for the tensor map.
+bool decode_supports_q(int b, int d_out, int d_in, int r) {
+    return r >= 32 && r % 32 == 0 && decode_supports(b, d_out, d_in, r);
 }
 
 bool decode_supports(int b, int d_out, int d_in, int r) {
@@ -809,11 +900,34 @@ static bool make_tile_map(CUtensorMap* map, const void* base, CUtensorMapDataTyp
            CUDA_SUCCESS;
 }
 
+static slim_status_t launch_decode_any(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
+                                       float s, const void* L, const void* R, const __nv_bfloat16* Ls, const __nv_bfloat16* Rs,
+                                       int r, int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
+                                       cudaStream_t st);
+
 slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
                             float s, const __nv_bfloat16* L, const __nv_bfloat16* R, int r,
                             int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
                             cudaStream_t st)
 {
+    return launch_decode_any(X, b, vals, meta, s, L, R, nullptr, nullptr, r, d_out, d_in, Y, ws, status_dev, st);
+}
+
+slim_status_t launch_decode_q(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta, float s,
+                              const uint8_t* Lq, const __nv_bfloat16* Ls, const uint8_t* Rq, const __nv_bfloat16* Rs, int r,
+                              int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev, cudaStream_t st)
+{
+    if (!decode_supports_q(b, d_out, d_in, r)) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    return launch_decode_any(X, b, vals, meta, s, Lq, Rq, Ls, Rs, r, d_out, d_in, Y, ws, status_dev, st);
+}
+
+// Ls == nullptr: L and R are bf16 matrices; else they are the code bytes of quantized adapters.
+static slim_status_t launch_decode_any(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
+                                       float s, const void* L, const void* R, const __nv_bfloat16* Ls, const __nv_bfloat16* Rs,
+                                       int r, int d_out, int d_in, __nv_bfloat16* Y, void* ws, uint32_t* status_dev,
+                                       cudaStream_t st)
+{
+    const bool qa = Ls != nullptr;
     slim_status_t err;
     const DeviceInfo* di = device_info(&err);
     if (!di) return err;
@@ -822,7 +936,9 @@ slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, 
     const int ctas = decode_ctas(nt);
     if (ctas < 1 || !make_plan(b, d_out, d_in, r, ctas, &pl)) return SLIM_ERR_UNSUPPORTED_SHAPE;
     DecodeParams p;
-    p.X = X; p.vals = vals; p.meta = meta; p.L = L; p.R = R; p.Y = Y;
+    p.X = X; p.vals = vals; p.meta = meta; p.Y = Y;
+    p.L = qa ? nullptr : static_cast<const __nv_bfloat16*>(L); p.R = qa ? nullptr : static_cast<const __nv_bfloat16*>(R);
+    p.Ls = Ls; p.Rs = Rs;
     char* base = reinterpret_cast<char*>(ws);
     p.departures = reinterpret_cast<unsigned long long*>(base);
     p.Tfinal = reinterpret_cast<uint2*>(base + SLIM_WORKSPACE_SYNC_BYTES);
@@ -836,16 +952,19 @@ slim_status_t launch_decode(const __nv_bfloat16* X, int b, const uint8_t* vals, 
     bool ok = make_tile_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, nt * 8) &&
               make_tile_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, 16) &&
               make_tile_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, 16);
-    if (ok && r > 0)
+    if (ok && r > 0 && qa)
+        ok = make_tile_map(&tmR, R, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 2, (uint64_t)r, 16) &&
+             make_tile_map(&tmL, L, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)r / 2, (uint64_t)d_out, 16);
+    else if (ok && r > 0)
         ok = make_tile_map(&tmR, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 16) &&
              make_tile_map(&tmL, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, 16);
     else if (ok) { tmR = tmV; tmL = tmV; }       // never used when r == 0
     if (!ok) return SLIM_ERR_CUDA;
     void* args[] = {&p, &tmX, &tmV, &tmM, &tmR, &tmL};
     const dim3 grid(ctas), block(kDecodeThreads);
-    cudaError_t e = nt == 1
-        ? cudaLaunchCooperativeKernel((const void*)decode_kernel<1>, grid, block, args, pl.smem, st)
-        : cudaLaunchCooperativeKernel((const void*)decode_kernel<2>, grid, block, args, pl.smem, st);
+    const void* fn = nt == 1 ? (qa ? (const void*)decode_kernel<1, true> : (const void*)decode_kernel<1, false>)
+                             : (qa ? (const void*)decode_kernel<2, true> : (const void*)decode_kernel<2, false>);
+    cudaError_t e = cudaLaunchCooperativeKernel(fn, grid, block, args, pl.smem, st);
     count_launch(1);
     return e == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
 }

@@ -79,14 +79,40 @@ def run_q(d_in, d_out, r, b, seed, wseed=None, rows=None):
 
 
 @pytest.mark.parametrize("d_in,d_out,r,b", [
-    (256, 64, 16, 1), (512, 512, 64, 8), (768, 208, 48, 16), (1024, 384, 144, 5),      # decode kernel
-    (320, 48, 32, 3),                                                                   # CUDA-core kernel (d_in % 256 != 0)
-    (512, 256, 64, 200), (640, 384, 144, 70),                                           # prefill kernel
+    # decode kernel reading codes and scales as they are (r % 32 == 0): short last group, two chunk widths,
+    # several k-slices, both token-tile counts
+    (256, 64, 32, 1), (512, 512, 64, 8), (768, 208, 96, 16), (1024, 384, 160, 5), (2304, 128, 416, 16), (4352, 96, 544, 3),
+    (1280, 1040, 1056, 9),
+    # adapters expanded first: decode kernel with r % 32 != 0, CUDA-core kernel, prefill kernel
+    (256, 64, 16, 1), (768, 208, 48, 16), (1024, 384, 144, 5),
+    (320, 48, 32, 3),
+    (512, 256, 64, 200), (640, 384, 144, 70),
 ])
 def test_forward_on_quantized_adapters_small(d_in, d_out, r, b):
     res = run_q(d_in, d_out, r, b, seed=300 + r + b)
     assert res["ok"], res
-    assert res["launches"] >= 3        # two expansions and the forward launches
+    fused = b <= 16 and d_in % 256 == 0 and r % 32 == 0
+    assert res["launches"] == 1 if fused else res["launches"] >= 3      # else two expansions and the forward launches
+
+
+def test_quantized_adapter_codes_reach_the_right_rows_and_columns():
+    """One non-zero code at a time in R and in L (scales a power of two): the output is one product, exactly."""
+    d_in, d_out, r, b = 1024, 64, 160, 4
+    s, codes, mask, ovals, ometa = cached_weights(d_out, d_in, 77)
+    vals, meta = K.slim_pack(to_dev(codes), to_dev(mask))
+    rng = np.random.default_rng(77)
+    X = inputs.f32_to_bf16_bits(rng.integers(-3, 4, (b, d_in)).astype(np.float32))
+    for (j, k, n) in [(0, 0, 0), (159, 1023, 63), (37, 515, 9), (128, 300, 40), (95, 64, 17)]:
+        R = np.zeros((r, d_in), np.float32); L = np.zeros((d_out, r), np.float32)
+        R[j, k] = -1.75                  # code -7 at scale 0.25
+        L[n, j] = 3.5                    # code 7 at scale 0.5
+        Rq, Rs = K.slim_pack_adapter(K.bf16_from_bits(inputs.f32_to_bf16_bits(R)))
+        Lq, Ls = K.slim_pack_adapter(K.bf16_from_bits(inputs.f32_to_bf16_bits(L)))
+        Y = K.slim_linear_fwd_q(K.bf16_from_bits(X), vals, meta, 0.0, Lq, Ls, Rq, Rs)
+        assert K.slim_last_launch_count() == 1
+        y = inputs.bf16_bits_to_f64(K.bits_from_bf16(Y))
+        want = np.zeros((b, d_out)); want[:, n] = inputs.bf16_bits_to_f64(X)[:, k] * -1.75 * 3.5
+        assert np.array_equal(y, want), (j, k, n)
 
 
 def full_q_cases():
