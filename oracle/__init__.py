@@ -62,6 +62,8 @@ def _load():
         lib.oracle_linear_fwd_q.argtypes = [P, ctypes.c_int, P, P, ctypes.c_float, P, P, P, P, ctypes.c_int,
                                             ctypes.c_int, ctypes.c_int, P, ctypes.c_int, P]
         lib.oracle_linear_fwd_q.restype = ctypes.c_int
+        lib.oracle_slim_quant.argtypes = [P, ctypes.c_int, ctypes.c_int, P, P, P, P]
+        lib.oracle_slim_quant.restype = ctypes.c_int
         lib.oracle_flop_reduction.argtypes = [ctypes.c_double] * 5
         lib.oracle_flop_reduction.restype = ctypes.c_double
         lib.oracle_num_threads.argtypes = []
@@ -179,6 +181,21 @@ def linear_fwd_q(X, vals, meta, s, Lq, Ls, Rq, Rs, rows=None) -> np.ndarray:
     if rc != OK:
         raise OracleError(rc)
     return Y
+
+
+def slim_quant(W: np.ndarray):
+    """SLiM-Quant scale search on a float32 matrix: (codes int8 like W, scale float32, alpha float64,
+    table float64 [29][2] of the (alpha, E(alpha)) pairs tried: ten coarse, then nineteen fine)."""
+    W = _c(W, np.float32)
+    d_out, d_in = W.shape
+    codes = np.empty((d_out, d_in), np.int8)
+    scale = np.zeros(1, np.float32)
+    alpha = np.zeros(1, np.float64)
+    table = np.zeros((29, 2), np.float64)
+    rc = _load().oracle_slim_quant(_p(W), d_out, d_in, _p(codes), _p(scale), _p(alpha), _p(table))
+    if rc != OK:
+        raise OracleError(rc)
+    return codes, np.float32(scale[0]), float(alpha[0]), table
 
 
 def linear_fwd_dense(X, vals, meta, s, L, R, return_weight=False):

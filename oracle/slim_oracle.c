@@ -465,6 +465,120 @@ int oracle_linear_fwd_q(const uint16_t *X, int b, const uint8_t *vals, const uin
     return ORACLE_OK;
 }
 
+/* ------------------------------------------------------------------------
+ * SLiM-Quant: the per-tensor scale search  [Sec. 3.1 "SLiM-Quant Quantization
+ * Method", Eq. 2-7 and Algorithm 1; number of histogram bins: App. "Settings
+ * and Hyperparameters"].
+ *
+ * The steps of Algorithm 1, in its order:
+ *   f_abs      histogram of |W| over [0, M], M = max |W|, with
+ *              B = max(512, min(d_in * d_out / 1000, 20000)) uniform bins; a bin
+ *              stands for its centre x_i = (i + 1/2) M / B with weight count_i / N
+ *   E(alpha)   = sum_{x_i <= alpha} p_i (alpha 2^(1-q) round(x_i 2^(q-1) / alpha) - x_i)^2
+ *              + sum_{x_i >  alpha} p_i (alpha - x_i)^2              [Eq. 5, Eq. 6, Eq. 7]
+ *   coarse     alpha = k M / 10, k = 1..10 ("10 uniform samples in (0, max W)"),
+ *              eta_low = M / 10; alpha_low = the first minimiser
+ *   fine       alpha = alpha_low - eta_low + j eta_high, j = 1..19, eta_high = eta_low / 10
+ *              (the open interval (alpha_low - eta_low, alpha_low + eta_low)), capped at M;
+ *              alpha* = the first minimiser over both grids
+ *   quantize   code = clamp(rint(W / alpha* 2^(q-1)), -8, 7), scale s = alpha* 2^(1-q)
+ * Readings where the text is garbled or silent: Eq. 2 / Eq. 5 are read as
+ * code = round(clip(W / alpha, -1, 1) 2^(q-1)), value = code alpha 2^(1-q); the error model keeps
+ * the paper's symmetric clip at alpha although int4 stores +8 as +7; the step sizes eta are not
+ * given: ten coarse samples as the text says, and a fine step of a tenth of the coarse one; ties
+ * go to the smaller alpha; q = 4.
+ *
+ * Floating point decides integers here (the bin of a weight, the argmin, the codes), so the
+ * precision of every such decision is fixed: bin = min(B - 1, (int)((|w| / M) * B)) in binary32
+ * (IEEE division, then multiplication, truncation); E(alpha) in binary64, bins added in
+ * ascending order, no fused multiply-add; codes in binary32: rint((w / alpha32) * 8).
+ * err_table (may be NULL) receives the 29 pairs (alpha, E(alpha)): coarse 1..10, then fine 1..19.
+ * ---------------------------------------------------------------------- */
+static double quant_search_error(const uint32_t *hist, int B, double M, double n_total, double alpha)
+{
+    double e = 0.0;
+    const double width = M / (double)B;
+    for (int i = 0; i < B; ++i) {
+        if (!hist[i]) continue;
+        const double x = ((double)i + 0.5) * width;
+        const double p = (double)hist[i] / n_total;
+        double d;
+        if (x <= alpha) {
+            const double level = rint((x * 8.0) / alpha);
+            d = (alpha * 0.125) * level - x;
+        } else {
+            d = alpha - x;
+        }
+        const double dd = d * d;
+        const double term = p * dd;
+        e = e + term;
+    }
+    return e;
+}
+
+int oracle_slim_quant(const float *W, int d_out, int d_in, int8_t *codes, float *scale, double *alpha_out,
+                      double *err_table)
+{
+    if (!W || !codes || !scale || d_out < 1 || d_in < 1) return ORACLE_BAD_ARG;
+    const size_t n = (size_t)d_out * (size_t)d_in;
+    float M = 0.0f;
+    for (size_t i = 0; i < n; ++i) {
+        const float a = fabsf(W[i]);
+        if (!(a <= 3.0e38f)) return ORACLE_BAD_ARG;          /* NaN or infinity */
+        if (a > M) M = a;
+    }
+    if (M == 0.0f) {                                          /* nothing to quantize */
+        memset(codes, 0, n);
+        *scale = 0.0f;
+        if (alpha_out) *alpha_out = 0.0;
+        if (err_table) memset(err_table, 0, sizeof(double) * 58);
+        return ORACLE_OK;
+    }
+    long long bins = (long long)n / 1000;
+    if (bins > 20000) bins = 20000;
+    if (bins < 512) bins = 512;
+    const int B = (int)bins;
+    uint32_t *hist = (uint32_t *)calloc((size_t)B, sizeof(uint32_t));
+    if (!hist) return ORACLE_BAD_ARG;
+    for (size_t i = 0; i < n; ++i) {
+        const float ratio = fabsf(W[i]) / M;
+        int b = (int)(ratio * (float)B);
+        if (b > B - 1) b = B - 1;
+        hist[b] += 1u;
+    }
+    const double Md = (double)M, eta_low = Md / 10.0, eta_high = eta_low / 10.0;
+    double best_a = 0.0, best_e = 0.0;
+    int have = 0, t = 0;
+    for (int k = 1; k <= 10; ++k) {
+        const double a = (Md * (double)k) / 10.0;
+        const double e = quant_search_error(hist, B, Md, (double)n, a);
+        if (err_table) { err_table[2 * t] = a; err_table[2 * t + 1] = e; }
+        ++t;
+        if (!have || e < best_e) { best_a = a; best_e = e; have = 1; }
+    }
+    const double a_low = best_a;
+    for (int j = 1; j <= 19; ++j) {
+        double a = (a_low - eta_low) + (double)j * eta_high;
+        if (a > Md) a = Md;
+        const double e = a > 0.0 ? quant_search_error(hist, B, Md, (double)n, a) : best_e + 1.0;
+        if (err_table) { err_table[2 * t] = a; err_table[2 * t + 1] = e; }
+        ++t;
+        if (a > 0.0 && (e < best_e || (e == best_e && a < best_a))) { best_a = a; best_e = e; }
+    }
+    free(hist);
+    const float a32 = (float)best_a;
+    for (size_t i = 0; i < n; ++i) {
+        const float v = (W[i] / a32) * 8.0f;
+        int q = (int)nearbyintf(v);
+        if (q > 7) q = 7;
+        if (q < -8) q = -8;
+        codes[i] = (int8_t)q;
+    }
+    *scale = a32 * 0.125f;
+    if (alpha_out) *alpha_out = best_a;
+    return ORACLE_OK;
+}
+
 /* Number of OpenMP threads oracle_linear_fwd will use (1 without OpenMP). */
 #ifdef _OPENMP
 #include <omp.h>

@@ -450,3 +450,80 @@ def test_linear_fwd_q_reduces_to_the_plain_layer_for_adapters_on_the_grid():
     assert np.array_equal(oracle.dequant_adapter(Lq, Ls), inputs.bf16_bits_to_f64(L))
     assert np.array_equal(oracle.dequant_adapter(Rq, Rs), inputs.bf16_bits_to_f64(R))
     assert np.array_equal(oracle.linear_fwd_q(X, vals, meta, s, Lq, Ls, Rq, Rs), oracle.linear_fwd(X, vals, meta, s, L, R))
+
+
+# ---------------------------------------------------------------- SLiM-Quant scale search (Sec. 3.1, Alg. 1)
+def true_mse(W, alpha):
+    """Eq. 3 on the weights themselves: mean |Q^-1(Q(w)) - w|^2 with the symmetric 4-bit grid of Eq. 2 / Eq. 5."""
+    w = W.astype(np.float64)
+    q = np.rint(np.clip(w / alpha, -1.0, 1.0) * 8.0)
+    return float(np.mean((q * alpha / 8.0 - w) ** 2))
+
+
+def bell(kind, shape, seed):
+    rng = np.random.default_rng(seed)
+    if kind == "normal":
+        w = rng.standard_normal(shape)
+    elif kind == "laplace":
+        w = rng.laplace(size=shape)
+    else:
+        w = rng.standard_t(4, shape)
+    return (w * 0.02).astype(np.float32)
+
+
+@pytest.mark.parametrize("kind,shape,seed", [("normal", (300, 400), 0), ("laplace", (64, 1000), 1), ("student", (700, 900), 2),
+                                              ("normal", (16, 32), 3)])
+def test_slim_quant_error_model_and_search(kind, shape, seed):
+    W = bell(kind, shape, seed)
+    M = float(np.abs(W).max())
+    codes, scale, alpha, table = oracle.slim_quant(W)
+    # the grid of Algorithm 1 as read: ten uniform samples of (0, M], then nineteen steps of a tenth around the best
+    assert np.allclose(table[:10, 0], M * np.arange(1, 11) / 10, rtol=1e-15)
+    k_low = int(np.argmin(table[:10, 1]))
+    a_low, eta = table[k_low, 0], M / 10
+    assert np.allclose(table[10:, 0], np.minimum(a_low - eta + np.arange(1, 20) * eta / 10, M), rtol=1e-12, atol=1e-18)
+    # the histogram integral follows the error of the definition, candidate by candidate
+    n_bins = max(512, min(W.size // 1000, 20000))
+    for a, e in table:
+        assert abs(e - true_mse(W, a)) <= 0.02 * true_mse(W, a) + (M / n_bins) ** 2, (a, e, true_mse(W, a))
+    # alpha* is the first minimiser of the table, and (to the accuracy of the integral) of the true error
+    i_best = int(np.argmin(table[:, 1]))
+    assert alpha == table[i_best, 0] and 0 < alpha <= M
+    best_true = min(true_mse(W, a) for a in table[:, 0])
+    assert true_mse(W, alpha) <= 1.02 * best_true
+    # clipping pays on bell-shaped weights: better than AbsMax (alpha = M), which is candidate 10
+    if W.size > 1000:
+        assert alpha < M and true_mse(W, alpha) < 0.8 * true_mse(W, M)
+    # codes and scale of the quantization step at alpha*
+    assert scale == np.float32(np.float32(alpha) * np.float32(0.125))
+    want = np.clip(np.rint(W.astype(np.float64) / np.float64(np.float32(alpha)) * 8.0), -8, 7)
+    assert np.mean(codes != want) < 1e-4 and np.abs(codes - want).max() <= 1          # binary32 decisions at ties only
+    assert codes.min() >= -8 and codes.max() <= 7
+
+
+def test_slim_quant_single_magnitude_by_hand():
+    # every |w| = c: all weights sit in the last bin (centre c (1 - 1/1024)); among alpha = k c / 10 only
+    # alpha = c avoids clipping it (error (c/1024)^2, level 8); the fine steps below c clip it again, so
+    # alpha* = c, the scale is c / 8 and the codes are +8 -> 7 (int4) and -8
+    c = np.float32(0.75)
+    W = np.full((6, 10), c, np.float32)
+    W[::2] *= -1
+    codes, scale, alpha, table = oracle.slim_quant(W)
+    assert alpha == 0.75 and scale == np.float32(0.09375)
+    assert np.array_equal(codes, np.where(W > 0, 7, -8))
+    assert table[9, 0] == 0.75 and abs(table[9, 1] - (0.75 / 1024) ** 2) < 1e-15
+    assert abs(table[8, 1] - (0.75 * (0.9 - (1 - 1 / 1024))) ** 2) < 1e-12     # alpha = 0.9 c clips the bin centre
+
+
+def test_slim_quant_scales_with_powers_of_two_and_handles_degenerate_input():
+    W = bell("normal", (128, 256), 5)
+    codes, scale, alpha, table = oracle.slim_quant(W)
+    codes4, scale4, alpha4, table4 = oracle.slim_quant(W * np.float32(4))
+    assert np.array_equal(codes, codes4) and scale4 == scale * 4 and alpha4 == alpha * 4
+    assert np.array_equal(table4[:, 0], table[:, 0] * 4) and np.allclose(table4[:, 1], table[:, 1] * 16, rtol=1e-12)
+    z = oracle.slim_quant(np.zeros((4, 8), np.float32))
+    assert not z[0].any() and z[1] == 0 and z[2] == 0
+    bad = np.zeros((4, 8), np.float32)
+    bad[1, 2] = np.nan
+    with pytest.raises(oracle.OracleError):
+        oracle.slim_quant(bad)
