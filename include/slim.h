@@ -225,6 +225,30 @@ slim_status_t slim_linear_fwd_host(const void* X_host, int b, const uint8_t* val
                                    uint32_t* status_dev, void* cuda_stream);
 
 /*
+ * SLiM-Quant: the scale of a weight matrix and its 4-bit codes (Sec. 3.1 "SLiM-Quant Quantization
+ * Method", Eq. 2-7, Algorithm 1; bins: App. "Settings and Hyperparameters").  The step before
+ * slim_pack: W[d_out][d_in] float32 in, dense int8 codes in [-8, 7] and the scale s out.
+ *   histogram of |W| over [0, M], M = max |W|, B = max(512, min(d_in d_out / 1000, 20000)) uniform bins,
+ *     a bin standing for its centre x_i with weight count_i / N;
+ *   E(alpha) = sum_{x_i <= alpha} p_i (alpha / 8 * round(8 x_i / alpha) - x_i)^2 + sum_{x_i > alpha} p_i (alpha - x_i)^2;
+ *   candidates alpha = k M / 10, k = 1..10, then alpha_low - M/10 + j M/100, j = 1..19, capped at M, around
+ *     the best coarse one; alpha* = the first minimiser (ties: the smaller alpha);
+ *   code = clamp(rint(8 W / alpha*), -8, 7), s = alpha* / 8.
+ * Decisions are taken in fixed precision so that the result is reproducible bit for bit: the bin of a
+ * weight is min(B - 1, (int)((|w| / M) * B)) in binary32; E in binary64, bins added in ascending order,
+ * every operation rounded on its own; codes rint((w / alpha32) * 8) in binary32.
+ * scale_alpha (DEVICE, 2 floats): [0] = s, [1] = alpha*.  The workspace (slim_quant_workspace_bytes,
+ * DEVICE, 16-byte aligned) also receives, after the histogram, the table of the 29 (alpha, E) pairs
+ * tried (float64 pairs, coarse then fine; a fine candidate that is not positive is listed with the
+ * best error so far plus one) followed by alpha* as float64: at byte offset 256 + round_up(4 B, 256).
+ * A NaN or infinity in W sets the SLIM_ERR_INVALID_ARG bit of *status_dev and gives scale 0; an
+ * all-zero W gives scale 0 and codes 0.  Four launches on the stream; nothing is synchronised.
+ */
+size_t slim_quant_workspace_bytes(int d_out, int d_in);
+slim_status_t slim_quant(const float* W, int d_out, int d_in, int8_t* codes, float* scale_alpha, void* workspace,
+                         size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream);
+
+/*
  * Quantized adapters (Sec. 3.3 "Low-rank Adapter Quantization": 4-bit AbsMax group quantization,
  * groups of 128 elements share one quantization parameter; grid of Sec. 3.1 Eq. 2 / Eq. 5).
  * An adapter is a row-major bf16 matrix A[rows][cols] whose rows run along the contraction axis

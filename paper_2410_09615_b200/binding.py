@@ -40,6 +40,8 @@ SIGNATURES = {
     "slim_linear_fwd_tiled": (_I, [_P, _I, _P, _I, _F, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P]),
     "slim_linear_fwd_tiled_host": (_I, [_P, _I, _P, _I, _F, _P, _P, _I, _I, _I, _P, _P, _P, _P, _SZ, _P, _P]),
     "slim_noalloc_scratch_needed": (_SZ, [_I, _I, _I, _I]),
+    "slim_quant_workspace_bytes": (_SZ, [_I, _I]),
+    "slim_quant": (_I, [_P, _I, _I, _P, _P, _P, _SZ, _P, _P]),
     "slim_adapter_code_bytes": (_SZ, [_I, _I]),
     "slim_adapter_scale_bytes": (_SZ, [_I, _I]),
     "slim_pack_adapter": (_I, [_P, _I, _I, _P, _P, _P]),
@@ -344,3 +346,19 @@ def slim_linear_fwd_q(X, vals, meta, s: float, Lq, Ls, Rq, Rs, Y=None, workspace
                                    d_out, d_in, _ptr(Y), _ptr(workspace), workspace.numel(), _ptr(status), _stream()),
            "slim_linear_fwd_q")
     return Y
+
+
+def slim_quant(W: torch.Tensor, status=None):
+    """SLiM-Quant on a float32 matrix: (codes int8 like W, scale_alpha float32[2] on the device = (s, alpha*),
+    table float64 [29, 2] of the candidates tried, alpha* as float64)."""
+    _dev(W, torch.float32, "W")
+    d_out, d_in = W.shape
+    n = int(lib().slim_quant_workspace_bytes(d_out, d_in))
+    ws = torch.empty(n, dtype=torch.uint8, device=W.device)
+    codes = torch.empty((d_out, d_in), dtype=torch.int8, device=W.device)
+    sa = torch.empty(4, dtype=torch.float32, device=W.device)
+    _check(lib().slim_quant(_ptr(W), d_out, d_in, _ptr(codes), _ptr(sa), _ptr(ws), n, _ptr(status), _stream()), "slim_quant")
+    bins = max(512, min(d_out * d_in // 1000, 20000))
+    off = 256 + (bins * 4 + 255) // 256 * 256
+    tab = ws[off:off + 59 * 8].view(torch.float64)
+    return codes, sa[:2], tab[:58].view(29, 2), tab[58]

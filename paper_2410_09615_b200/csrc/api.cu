@@ -193,6 +193,22 @@ slim_status_t slim_linear_fwd(const void* X, int b, const uint8_t* vals, const u
                               status_dev, cuda_stream, SLIM_KERNEL_AUTO);
 }
 
+size_t slim_quant_workspace_bytes(int d_out, int d_in)
+{
+    return d_out < 1 || d_in < 1 ? 0 : quant_workspace_bytes(d_out, d_in);
+}
+
+slim_status_t slim_quant(const float* W, int d_out, int d_in, int8_t* codes, float* scale_alpha, void* workspace,
+                         size_t workspace_bytes_, uint32_t* status_dev, void* cuda_stream)
+{
+    reset_launch_count();
+    if (!W || !codes || !scale_alpha || d_out < 1 || d_in < 1) return SLIM_ERR_INVALID_ARG;
+    if (!aligned16(W) || !aligned16(codes) || !aligned16(scale_alpha) || !aligned16(workspace)) return SLIM_ERR_INVALID_ARG;
+    if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return SLIM_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes_ < quant_workspace_bytes(d_out, d_in)) return SLIM_ERR_WORKSPACE;
+    return launch_quant(W, d_out, d_in, codes, scale_alpha, workspace, status_dev, (cudaStream_t)cuda_stream);
+}
+
 size_t slim_adapter_code_bytes(int rows, int cols)
 {
     return rows < 1 || cols < 2 || cols % 2 != 0 ? 0 : (size_t)rows * (size_t)(cols / 2);

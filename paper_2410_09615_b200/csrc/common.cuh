@@ -72,6 +72,10 @@ slim_status_t launch_pack_adapter(const __nv_bfloat16* A, int rows, int cols, ui
 slim_status_t launch_unpack_adapter(const uint8_t* codes, const __nv_bfloat16* scales, int rows, int cols, __nv_bfloat16* out,
                                     cudaStream_t st);
 
+size_t quant_workspace_bytes(int d_out, int d_in);
+slim_status_t launch_quant(const float* W, int d_out, int d_in, int8_t* codes, float* scale_alpha, void* ws,
+                           uint32_t* status_dev, cudaStream_t st);
+
 bool prefill_supports(int b, int d_out, int d_in, int r);
 size_t prefill_workspace_bytes(int b, int d_out, int d_in, int r);
 slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals, const uint8_t* meta,
