@@ -64,6 +64,8 @@ def _load():
         lib.oracle_linear_fwd_q.restype = ctypes.c_int
         lib.oracle_slim_quant.argtypes = [P, ctypes.c_int, ctypes.c_int, P, P, P, P]
         lib.oracle_slim_quant.restype = ctypes.c_int
+        lib.oracle_mask_top2.argtypes = [P, P, ctypes.c_int, ctypes.c_int, P]
+        lib.oracle_mask_top2.restype = ctypes.c_int
         lib.oracle_flop_reduction.argtypes = [ctypes.c_double] * 5
         lib.oracle_flop_reduction.restype = ctypes.c_double
         lib.oracle_num_threads.argtypes = []
@@ -196,6 +198,19 @@ def slim_quant(W: np.ndarray):
     if rc != OK:
         raise OracleError(rc)
     return codes, np.float32(scale[0]), float(alpha[0]), table
+
+
+def mask_top2(codes: np.ndarray, xbar=None) -> np.ndarray:
+    """2:4 mask of int8 codes: per group of four along d_in the two largest |code| * xbar[k] (xbar None: |code|)."""
+    codes = _c(codes, np.int8)
+    d_out, d_in = codes.shape
+    xb = None if xbar is None else _c(xbar, np.float32)
+    assert xb is None or xb.shape == (d_in,)
+    mask = np.empty((d_out, d_in), np.uint8)
+    rc = _load().oracle_mask_top2(_p(codes), _p(xb), d_out, d_in, _p(mask))
+    if rc != OK:
+        raise OracleError(rc)
+    return mask
 
 
 def linear_fwd_dense(X, vals, meta, s, L, R, return_weight=False):

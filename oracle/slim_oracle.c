@@ -579,6 +579,38 @@ int oracle_slim_quant(const float *W, int d_out, int d_in, int8_t *codes, float 
     return ORACLE_OK;
 }
 
+/* ------------------------------------------------------------------------
+ * The 2:4 mask of the pipeline's second step  [Sec. 3 and Fig. 1: the quantized weights are
+ * sparsified by a one-shot pruning method; Sec. 3.2: "the product of the magnitude of the weights
+ * and activations is a useful metric for identifying important weights"].
+ * In every aligned group of four along d_in the two entries with the largest metric
+ *     m[n][k] = |Q[n][k]| * xbar[k]        (xbar == NULL: m = |Q|, magnitude pruning)
+ * are kept; equal metrics go to the lower index.  The metric is one binary32 multiplication.
+ * xbar is the average input magnitude per input channel (non-negative, finite).
+ * ---------------------------------------------------------------------- */
+int oracle_mask_top2(const int8_t *codes, const float *xbar, int d_out, int d_in, uint8_t *mask)
+{
+    if (!codes || !mask || d_out < 1 || d_in < 4 || d_in % 4 != 0) return ORACLE_BAD_ARG;
+    for (int n = 0; n < d_out; ++n)
+        for (int g = 0; g < d_in / 4; ++g) {
+            float m[4];
+            for (int i = 0; i < 4; ++i) {
+                const int k = 4 * g + i;
+                const int c = codes[(size_t)n * d_in + k];
+                const float a = (float)(c < 0 ? -c : c);
+                if (xbar && !(xbar[k] >= 0.0f && xbar[k] <= 3.0e38f)) return ORACLE_BAD_ARG;
+                m[i] = xbar ? a * xbar[k] : a;
+            }
+            for (int i = 0; i < 4; ++i) {
+                int beaten = 0;                       /* entries that come before i in the order */
+                for (int j = 0; j < 4; ++j)
+                    if (j != i && (m[j] > m[i] || (m[j] == m[i] && j < i))) ++beaten;
+                mask[(size_t)n * d_in + 4 * g + i] = (uint8_t)(beaten < 2);
+            }
+        }
+    return ORACLE_OK;
+}
+
 /* Number of OpenMP threads oracle_linear_fwd will use (1 without OpenMP). */
 #ifdef _OPENMP
 #include <omp.h>

@@ -527,3 +527,30 @@ def test_slim_quant_scales_with_powers_of_two_and_handles_degenerate_input():
     bad[1, 2] = np.nan
     with pytest.raises(oracle.OracleError):
         oracle.slim_quant(bad)
+
+
+# ---------------------------------------------------------------- 2:4 mask producer (pipeline step 2)
+def test_mask_top2_by_hand():
+    codes = np.array([[3, -3, 3, 1,   0, 0, 0, 0,   -8, 7, -7, 8 - 16,   1, 2, 3, 4]], np.int8)
+    # group 0: |3| three times: the two lowest indices win the tie; group 1: all zero -> positions 0, 1;
+    # group 2: magnitudes 8, 7, 7, 8 -> positions 0 and 3; group 3: 3 and 4
+    assert oracle.mask_top2(codes).tolist() == [[1, 1, 0, 0,  1, 1, 0, 0,  1, 0, 0, 1,  0, 0, 1, 1]]
+    # input magnitudes re-rank the entries: |q| * xbar = (3, 0.75, 6, 2 | ... | 8, 14, 3.5, 8 | 0.5, 2, 0, 8)
+    xbar = np.array([1, 0.25, 2, 2,  5, 0, 1, 1,  1, 2, 0.5, 1,  0.5, 1, 0, 2], np.float32)
+    # group 1: metrics all zero whatever xbar says: positions 0, 1 again
+    assert oracle.mask_top2(codes, xbar).tolist() == [[1, 0, 1, 0,  1, 1, 0, 0,  1, 1, 0, 0,  0, 1, 0, 1]]
+
+
+@pytest.mark.parametrize("d_out,d_in,seed", [(7, 64, 1), (33, 1000, 2)])
+def test_mask_top2_agrees_with_the_generators_mask_and_keeps_two_per_group(d_out, d_in, seed):
+    rng = np.random.default_rng(seed)
+    codes = rng.integers(-8, 8, (d_out, d_in)).astype(np.int8)
+    m = oracle.mask_top2(codes)
+    assert np.array_equal(m, inputs.top2_mask(codes.astype(np.float32)))      # numpy's own statement of the rule
+    xbar = rng.random(d_in).astype(np.float32)
+    mx = oracle.mask_top2(codes, xbar)
+    assert np.array_equal(mx, inputs.top2_mask(np.abs(codes).astype(np.float32) * xbar[None, :]))
+    for mask in (m, mx):
+        assert np.all(mask.reshape(d_out, d_in // 4, 4).sum(-1) == 2)
+    with pytest.raises(oracle.OracleError):
+        oracle.mask_top2(codes, np.full(d_in, np.nan, np.float32))
