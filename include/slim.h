@@ -249,6 +249,19 @@ slim_status_t slim_quant(const float* W, int d_out, int d_in, int8_t* codes, flo
                          size_t workspace_bytes, uint32_t* status_dev, void* cuda_stream);
 
 /*
+ * The 2:4 mask of the pipeline's second step (Sec. 3 and Fig. 1: the quantized weights are sparsified by a
+ * one-shot pruning method; metric of Sec. 3.2: the product of the magnitudes of weight and input).
+ * In every aligned group of four along d_in the two entries with the largest |codes[n][k]| * xbar[k]
+ * are kept (mask 1), equal metrics go to the lower index; xbar NULL: magnitude pruning.  The metric is
+ * one binary32 multiplication, so the mask is reproducible bit for bit.  codes [d_out][d_in] int8,
+ * xbar [d_in] float32 (average input magnitude per channel: non-negative and finite, else the
+ * SLIM_ERR_INVALID_ARG bit of *status_dev is set), mask [d_out][d_in] uint8; d_in % 4 == 0; DEVICE
+ * pointers, 16-byte aligned.  The output is slim_pack's `mask` argument.
+ */
+slim_status_t slim_mask_top2(const int8_t* codes, const float* xbar, int d_out, int d_in, uint8_t* mask, uint32_t* status_dev,
+                             void* cuda_stream);
+
+/*
  * Quantized adapters (Sec. 3.3 "Low-rank Adapter Quantization": 4-bit AbsMax group quantization,
  * groups of 128 elements share one quantization parameter; grid of Sec. 3.1 Eq. 2 / Eq. 5).
  * An adapter is a row-major bf16 matrix A[rows][cols] whose rows run along the contraction axis

@@ -40,6 +40,7 @@ SIGNATURES = {
     "slim_linear_fwd_tiled": (_I, [_P, _I, _P, _I, _F, _P, _P, _I, _I, _I, _P, _P, _SZ, _P, _P]),
     "slim_linear_fwd_tiled_host": (_I, [_P, _I, _P, _I, _F, _P, _P, _I, _I, _I, _P, _P, _P, _P, _SZ, _P, _P]),
     "slim_noalloc_scratch_needed": (_SZ, [_I, _I, _I, _I]),
+    "slim_mask_top2": (_I, [_P, _P, _I, _I, _P, _P, _P]),
     "slim_quant_workspace_bytes": (_SZ, [_I, _I]),
     "slim_quant": (_I, [_P, _I, _I, _P, _P, _P, _SZ, _P, _P]),
     "slim_adapter_code_bytes": (_SZ, [_I, _I]),
@@ -362,3 +363,14 @@ def slim_quant(W: torch.Tensor, status=None):
     off = 256 + (bins * 4 + 255) // 256 * 256
     tab = ws[off:off + 59 * 8].view(torch.float64)
     return codes, sa[:2], tab[:58].view(29, 2), tab[58]
+
+
+def slim_mask_top2(codes: torch.Tensor, xbar=None, status=None) -> torch.Tensor:
+    """2:4 mask (uint8, like codes) of int8 codes; xbar: float32 [d_in] average input magnitudes, or None."""
+    _dev(codes, torch.int8, "codes")
+    d_out, d_in = codes.shape
+    if xbar is not None:
+        _dev(xbar, torch.float32, "xbar")
+    mask = torch.empty((d_out, d_in), dtype=torch.uint8, device=codes.device)
+    _check(lib().slim_mask_top2(_ptr(codes), _ptr(xbar), d_out, d_in, _ptr(mask), _ptr(status), _stream()), "slim_mask_top2")
+    return mask

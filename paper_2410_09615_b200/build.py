@@ -9,7 +9,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libslim.so")
 SOURCES = ["api.cu", "pack.cu", "repack.cu", "fwd_simple.cu", "fwd_decode.cu", "fwd_decode_tiled.cu", "fwd_prefill.cu",
-           "fwd_noalloc.cu", "adapter_q.cu", "quant_search.cu"]
+           "fwd_noalloc.cu", "adapter_q.cu", "quant_search.cu", "mask.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math"]
 

@@ -209,6 +209,17 @@ slim_status_t slim_quant(const float* W, int d_out, int d_in, int8_t* codes, flo
     return launch_quant(W, d_out, d_in, codes, scale_alpha, workspace, status_dev, (cudaStream_t)cuda_stream);
 }
 
+slim_status_t slim_mask_top2(const int8_t* codes, const float* xbar, int d_out, int d_in, uint8_t* mask, uint32_t* status_dev,
+                             void* cuda_stream)
+{
+    reset_launch_count();
+    if (!codes || !mask || d_out < 1 || d_in < 4) return SLIM_ERR_INVALID_ARG;
+    if (d_in % 4 != 0) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(codes) || !aligned16(mask) || !aligned16(xbar)) return SLIM_ERR_INVALID_ARG;
+    if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return SLIM_ERR_INVALID_ARG;
+    return launch_mask_top2(codes, xbar, d_out, d_in, mask, status_dev, (cudaStream_t)cuda_stream);
+}
+
 size_t slim_adapter_code_bytes(int rows, int cols)
 {
     return rows < 1 || cols < 2 || cols % 2 != 0 ? 0 : (size_t)rows * (size_t)(cols / 2);

@@ -72,6 +72,8 @@ slim_status_t launch_pack_adapter(const __nv_bfloat16* A, int rows, int cols, ui
 slim_status_t launch_unpack_adapter(const uint8_t* codes, const __nv_bfloat16* scales, int rows, int cols, __nv_bfloat16* out,
                                     cudaStream_t st);
 
+slim_status_t launch_mask_top2(const int8_t* codes, const float* xbar, int d_out, int d_in, uint8_t* mask, uint32_t* status_dev,
+                               cudaStream_t st);
 size_t quant_workspace_bytes(int d_out, int d_in);
 slim_status_t launch_quant(const float* W, int d_out, int d_in, int8_t* codes, float* scale_alpha, void* ws,
                            uint32_t* status_dev, cudaStream_t st);

@@ -70,8 +70,12 @@ def test_quantize_then_pack_then_forward():
     s = float(sa[0])
     ocodes, oscale, _, _ = oracle.slim_quant(W)
     assert s == float(oscale) and np.array_equal(codes.cpu().numpy(), ocodes)
-    mask = inputs.top2_mask(W)
-    vals, meta = K.slim_pack(codes, to_dev(mask))
+    rng = np.random.default_rng(21)
+    xbar = (np.abs(rng.standard_normal(d_in)) + 0.1).astype(np.float32)          # synthetic average input magnitudes
+    mask_d = K.slim_mask_top2(codes, to_dev(xbar))
+    mask = oracle.mask_top2(ocodes, xbar)
+    assert np.array_equal(mask_d.cpu().numpy(), mask)
+    vals, meta = K.slim_pack(codes, mask_d)
     ovals, ometa = oracle.pack(ocodes, mask)
     assert np.array_equal(vals.cpu().numpy(), ovals) and np.array_equal(meta.cpu().numpy(), ometa)
     L, R = inputs.make_adapters(d_out, d_in, r, 21)
@@ -79,3 +83,20 @@ def test_quantize_then_pack_then_forward():
     Y = K.slim_linear_fwd(K.bf16_from_bits(X), vals, meta, s, K.bf16_from_bits(L), K.bf16_from_bits(R))
     res = parity.compare(inputs.bf16_bits_to_f64(K.bits_from_bf16(Y)), oracle.linear_fwd(X, ovals, ometa, oscale, L, R))
     assert res["ok"], res
+
+
+@pytest.mark.parametrize("d_out,d_in,seed,with_x", [(3, 8, 1, False), (64, 1000, 2, True), (4096, 4096, 3, True), (1000, 11008, 4, False)])
+def test_mask_top2_is_bit_exact(d_out, d_in, seed, with_x):
+    rng = np.random.default_rng([seed, 13])
+    codes = rng.integers(-8, 8, (d_out, d_in)).astype(np.int8)
+    xbar = rng.random(d_in).astype(np.float32) if with_x else None
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = K.slim_mask_top2(to_dev(codes), None if xbar is None else to_dev(xbar), status=status)
+    assert K.slim_last_launch_count() == 1
+    assert np.array_equal(got.cpu().numpy(), oracle.mask_top2(codes, xbar))
+    assert K.read_status(status) == 0
+    if with_x:
+        bad = xbar.copy(); bad[5] = -1.0
+        K.slim_mask_top2(to_dev(codes), to_dev(bad), status=status)
+        torch.cuda.synchronize()
+        assert K.read_status(status) & (1 << K.SLIM_ERR_INVALID_ARG)
