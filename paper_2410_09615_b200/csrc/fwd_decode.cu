@@ -78,6 +78,7 @@ struct DecodeParams {
     float s;
     int b, r, d_out, d_in;
     int KS, nblk, G, QT, r_pad;
+    int chunk_blocks;             // 256-column blocks of one R chunk: 2 (bf16 adapters), 8 (quantized adapters)
     int n_slots;
 };
 
@@ -257,11 +258,11 @@ __device__ __forceinline__ Share make_share(const DecodeParams& p, int cta) {
     sh.ks = cta % p.KS; sh.grp = cta / p.KS;
     sh.blk_begin = (int)((long long)sh.ks * p.nblk / p.KS);
     sh.nb = (int)((long long)(sh.ks + 1) * p.nblk / p.KS) - sh.blk_begin;
-    sh.Qk = (sh.nb + 1) / 2;
+    sh.Qk = (sh.nb + p.chunk_blocks - 1) / p.chunk_blocks;
     int qoff = 0;
     for (int k = 0; k < sh.ks; ++k) {
         const int nbk = (int)((long long)(k + 1) * p.nblk / p.KS) - (int)((long long)k * p.nblk / p.KS);
-        qoff += (nbk + 1) / 2;
+        qoff += (nbk + p.chunk_blocks - 1) / p.chunk_blocks;
     }
     sh.qoff = qoff;
     // R chunks: the first CTAs of the group take the remainder; weight tiles: the last ones do
@@ -385,7 +386,12 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
     const int n_ctas = gridDim.x;
     const Share sh = make_share(p, blockIdx.x);
     const int n_slots = p.n_slots;
-    const int l_chunks = p.r > 0 ? ceil_div(p.r, kLChunkCols) : 0;
+    // Chunks of quantized adapters are wider, so that a synchronisation covers more columns.  R: 2048 columns
+    // of codes fill a ring slot, a warp owns a whole 256-column block (four sub-steps of 64 columns, two groups
+    // of 128 with their own scales).  L: 1024 columns of r, a warp owns one group of 128 (two sub-steps), so
+    // that all warps work on the ranks in use (r <= 1024 is one chunk per output tile).
+    constexpr int kRC = QA ? 2048 : kRChunkCols, kLC = QA ? 1024 : kLChunkCols;
+    const int l_chunks = p.r > 0 ? ceil_div(p.r, kLC) : 0;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < n_slots; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], kConsumerWarps); }
@@ -416,12 +422,12 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
         // ---- R chunks: 16 rows x (256 or 512) columns of bf16 = 4 or 8 tiles of 64 columns
         for (int u = sh.r_begin; u < sh.r_begin + sh.r_count; ++u) {
             const int tile = u / sh.Qk, q = u % sh.Qk;
-            const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
+            const int cols = min(kRC, sh.nb * 256 - q * kRC);
             const int n_sub = QA ? cols / 256 : cols / 64;
             const int slot = acquire((uint32_t)n_sub * kSubTile);
             if (lane < n_sub) {
-                const int x = QA ? (sh.blk_begin * 256 + q * kRChunkCols) / 2 + 128 * lane      // bytes of codes
-                                 : sh.blk_begin * 256 + q * kRChunkCols + 64 * lane;
+                const int x = QA ? (sh.blk_begin * 256 + q * kRC) / 2 + 128 * lane      // bytes of codes
+                                 : sh.blk_begin * 256 + q * kRC + 64 * lane;
                 tma_tile(ring + (size_t)slot * kSlotBytes + lane * kSubTile, &tmR, x, tile * 16, &full_bar[slot]);
             }
         }
@@ -438,12 +444,12 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
         // ---- L chunks of the output tiles this CTA finishes (512 columns of r = 8 tiles)
         for (int tile = blockIdx.x; tile < tilesW && p.r > 0; tile += n_ctas) {
             for (int lc = 0; lc < l_chunks; ++lc) {
-                const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
+                const int cols = min(kLC, p.r - lc * kLC);
                 const int n_sub = QA ? ceil_div(cols, 256) : ceil_div(cols, 64);
                 const int slot = acquire((uint32_t)n_sub * kSubTile);
                 if (lane < n_sub)
                     tma_tile(ring + (size_t)slot * kSlotBytes + lane * kSubTile, &tmL,
-                             QA ? lc * (kLChunkCols / 2) + 128 * lane : lc * kLChunkCols + 64 * lane, tile * 16, &full_bar[slot]);
+                             QA ? lc * (kLC / 2) + 128 * lane : lc * kLC + 64 * lane, tile * 16, &full_bar[slot]);
             }
         }
         if (lane == 0 && !ok) flag_error(p.status, SLIM_ERR_TIMEOUT);
@@ -528,20 +534,22 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
             for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int h = 0; h < NT; ++h) {
-                    const int tile64 = q * 8 + warp;        // 64-column tile of the slice
+                    const int tile64 = QA ? warp * 4 + q : q * 8 + warp;   // 64-column tile of the slice (quantized: q = sub-step of the warp's block)
                     xd[q][jj][h] = tile64 < sh.nb * 4 ? lds128(xs + tile64 * x_sub + swz(g + 8 * h, jj * 64 + t * 16))
                                                       : make_uint4(0, 0, 0, 0);
                     if (QA) xd[q][jj][h] = pair_four_apart(xd[q][jj][h]);
                 }
         for (int u = sh.r_begin; u < sh.r_begin + sh.r_count; ++u) {
             const int tile = u / sh.Qk, q = u % sh.Qk;
-            const int cols = min(kRChunkCols, sh.nb * 256 - q * kRChunkCols);
-            const bool active = warp * 64 < cols;
-            float sc0 = 1.f, sc1 = 1.f;                   // quantized R: scales of rows g and g + 8 in the warp's group
+            const int cols = min(kRC, sh.nb * 256 - q * kRC);
+            const bool active = QA ? warp * 256 < cols : warp * 64 < cols;
+            float scA0 = 1.f, scA1 = 1.f, scB0 = 1.f, scB1 = 1.f;   // quantized R: scales of rows g, g + 8 in the block's two groups
             if (QA && active) {
-                const size_t grp = (size_t)((sh.blk_begin * 256 + q * kRChunkCols + warp * 64) >> 7), per_row = (size_t)(p.d_in >> 7);
-                sc0 = __bfloat162float(p.Rs[(size_t)(tile * 16 + g) * per_row + grp]);
-                sc1 = __bfloat162float(p.Rs[(size_t)(tile * 16 + g + 8) * per_row + grp]);
+                const size_t grp = (size_t)((sh.blk_begin * 256 + q * kRC + warp * 256) >> 7), per_row = (size_t)(p.d_in >> 7);
+                const __nv_bfloat16* s0 = p.Rs + (size_t)(tile * 16 + g) * per_row + grp;
+                const __nv_bfloat16* s1 = p.Rs + (size_t)(tile * 16 + g + 8) * per_row + grp;
+                scA0 = __bfloat162float(s0[0]); scB0 = __bfloat162float(s0[1]);
+                scA1 = __bfloat162float(s1[0]); scB1 = __bfloat162float(s1[1]);
             }
             const unsigned char* base = wait_full();
             if (u == sh.r_begin) STAMP(2);
@@ -551,27 +559,40 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
             if (QA && active) {
-                // warp w owns 64 columns = 32 bytes of codes in the 256-column tile w / 4
-                const unsigned char* sub = base + (warp >> 2) * kSubTile;
+                // warp w owns block w of the chunk = tile w of 256 codes per row; sub-steps of 64 columns
+                const unsigned char* sub = base + warp * kSubTile;
 #pragma unroll
-                for (int jj = 0; jj < 2; ++jj) {
-                    const uint32_t wa = lds32(sub + swz(g, (warp & 3) * 32 + jj * 16 + t * 4));
-                    const uint32_t wb = lds32(sub + swz(g + 8, (warp & 3) * 32 + jj * 16 + t * 4));
-                    uint32_t a[4], c[4];
+                for (int half = 0; half < 2; ++half) {             // the block's two groups of 128 columns
+                    float part[NT][4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) { a[i] = nib_pair(wa >> (4 * i)); c[i] = nib_pair(wb >> (4 * i)); }
+                    for (int h = 0; h < NT; ++h)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) part[h][e] = 0.f;
+#pragma unroll
+                    for (int ss = 0; ss < 2; ++ss) {
+                        const int sq = half * 2 + ss;
+#pragma unroll
+                        for (int jj = 0; jj < 2; ++jj) {
+                            const uint32_t wa = lds32(sub + swz(g, sq * 32 + jj * 16 + t * 4));
+                            const uint32_t wb = lds32(sub + swz(g + 8, sq * 32 + jj * 16 + t * 4));
+                            uint32_t a[4], c[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) { a[i] = nib_pair(wa >> (4 * i)); c[i] = nib_pair(wb >> (4 * i)); }
+#pragma unroll
+                            for (int h = 0; h < NT; ++h) {
+                                const uint4 xb = xd[sq][jj][h];
+                                mma_16816(part[h], a[0], c[0], a[1], c[1], xb.x, xb.y);
+                                mma_16816(part[h], a[2], c[2], a[3], c[3], xb.z, xb.w);
+                            }
+                        }
+                    }
+                    const float r0 = half ? scB0 : scA0, r1 = half ? scB1 : scA1;
 #pragma unroll
                     for (int h = 0; h < NT; ++h) {
-                        uint4 xb = xd[0][jj][h];
-                        if (q == 1) xb = xd[1][jj][h];
-                        if (q == 2) xb = xd[2][jj][h];
-                        if (q == 3) xb = xd[3][jj][h];
-                        mma_16816(acc[h], a[0], c[0], a[1], c[1], xb.x, xb.y);
-                        mma_16816(acc[h], a[2], c[2], a[3], c[3], xb.z, xb.w);
+                        acc[h][0] = fmaf(part[h][0], r0, acc[h][0]); acc[h][1] = fmaf(part[h][1], r0, acc[h][1]);
+                        acc[h][2] = fmaf(part[h][2], r1, acc[h][2]); acc[h][3] = fmaf(part[h][3], r1, acc[h][3]);
                     }
                 }
-#pragma unroll
-                for (int h = 0; h < NT; ++h) { acc[h][0] *= sc0; acc[h][1] *= sc0; acc[h][2] *= sc1; acc[h][3] *= sc1; }
             } else if (active) {
                 // warp w owns the 64-column tile w of the chunk
                 const unsigned char* sub = base + warp * kSubTile;
@@ -595,7 +616,7 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
                     }
             }
             release();
-            const float sum = block_tile_sum<NT>(next_red(), acc, active, min(kConsumerWarps, cols / 64));
+            const float sum = block_tile_sum<NT>(next_red(), acc, active, QA ? cols / 256 : min(kConsumerWarps, cols / 64));
             if (threadIdx.x < frag)
                 st_gpu(p.Tpart + ((size_t)tile * p.QT + sh.qoff + q) * frag + threadIdx.x, slot_bits(sum));
         }
@@ -729,10 +750,11 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
         if (tile == (int)blockIdx.x) STAMP(9);
         float ysum = 0.f;
         for (int lc = 0; lc < l_chunks; ++lc) {
-            const int cols = min(kLChunkCols, p.r - lc * kLChunkCols);
-            float sc0 = 1.f, sc1 = 1.f;                   // quantized L: scales of rows g and g + 8 in the warp's group
-            if (QA && warp * 64 < cols) {
-                const size_t grp = (size_t)((lc * kLChunkCols + warp * 64) >> 7), per_row = (size_t)((p.r + 127) >> 7);
+            const int cols = min(kLC, p.r - lc * kLC);
+            const bool q_active = QA && warp * 128 < cols;
+            float sc0 = 0.f, sc1 = 0.f;                   // quantized L: scales of rows g, g + 8 in the warp's group
+            if (q_active) {
+                const size_t grp = (size_t)((lc * kLC + warp * 128) >> 7), per_row = (size_t)((p.r + 127) >> 7);
                 sc0 = __bfloat162float(p.Ls[(size_t)(tile * 16 + g) * per_row + grp]);
                 sc1 = __bfloat162float(p.Ls[(size_t)(tile * 16 + g + 8) * per_row + grp]);
             }
@@ -743,26 +765,32 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[h][e] = 0.f;
             // warp w owns the 64-column tile w of the chunk (two 32-column blocks)
-            if (QA && warp * 64 < cols) {
-                const unsigned char* sub = base + (warp >> 2) * kSubTile;   // codes past r read as zero
+            if (q_active) {
+                // quantized: the warp's group = 64 bytes of codes per row in the tile of 256 codes w / 2; codes past r read as zero
+                const unsigned char* sub = base + (warp >> 1) * kSubTile;
 #pragma unroll
-                for (int jj = 0; jj < 2; ++jj) {
-                    const int kk = warp * 64 + jj * 32 + 8 * t;
-                    const uint32_t wa = lds32(sub + swz(g, (warp & 3) * 32 + jj * 16 + t * 4));
-                    const uint32_t wb = lds32(sub + swz(g + 8, (warp & 3) * 32 + jj * 16 + t * 4));
-                    uint32_t a[4], c[4];
+                for (int ss = 0; ss < 2; ++ss) {
+                    if (warp * 128 + ss * 64 < cols) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) { a[i] = nib_pair(wa >> (4 * i)); c[i] = nib_pair(wb >> (4 * i)); }
+                        for (int jj = 0; jj < 2; ++jj) {
+                            const int kk = warp * 128 + ss * 64 + jj * 32 + 8 * t;          // column inside the chunk
+                            const uint32_t wa = lds32(sub + swz(g, (warp & 1) * 64 + ss * 32 + jj * 16 + t * 4));
+                            const uint32_t wb = lds32(sub + swz(g + 8, (warp & 1) * 64 + ss * 32 + jj * 16 + t * 4));
+                            uint32_t a[4], c[4];
 #pragma unroll
-                    for (int h = 0; h < NT; ++h) {
-                        const uint4 tb = pair_four_apart(lds128(Ts + (size_t)(g + 8 * h) * p.r_pad + lc * kLChunkCols + kk));
-                        mma_16816(acc[h], a[0], c[0], a[1], c[1], tb.x, tb.y);
-                        mma_16816(acc[h], a[2], c[2], a[3], c[3], tb.z, tb.w);
+                            for (int i = 0; i < 4; ++i) { a[i] = nib_pair(wa >> (4 * i)); c[i] = nib_pair(wb >> (4 * i)); }
+#pragma unroll
+                            for (int h = 0; h < NT; ++h) {
+                                const uint4 tb = pair_four_apart(lds128(Ts + (size_t)(g + 8 * h) * p.r_pad + lc * kLC + kk));
+                                mma_16816(acc[h], a[0], c[0], a[1], c[1], tb.x, tb.y);
+                                mma_16816(acc[h], a[2], c[2], a[3], c[3], tb.z, tb.w);
+                            }
+                        }
                     }
                 }
 #pragma unroll
                 for (int h = 0; h < NT; ++h) { acc[h][0] *= sc0; acc[h][1] *= sc0; acc[h][2] *= sc1; acc[h][3] *= sc1; }
-            } else if (warp * 64 < cols) {
+            } else if (!QA && warp * 64 < cols) {
                 const unsigned char* sub = base + warp * kSubTile;
 #pragma unroll
                 for (int jj = 0; jj < 2; ++jj) {
@@ -771,7 +799,7 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
                     const uint4 lb = lds128(sub + swz(g + 8, jj * 64 + t * 16));
 #pragma unroll
                     for (int h = 0; h < NT; ++h) {
-                        const uint4 tb = lds128(Ts + (size_t)(g + 8 * h) * p.r_pad + lc * kLChunkCols + kk);
+                        const uint4 tb = lds128(Ts + (size_t)(g + 8 * h) * p.r_pad + lc * kLC + kk);
                         mma_16816(acc[h], la.x, lb.x, la.y, lb.y, tb.x, tb.y);
                         mma_16816(acc[h], la.z, lb.z, la.w, lb.w, tb.z, tb.w);
                     }
@@ -812,7 +840,7 @@ static bool shape_ok(int b, int d_out, int d_in, int r) {
            d_in / 256 <= kMaxSlices * kConsumerWarps;
 }
 
-static bool make_plan(int b, int d_out, int d_in, int r, int ctas, DecodePlan* pl) {
+static bool make_plan(int b, int d_out, int d_in, int r, int ctas, DecodePlan* pl, bool qa = false) {
     if (!shape_ok(b, d_out, d_in, r)) return false;
     pl->nt = b <= 8 ? 1 : 2;
     pl->nblk = d_in / 256;
@@ -822,7 +850,7 @@ static bool make_plan(int b, int d_out, int d_in, int r, int ctas, DecodePlan* p
     int qt = 0;
     for (int k = 0; k < pl->KS; ++k) {
         const int nbk = (int)((long long)(k + 1) * pl->nblk / pl->KS) - (int)((long long)k * pl->nblk / pl->KS);
-        qt += (nbk + 1) / 2;
+        qt += qa ? (nbk + 7) / 8 : (nbk + 1) / 2;       // R chunks of 8 blocks (quantized adapters) or 2
     }
     pl->QT = qt;
     pl->r_pad = pad_rank(r);
@@ -934,7 +962,7 @@ static slim_status_t launch_decode_any(const __nv_bfloat16* X, int b, const uint
     DecodePlan pl;
     const int nt = b <= 8 ? 1 : 2;
     const int ctas = decode_ctas(nt);
-    if (ctas < 1 || !make_plan(b, d_out, d_in, r, ctas, &pl)) return SLIM_ERR_UNSUPPORTED_SHAPE;
+    if (ctas < 1 || !make_plan(b, d_out, d_in, r, ctas, &pl, qa)) return SLIM_ERR_UNSUPPORTED_SHAPE;
     DecodeParams p;
     p.X = X; p.vals = vals; p.meta = meta; p.Y = Y;
     p.L = qa ? nullptr : static_cast<const __nv_bfloat16*>(L); p.R = qa ? nullptr : static_cast<const __nv_bfloat16*>(R);
@@ -947,7 +975,7 @@ static slim_status_t launch_decode_any(const __nv_bfloat16* X, int b, const uint
     p.status = status_dev;
     p.s = s; p.b = b; p.r = r; p.d_out = d_out; p.d_in = d_in;
     p.KS = pl.KS; p.nblk = pl.nblk; p.G = pl.G; p.QT = pl.QT; p.r_pad = pl.r_pad;
-    p.n_slots = pl.n_slots;
+    p.n_slots = pl.n_slots; p.chunk_blocks = qa ? 8 : 2;
     CUtensorMap tmX, tmV, tmM, tmR, tmL;
     bool ok = make_tile_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, nt * 8) &&
               make_tile_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, 16) &&
