@@ -748,7 +748,12 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
                 slots_request(pb, p.Ppart + (size_t)(tile + n_ctas) * frag + threadIdx.x, p_stride, p.KS);
         }
         if (tile == (int)blockIdx.x) STAMP(9);
-        float ysum = 0.f;
+        // every chunk of L adds into the same accumulators: one cross-warp sum per output tile
+        float ytot[NT][4];
+#pragma unroll
+        for (int h = 0; h < NT; ++h)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) ytot[h][e] = 0.f;
         for (int lc = 0; lc < l_chunks; ++lc) {
             const int cols = min(kLC, p.r - lc * kLC);
             const bool q_active = QA && warp * 128 < cols;
@@ -789,7 +794,10 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
                     }
                 }
 #pragma unroll
-                for (int h = 0; h < NT; ++h) { acc[h][0] *= sc0; acc[h][1] *= sc0; acc[h][2] *= sc1; acc[h][3] *= sc1; }
+                for (int h = 0; h < NT; ++h) {
+                    ytot[h][0] = fmaf(acc[h][0], sc0, ytot[h][0]); ytot[h][1] = fmaf(acc[h][1], sc0, ytot[h][1]);
+                    ytot[h][2] = fmaf(acc[h][2], sc1, ytot[h][2]); ytot[h][3] = fmaf(acc[h][3], sc1, ytot[h][3]);
+                }
             } else if (!QA && warp * 64 < cols) {
                 const unsigned char* sub = base + warp * kSubTile;
 #pragma unroll
@@ -805,9 +813,15 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
                     }
                 }
             }
+            if (!QA) {
+#pragma unroll
+                for (int h = 0; h < NT; ++h)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) ytot[h][e] += acc[h][e];
+            }
             release();
-            ysum += block_tile_sum<NT>(next_red(), acc, true, kConsumerWarps);
         }
+        const float ysum = l_chunks > 0 ? block_tile_sum<NT>(next_red(), ytot, true, kConsumerWarps) : 0.f;
         if (threadIdx.x < frag) {
             const int hq = threadIdx.x >> 5, ln = threadIdx.x & 31;
             const int h = hq >> 2, q = hq & 3;
