@@ -432,6 +432,13 @@ def run_ours(args):
             prefill_rows += prefill_table(K, small, model, stream, 2048)
             del small
         line["per_case"] = tables
+        # batches between the two of the step, on the two large 70B layers: where the layout hint changes sides
+        big = [ly for ly in host70 if ly["d_in"] * ly["d_out"] >= (1 << 27)]
+        ws_mid = torch.empty(max(K.slim_workspace_bytes(b, l["d_out"], l["d_in"], l["r"]) for l in big for b in (2, 4, 8)),
+                             dtype=torch.uint8, device=dev)
+        K.slim_workspace_reset(ws_mid)
+        line["per_case_batch_sweep"] = per_case_table(K, lib, big, "70b", ws_mid, ws_mid.numel(), status, stream, peak, batches=(2, 4, 8))
+        del ws_mid
         # the step's two kernels apart: bytes and time of the 70B rows each of them serves, weighted by
         # the number of such linears in the block
         count = {ly["name"]: ly["count"] for ly in host70}
@@ -485,7 +492,7 @@ def time_graph_of_calls(fn, calls, stream, replays=10):
     return float(np.median(times)), float(np.min(times))
 
 
-def per_case_table(K, lib, layers, model, ws, ws_bytes, status, stream, peak):
+def per_case_table(K, lib, layers, model, ws, ws_bytes, status, stream, peak, batches=BATCHES):
     """Per (layer, batch): us/call of both small-batch kernels over rotating copies (> 2x L2 between
     reuses); `us` is the one slim_decode_layout_hint names, with its algorithmic GB/s and fraction of
     the HBM roofline."""
@@ -496,7 +503,12 @@ def per_case_table(K, lib, layers, model, ws, ws_bytes, status, stream, peak):
         n_copies = int(np.ceil(2 * L2_BYTES / per_copy)) + 1
         copies = [weight_copy(ly) for _ in range(n_copies)]
         torch.cuda.synchronize()
-        for b in BATCHES:
+        for b in batches:
+            if b not in ly["Xd"]:
+                g = torch.Generator(device=ly["Ld"].device)
+                g.manual_seed(1000 + b)
+                ly["Xd"][b] = torch.randn((b, ly["d_in"]), device=ly["Ld"].device, generator=g).bfloat16()
+                ly["Yd"][b] = torch.empty((b, ly["d_out"]), dtype=torch.bfloat16, device=ly["Ld"].device)
             hint_tiled = K.slim_decode_layout_hint(b, ly["d_out"], ly["d_in"], ly["r"]) == K.LAYOUT_DECODE_TILED
             t = {}
             for tiled in (False, True):
