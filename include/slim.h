@@ -285,9 +285,10 @@ slim_status_t slim_unpack_adapter(const uint8_t* codes, const void* scales, int 
 /*
  * The layer forward with quantized adapters (SLiM-LoRA^Q; Sec. 3.3, with the layer of Sec. 3.2):
  * slim_linear_fwd with L and R given as codes and scales (Lq/Ls for L[d_out][r], Rq/Rs for
- * R[r][d_in]).  r >= 16.  For b <= 16, shapes the decode kernel takes and r % 32 == 0 (the rows of
- * L's codes must be 16-byte multiples) the decode kernel reads codes and scales as they are: it
- * multiplies the exact integer codes and scales its accumulator once per group, and a call moves
+ * R[r][d_in]).  r >= 16.  For b <= 16 and shapes the decode kernel takes, the decode kernel reads codes
+ * and scales as they are (through tensor maps; L's codes with plain loads when their rows of r / 2 bytes
+ * are no 16-byte multiples): it multiplies the exact integer codes and scales its accumulator once
+ * per group, and a call moves
  * 4.125 bits per adapter element instead of 16 (Sec. 4 "Speedup": quantized adapters cut the
  * adapters' share of the layer's time).  Otherwise the adapters are expanded to bf16 (each value
  * rounded once, nearest even) into the tail of the workspace and the kernel slim_linear_fwd would

@@ -79,6 +79,8 @@ struct DecodeParams {
     int b, r, d_out, d_in;
     int KS, nblk, G, QT, r_pad;
     int chunk_blocks;             // 256-column blocks of one R chunk: 2 (bf16 adapters), 8 (quantized adapters)
+    int l_direct;                 // quantized adapters whose rows of L codes are no 16-byte multiples: read with plain loads
+    const uint8_t* Lq;            // codes of L (used when l_direct)
     int n_slots;
 };
 
@@ -442,7 +444,7 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
                 tma_tile(dst + lane * kSubTile, &tmM, sh.blk_begin * 32 + 128 * (lane - 4), tile * 16, &full_bar[slot]);
         }
         // ---- L chunks of the output tiles this CTA finishes (512 columns of r = 8 tiles)
-        for (int tile = blockIdx.x; tile < tilesW && p.r > 0; tile += n_ctas) {
+        for (int tile = blockIdx.x; tile < tilesW && p.r > 0 && !(QA && p.l_direct); tile += n_ctas) {
             for (int lc = 0; lc < l_chunks; ++lc) {
                 const int cols = min(kLC, p.r - lc * kLC);
                 const int n_sub = QA ? ceil_div(cols, 256) : ceil_div(cols, 64);
@@ -763,7 +765,24 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
                 sc0 = __bfloat162float(p.Ls[(size_t)(tile * 16 + g) * per_row + grp]);
                 sc1 = __bfloat162float(p.Ls[(size_t)(tile * 16 + g + 8) * per_row + grp]);
             }
-            const unsigned char* base = wait_full();
+            const bool direct = QA && p.l_direct;
+            // codes of L straight from global memory (rows of r / 2 bytes, 4-byte aligned words; past r: zero)
+            uint32_t dw[2][2][2] = {};
+            if (direct && q_active) {
+                const uint8_t* row0 = p.Lq + (size_t)(tile * 16 + g) * (size_t)(p.r / 2);
+                const uint8_t* row1 = row0 + (size_t)8 * (size_t)(p.r / 2);
+#pragma unroll
+                for (int ss = 0; ss < 2; ++ss)
+#pragma unroll
+                    for (int jj = 0; jj < 2; ++jj) {
+                        const int col = lc * kLC + warp * 128 + ss * 64 + jj * 32 + 8 * t;
+                        if (col < p.r) {
+                            dw[ss][jj][0] = __ldg(reinterpret_cast<const uint32_t*>(row0 + col / 2));
+                            dw[ss][jj][1] = __ldg(reinterpret_cast<const uint32_t*>(row1 + col / 2));
+                        }
+                    }
+            }
+            const unsigned char* base = direct ? nullptr : wait_full();
             float acc[NT][4];
 #pragma unroll
             for (int h = 0; h < NT; ++h)
@@ -779,8 +798,8 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
 #pragma unroll
                         for (int jj = 0; jj < 2; ++jj) {
                             const int kk = warp * 128 + ss * 64 + jj * 32 + 8 * t;          // column inside the chunk
-                            const uint32_t wa = lds32(sub + swz(g, (warp & 1) * 64 + ss * 32 + jj * 16 + t * 4));
-                            const uint32_t wb = lds32(sub + swz(g + 8, (warp & 1) * 64 + ss * 32 + jj * 16 + t * 4));
+                            const uint32_t wa = direct ? dw[ss][jj][0] : lds32(sub + swz(g, (warp & 1) * 64 + ss * 32 + jj * 16 + t * 4));
+                            const uint32_t wb = direct ? dw[ss][jj][1] : lds32(sub + swz(g + 8, (warp & 1) * 64 + ss * 32 + jj * 16 + t * 4));
                             uint32_t a[4], c[4];
 #pragma unroll
                             for (int i = 0; i < 4; ++i) { a[i] = nib_pair(wa >> (4 * i)); c[i] = nib_pair(wb >> (4 * i)); }
@@ -819,7 +838,7 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
 #pragma unroll
                     for (int e = 0; e < 4; ++e) ytot[h][e] += acc[h][e];
             }
-            release();
+            if (!direct) release();
         }
         const float ysum = l_chunks > 0 ? block_tile_sum<NT>(next_red(), ytot, true, kConsumerWarps) : 0.f;
         if (threadIdx.x < frag) {
@@ -906,9 +925,10 @@ static int decode_ctas(int nt) {
     return di->sm_count * (di->decode_ctas_per_sm[nt - 1] > 0 ? 1 : 0);
 }
 
-// Quantized adapters: the rows of L's codes (r / 2 bytes) must be 16-byte multiples for the tensor map.
+// Quantized adapters: when the rows of L's codes (r / 2 bytes) are no 16-byte multiples no tensor map can
+// describe them, and the kernel reads them with plain loads.
 bool decode_supports_q(int b, int d_out, int d_in, int r) {
-    return r >= 32 && r % 32 == 0 && decode_supports(b, d_out, d_in, r);
+    return r >= 16 && decode_supports(b, d_out, d_in, r);
 }
 
 bool decode_supports(int b, int d_out, int d_in, int r) {
@@ -990,13 +1010,15 @@ static slim_status_t launch_decode_any(const __nv_bfloat16* X, int b, const uint
     p.s = s; p.b = b; p.r = r; p.d_out = d_out; p.d_in = d_in;
     p.KS = pl.KS; p.nblk = pl.nblk; p.G = pl.G; p.QT = pl.QT; p.r_pad = pl.r_pad;
     p.n_slots = pl.n_slots; p.chunk_blocks = qa ? 8 : 2;
+    p.l_direct = qa && r % 32 != 0; p.Lq = qa ? static_cast<const uint8_t*>(L) : nullptr;
     CUtensorMap tmX, tmV, tmM, tmR, tmL;
     bool ok = make_tile_map(&tmX, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, nt * 8) &&
               make_tile_map(&tmV, vals, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 4, (uint64_t)d_out, 16) &&
               make_tile_map(&tmM, meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 8, (uint64_t)d_out, 16);
     if (ok && r > 0 && qa)
         ok = make_tile_map(&tmR, R, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)d_in / 2, (uint64_t)r, 16) &&
-             make_tile_map(&tmL, L, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)r / 2, (uint64_t)d_out, 16);
+             (r % 32 != 0 ? (tmL = tmV, true)       // not used: those codes are read with plain loads
+                          : make_tile_map(&tmL, L, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)r / 2, (uint64_t)d_out, 16));
     else if (ok && r > 0)
         ok = make_tile_map(&tmR, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 16) &&
              make_tile_map(&tmL, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, 16);

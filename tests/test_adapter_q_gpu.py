@@ -79,19 +79,19 @@ def run_q(d_in, d_out, r, b, seed, wseed=None, rows=None):
 
 
 @pytest.mark.parametrize("d_in,d_out,r,b", [
-    # decode kernel reading codes and scales as they are (r % 32 == 0): short last group, two chunk widths,
-    # several k-slices, both token-tile counts
+    # decode kernel reading codes and scales as they are: short last group, two chunk widths, several
+    # k-slices, both token-tile counts; ranks whose rows of L codes are no 16-byte multiples (plain loads)
     (256, 64, 32, 1), (512, 512, 64, 8), (768, 208, 96, 16), (1024, 384, 160, 5), (2304, 128, 416, 16), (4352, 96, 544, 3),
     (1280, 1040, 1056, 9),
-    # adapters expanded first: decode kernel with r % 32 != 0, CUDA-core kernel, prefill kernel
-    (256, 64, 16, 1), (768, 208, 48, 16), (1024, 384, 144, 5),
+    (256, 64, 16, 1), (768, 208, 48, 16), (1024, 384, 144, 5), (8192, 1024, 112, 16), (2048, 160, 1040, 2),
+    # adapters expanded first: CUDA-core kernel, prefill kernel
     (320, 48, 32, 3),
     (512, 256, 64, 200), (640, 384, 144, 70),
 ])
 def test_forward_on_quantized_adapters_small(d_in, d_out, r, b):
     res = run_q(d_in, d_out, r, b, seed=300 + r + b)
     assert res["ok"], res
-    fused = b <= 16 and d_in % 256 == 0 and r % 32 == 0
+    fused = b <= 16 and d_in % 256 == 0
     assert res["launches"] == 1 if fused else res["launches"] >= 3      # else two expansions and the forward launches
 
 
