@@ -15,12 +15,12 @@ operands from HBM (the L2 holds 126 MB).  The step is captured in a CUDA graph a
 is taken with CUDA events on the launching stream, max over ranks.  Prints one JSON line, which
 also carries per-case tables for the 7B / 13B / 70B shapes, prefill tables (2048 and 4096 tokens,
 rank sweep on the 70B shapes), an end-to-end figure through the host-buffer entry point and the CPU
-oracle timed on this machine.
+oracle timed on the host's cores.
 
 With N > 1 every rank runs the same step on its own GPU (independent replicas, no collective on
 the data path).
 
---impl reference times the CPU oracle (oracle/) on this machine's host cores on the same workload:
+--impl reference times the CPU oracle (oracle/) on the host's cores on the same workload:
 each step runs each distinct (shape, batch) call once and weights it by how often the block uses it.
 """
 from __future__ import annotations
@@ -730,7 +730,7 @@ def time_e2e(K, lib, layers, step_calls, ws, ws_bytes, status, stream, args, wor
 
 
 def time_cpu_baseline(layers, repeats=2):
-    """The oracle, as it stands, on this machine's host cores: the whole step (a bounded sample: one pass over
+    """The oracle, as it stands, on the host's cores: the whole step (a bounded sample: one pass over
     each distinct (shape, batch) pair per repeat), plus a single-thread timing of the smallest layer."""
     import oracle
     host = []
