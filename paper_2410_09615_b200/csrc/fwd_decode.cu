@@ -119,6 +119,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     }
     return false;
 }
+// Has the phase completed?  Does not wait: the answer takes a couple of hundred cycles to come back, so it
+// is asked one slot ahead and looked at when the slot is needed.
+__device__ __forceinline__ uint32_t mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return done;
+}
 // One TMA tile (box of the tensor behind `tmap`, starting at element column x,
 // row y) into shared memory; completion in bytes on `bar`.
 __device__ __forceinline__ void tma_tile(void* dst, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
@@ -496,15 +507,21 @@ decode_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmX,
     uint32_t it = 0;
     int red_buf = 0;
     bool ok = true;
+    // Ring position kept as running (slot, phase); the next slot's barrier is asked about while the current
+    // slot is being consumed (an answer takes about 200 cycles even when the phase is long complete).
+    int c_slot = 0;
+    uint32_t c_phase = 0, ahead = 0;                       // ahead: the current slot was already seen full
     auto wait_full = [&]() -> unsigned char* {
-        const int slot = it % n_slots;
-        ok = mbar_wait(&full_bar[slot], (it / n_slots) & 1) && ok;
-        return ring + (size_t)slot * kSlotBytes;
+        if (!ahead) ok = mbar_wait(&full_bar[c_slot], c_phase) && ok;
+        const int ns = c_slot + 1 == n_slots ? 0 : c_slot + 1;
+        ahead = mbar_test(&full_bar[ns], ns == 0 ? c_phase ^ 1u : c_phase);
+        return ring + (size_t)c_slot * kSlotBytes;
     };
     auto release = [&]() {
         __syncwarp();
-        if (lane == 0) mbar_arrive(&empty_bar[it % n_slots]);
+        if (lane == 0) mbar_arrive(&empty_bar[c_slot]);
         ++it;
+        if (++c_slot == n_slots) { c_slot = 0; c_phase ^= 1u; }
     };
     auto next_red = [&]() -> float* {
         float* r = red_base + red_buf * kConsumerWarps * frag;
