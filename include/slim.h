@@ -196,7 +196,8 @@ slim_status_t slim_linear_fwd_tiled(const void* X, int b, const void* tiled, int
  * 0 = the packed format (slim_linear_fwd), SLIM_LAYOUT_DECODE_TILED = the decode-tiled copy
  * (slim_linear_fwd_tiled).  The tiled kernel streams large weights at a higher rate but has a
  * longer fixed start and end that grows with the batch (activations and T are staged by few warps):
- * the rule is "tiled when b <= 4 and the packed weight has 64 MiB or more", from timings of both
+ * the rule is "tiled when the packed weight has 64 MiB or more and b <= 4 (b <= 2 when d_out < d_in)",
+ * from timings of both
  * kernels on the LLaMA-2 layer shapes.  Returns 0 as well for shapes the tiled kernel does not take
  * and for illegal arguments.  (Storage layout is the implementation's choice: Sec. 4 "Speedup"
  * measures the layer, the paper fixes no format.)

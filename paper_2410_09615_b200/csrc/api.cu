@@ -129,7 +129,7 @@ slim_status_t slim_workspace_reset(void* workspace, size_t workspace_bytes_, voi
 
 int slim_decode_layout_hint(int b, int d_out, int d_in, int r)
 {
-    if (b < 1 || b > 4 || r < 0 || r % 16 != 0 || check_weight_shape(d_out, d_in) != SLIM_OK) return 0;
+    if (b < 1 || b > (d_out >= d_in ? 4 : 2) || r < 0 || r % 16 != 0 || check_weight_shape(d_out, d_in) != SLIM_OK) return 0;
     if ((size_t)d_out * (size_t)d_in * 3 / 8 < ((size_t)64 << 20)) return 0;
     slim_status_t err;
     const DeviceInfo* di = device_info(&err);
