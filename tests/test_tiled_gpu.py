@@ -217,3 +217,17 @@ def test_full_size_tiled_decode_configs(d_in, d_out, r, b, seed, wseed):
     the benchmark times); all tokens and all output columns compared."""
     res = run_tiled(d_in, d_out, r, b, seed, wseed, check_repack=(d_out * d_in <= 5120 * 13824))
     assert res["ok"], res
+
+
+def test_layout_hint_follows_the_stated_rule():
+    """Tiled when the packed weight has 64 MiB or more and b <= 4 (b <= 2 when d_out < d_in); packed otherwise."""
+    T = K.LAYOUT_DECODE_TILED
+    assert K.slim_decode_layout_hint(1, 28672, 8192, 832) == T
+    assert K.slim_decode_layout_hint(4, 28672, 8192, 832) == T
+    assert K.slim_decode_layout_hint(5, 28672, 8192, 832) == 0
+    assert K.slim_decode_layout_hint(2, 8192, 28672, 832) == T
+    assert K.slim_decode_layout_hint(4, 8192, 28672, 832) == 0
+    assert K.slim_decode_layout_hint(16, 28672, 8192, 832) == 0
+    assert K.slim_decode_layout_hint(1, 8192, 8192, 832) == 0          # 24 MiB of packed weight
+    assert K.slim_decode_layout_hint(1, 28672, 8192, 8) == 0           # not a legal rank
+    assert K.slim_decode_layout_hint(0, 28672, 8192, 832) == 0
