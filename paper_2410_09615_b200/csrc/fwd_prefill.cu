@@ -322,6 +322,10 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
 {
     using namespace pf;
     using Cfg = PfCfg<N, TWO, PRE>;
+    // The dense-only launch lets the launches behind it start at once (programmatic dependent launch): the
+    // main launch's sparse stages do not need T', and it waits (griddepcontrol.wait) just before its first
+    // request of a T' tile.
+    if (PRE) asm volatile("griddepcontrol.launch_dependents;");
     constexpr int kBTile = Cfg::kBTile, kStageBytes = Cfg::kStageBytes, kECol = Cfg::kECol, kPStages = Cfg::kStages;
     constexpr int kPkSlots = Cfg::kPkSlots, kDK = Cfg::kDK;
     extern __shared__ unsigned char smem_raw[];
@@ -386,9 +390,15 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
         // a barrier would mistake an old phase for the one it needs).  Sparse stage: lane 0
         // requests the token tile.  Dense stage: lanes 0 and 1 request the token tile and the A2
         // tile with one instruction.
+        bool t_ready = PRE;                                 // main launch: T' (and everything before it) is complete
         for (int it = warp == kWarpXEven ? 0 : 1; it < n_total; it += 2) {
             const int st = it % kPStages;
             const bool sparse = it < p.n1;
+            if (!sparse && !t_ready) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                asm volatile("fence.proxy.async;" ::: "memory");   // the tiles are read by the async proxy
+                t_ready = true;
+            }
             // The whole warp waits (no lane is left behind at a warp barrier while another
             // spins: that costs some hundred nanoseconds per stage); lane 0 arms the barrier.
             if (it >= kPStages) ok = mbar_wait(&empty[st], ((it / kPStages) & 1) ^ 1, abort_flag) && ok;
@@ -579,16 +589,19 @@ prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tmV,
 // Sum of the K slices' partial tiles, scaled and rounded to bf16 (fixed order: deterministic).
 __global__ void pre_reduce_kernel(const float* __restrict__ part, int slices, size_t n, float scale, __nv_bfloat16* __restrict__ out)
 {
-    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-    if (i >= n) return;
-    float4 acc = *reinterpret_cast<const float4*>(part + i);
-    for (int z = 1; z < slices; ++z) {
-        const float4 v = *reinterpret_cast<const float4*>(part + (size_t)z * n + i);
-        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    // lets the main launch start, then waits for the dense-only launch whose partial tiles it adds
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < n; i += (size_t)gridDim.x * blockDim.x * 4) {
+        float4 acc = *reinterpret_cast<const float4*>(part + i);
+        for (int z = 1; z < slices; ++z) {
+            const float4 v = *reinterpret_cast<const float4*>(part + (size_t)z * n + i);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        __nv_bfloat162 lo = __floats2bfloat162_rn(scale * acc.x, scale * acc.y), hi = __floats2bfloat162_rn(scale * acc.z, scale * acc.w);
+        uint2 o; o.x = *reinterpret_cast<uint32_t*>(&lo); o.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(out + i) = o;
     }
-    __nv_bfloat162 lo = __floats2bfloat162_rn(scale * acc.x, scale * acc.y), hi = __floats2bfloat162_rn(scale * acc.z, scale * acc.w);
-    uint2 o; o.x = *reinterpret_cast<uint32_t*>(&lo); o.y = *reinterpret_cast<uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(out + i) = o;
 }
 
 // ------------------------------------------------------------------ host side
@@ -649,16 +662,19 @@ static std::atomic<bool> g_prefill_attr_set[64];   // attributes set once per de
 template <int N, bool TWO, bool PRE = false>
 static slim_status_t launch_tile_kernel(const PrefillParams& q, int m_rows, const CUtensorMap& tmV, const CUtensorMap& tmM,
                                         const CUtensorMap& tmX, const CUtensorMap& tmA2, const CUtensorMap& tmB2,
-                                        cudaStream_t st, int slices = 1) {
+                                        cudaStream_t st, int slices = 1, bool after_dense_only = false) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ceil_div(m_rows, kPM), ceil_div(q.b, N), slices);
     cfg.blockDim = dim3(kPThreads);
     cfg.dynamicSmemBytes = PfCfg<N, TWO, PRE>::kSmem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = TWO ? 2 : 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    // may start while the launch before it (the dense-only launch or its reduction) still runs
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = after_dense_only ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, prefill_kernel<N, TWO, PRE>, q, tmV, tmM, tmX, tmA2, tmB2);
     count_launch(1);
     return e == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
@@ -716,9 +732,17 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
         if (rc != SLIM_OK) return rc;
         if (q.part) {
             const size_t n = (size_t)b * r;
-            pre_reduce_kernel<<<(unsigned)((n / 4 + 255) / 256), 256, 0, st>>>(q.part, pl.slices, n, q.scale, Tq);
+            // a small grid: its blocks wait beside the dense-only launch's and must leave room for the main launch's
+            cudaLaunchConfig_t rc_cfg = {};
+            const unsigned want = (unsigned)((n / 4 + 255) / 256), cap = (unsigned)(2 * di->sm_count);
+            rc_cfg.gridDim = dim3(want < cap ? want : cap); rc_cfg.blockDim = dim3(256); rc_cfg.dynamicSmemBytes = 0; rc_cfg.stream = st;
+            cudaLaunchAttribute rc_attr[1];
+            rc_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            rc_attr[0].val.programmaticStreamSerializationAllowed = 1;
+            rc_cfg.attrs = rc_attr; rc_cfg.numAttrs = 1;
+            const cudaError_t re = cudaLaunchKernelEx(&rc_cfg, pre_reduce_kernel, (const float*)q.part, pl.slices, n, q.scale, Tq);
             count_launch(1);
-            if (cudaGetLastError() != cudaSuccess) return SLIM_ERR_CUDA;
+            if (re != cudaSuccess) return SLIM_ERR_CUDA;
         }
         // dense stages of the main kernel: 64 columns (128-byte rows), or 32 (64-byte rows) in the pair kernel
         ok = pf_map(&tmA2, L, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)r, (uint64_t)d_out, dk, kPM, dk == 64 ? 128 : 64) &&
@@ -736,9 +760,10 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
         return cudaMemsetAsync(Y, 0, (size_t)b * d_out * 2, st) == cudaSuccess ? SLIM_OK : SLIM_ERR_CUDA;
     note_token_tile(wide ? 256 : 64);
     slim_status_t rc;
-    if (!wide) rc = launch_tile_kernel<64, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
-    else rc = pair ? launch_tile_kernel<256, true>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st)
-                   : launch_tile_kernel<256, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st);
+    const bool dep = r > 0 && p.n1 > 0;               // sparse stages to run while T' is being made
+    if (!wide) rc = launch_tile_kernel<64, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st, 1, dep);
+    else rc = pair ? launch_tile_kernel<256, true>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st, 1, dep)
+                   : launch_tile_kernel<256, false>(p, d_out, tmV, tmM, tmX, tmA2, tmB2, st, 1, dep);
     if (rc != SLIM_OK) return rc;
     // T' and the partial tiles were written where the decode kernels keep their hand-over slots
     // (all ones = empty): leave the region as they expect it.
