@@ -608,12 +608,16 @@ __global__ void pre_reduce_kernel(const float* __restrict__ part, int slices, si
 // Shape of the dense-only launch T' = X R^T: token tile, K slices, stages per slice.  The product
 // has few tiles (r / 128 x tokens / tile), so K is split until they about fill the machine.
 struct PrePlan { int n_tok; int slices; int k_per; };
-static PrePlan pre_plan(int b, int d_in, int r, int sm_count) {
+// `overlapped`: the main launch has sparse stages to run meanwhile.  A short product with few tiles is then
+// better left whole on few SMs -- no partial tiles, no reduction, and the other SMs go to the main launch at
+// once -- than split over the machine (measured: 4096 columns and 32 tiles gain 2-6 %; longer or wider
+// products lose, their T' arrives after the main launch's first CTAs want it).
+static PrePlan pre_plan(int b, int d_in, int r, int sm_count, bool overlapped = false) {
     PrePlan pl;
     pl.n_tok = b >= 192 ? 256 : 64;
     const int tiles = ceil_div(r, kPM) * ceil_div(b, pl.n_tok);
     const int n2 = d_in / kPBK;
-    int ks = sm_count / (tiles > 0 ? tiles : 1);
+    int ks = overlapped && n2 <= 64 && tiles <= sm_count / 4 ? 1 : sm_count / (tiles > 0 ? tiles : 1);
     ks = ks < 1 ? 1 : (ks > 8 ? 8 : ks);
     if (ks > n2) ks = n2 > 0 ? n2 : 1;
     pl.k_per = ceil_div(n2, ks);
@@ -718,7 +722,7 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     if (!ok) return SLIM_ERR_CUDA;
     if (r > 0) {
         // T' = (X R^T) / s : dense phase only, output rows = adapter index
-        const PrePlan pl = pre_plan(b, d_in, r, di->sm_count);
+        const PrePlan pl = pre_plan(b, d_in, r, di->sm_count, s != 0.f);
         ok = pf_map(&tmA2, R, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)r, 64, kPM, 128) &&
              pf_map(&tmXpre, X, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)d_in, (uint64_t)b, 64, pl.n_tok, 128);
         if (!ok) return SLIM_ERR_CUDA;
