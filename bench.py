@@ -450,6 +450,7 @@ def run_ours(args):
                 k["bytes"] += n * algorithmic_bytes(row["d_in"], row["d_out"], row["r"], row["b"])
                 k["us"] += n * row["us"]
                 k["launches"] += n
+        line["roofline"]["dominant_kernel"] = max(by, key=lambda k: by[k]["us"])      # its own figures: by_kernel
         line["roofline"]["by_kernel"] = {
             name: {"launches_per_step": k["launches"], "avg_launch_us": round(k["us"] / k["launches"], 3),
                    "achieved": round(k["bytes"] / k["us"] / 1e3, 1), "frac": round(k["bytes"] / k["us"] / 1e3 / peak, 4),
