@@ -325,3 +325,33 @@ def test_full_size_prefill_configs(d_in, d_out, r, b, seed, wseed):
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     assert res["token_tile"] == (256 if (d_out // 128) * ((b + 255) // 256) >= sms else 64)
     assert_ok(res)
+
+
+def test_prefill_chain_replays_from_a_cuda_graph():
+    """The prefill call's launches depend on one another programmatically (the main launch starts before the
+    dense-only launch has ended): captured in a CUDA graph and replayed, the call gives the same bits."""
+    d_in, d_out, r, b = 1024, 512, 64, 600
+    s, codes, mask, ovals, ometa = cached_weights(d_out, d_in, 91)
+    ly = inputs.make_layer(d_in, d_out, r, b, 91, weights=(s, codes, mask))
+    vals, meta = binding.slim_pack(to_dev(codes), to_dev(mask))
+    X, L, R = binding.bf16_from_bits(ly.X), binding.bf16_from_bits(ly.L), binding.bf16_from_bits(ly.R)
+    ws = binding.new_workspace(b, d_out, d_in, r)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Y = torch.empty((b, d_out), dtype=torch.bfloat16, device="cuda")
+    assert binding.slim_select_kernel(b, d_out, d_in, r) == binding.KERNEL_PREFILL
+    binding.slim_linear_fwd(X, vals, meta, s, L, R, Y=Y, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    direct = Y.clone()
+    stream = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            binding.slim_linear_fwd(X, vals, meta, s, L, R, Y=Y, workspace=ws, status=status)
+        for _ in range(3):
+            Y.zero_()
+            g.replay()
+            stream.synchronize()
+            assert torch.equal(Y.view(torch.int16), direct.view(torch.int16))
+    assert binding.read_status(status) == 0
+    res = parity.compare(inputs.bf16_bits_to_f64(binding.bits_from_bf16(direct)), oracle.linear_fwd(ly.X, ovals, ometa, s, ly.L, ly.R))
+    assert res["ok"], res
