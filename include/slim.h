@@ -352,7 +352,7 @@ int slim_last_launch_count(void);
 /*
  * Token-tile width (64 or 256 tokens) of the prefill kernel the last slim_linear_fwd* call on this host
  * thread launched, 0 if that call ran another kernel.  The prefill kernel has a wide variant for problems
- * that give every SM a 128-row x 256-token tile and a narrow one for the rest; tests use this query to
+ * with enough 128-row x 256-token tiles for a quarter of the SMs or more and a narrow one for the rest; tests use this query to
  * make sure they exercise the variant they mean to.
  */
 int slim_last_token_tile(void);

@@ -706,8 +706,9 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     }
     __nv_bfloat16* Tq = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<char*>(ws) + SLIM_WORKSPACE_SYNC_BYTES);
     const float s_eff = s != 0.f ? s : 1.f;       // with s == 0 only the adapter term remains
-    // token tile: 256 when that still gives every SM a tile, else 64
-    const bool wide = force_pair || (long long)(d_out / kPM) * ceil_div(b, 256) >= di->sm_count;
+    // token tile: 256 when that gives a quarter of the SMs or more a tile, else 64 (measured: with 64 tiles of
+    // 128 x 256 on 148 SMs the wide variant is a third faster than 256 tiles of 128 x 64; with 32 it is slower)
+    const bool wide = force_pair || (long long)(d_out / kPM) * ceil_div(b, 256) * 4 >= (long long)di->sm_count;
     const int n_pre = 64;                         // the T' product has few row tiles: narrow token tiles fill the machine
     // The CTA-pair kernel (prefill_kernel<256, true>) measures no faster than one CTA per tile, so
     // it runs only when asked for by name.
