@@ -710,10 +710,12 @@ slim_status_t launch_prefill(const __nv_bfloat16* X, int b, const uint8_t* vals,
     // 128 x 256 on 148 SMs the wide variant is a third faster than 256 tiles of 128 x 64; with 32 it is slower)
     const bool wide = force_pair || (long long)(d_out / kPM) * ceil_div(b, 256) * 4 >= (long long)di->sm_count;
     const int n_pre = 64;                         // the T' product has few row tiles: narrow token tiles fill the machine
-    // The CTA-pair kernel (prefill_kernel<256, true>) measures no faster than one CTA per tile, so
-    // it runs only when asked for by name.
+    // The CTA-pair kernel (prefill_kernel<256, true>) measures 3-8 % faster than one CTA per tile on
+    // problems with adapters and a thousand tiles or more (the 70B layers at 4096 tokens) and the same or
+    // a little slower below that: it runs for those, or when asked for by name.
     if (force_pair && (d_out / kPM) % 2 != 0) return SLIM_ERR_UNSUPPORTED_SHAPE;
-    const bool pair = force_pair;
+    const bool pair = force_pair || (wide && r > 0 && (d_out / kPM) % 2 == 0 &&
+                                     (long long)(d_out / kPM) * ceil_div(b, 256) >= 1024);
     const int xbox = wide ? (pair ? 128 : 256) : 64;      // token rows one CTA loads per stage = one TMA box
     const int dk = PfCfg<256, false>::kDK;                // columns of a dense stage of the main kernels
     CUtensorMap tmV, tmM, tmX, tmXpre, tmA2, tmB2;
